@@ -1,0 +1,234 @@
+/*
+ * slaq.h - C ABI of the per-epoch scheduling path of a quality-driven scheduler for
+ * ML training jobs (Zhang et al., "SLAQ: Quality-Driven Scheduling for Distributed
+ * Machine Learning", Design section), as CUDA kernels for one sm_100a GPU.
+ *
+ * The problem (Design, "Scheduling Based on Quality Improvements"): J jobs run
+ * concurrently, each reports one loss value per iteration; every epoch of T seconds
+ * the scheduler chooses a_j cores for each job, sum_j a_j <= C, to maximise the total
+ * normalised loss reduction  sum_j [Loss_j(a_j, t) - Loss_j(a_j, t+T)].
+ * One call of slaq_schedule() runs the paper's three duties for every active job:
+ *   - normalise  ("Normalizing Quality Metrics"): change in loss between iterations
+ *     over the largest change seen so far;
+ *   - predict    ("Predicting Quality Improvement"): exponentially weighted least
+ *     squares of f(k) = 1/(a k^2 + b k + c) + d and f(k) = mu^(k-b) + c, the lower
+ *     weighted residual wins, then the loss reduction over one epoch for each core
+ *     count n = 1..max_cores_per_job, an iteration on n cores taking s + w/n seconds;
+ *   - allocate   (the greedy loop of "Scheduling Based on Quality Improvements"): one
+ *     core each, then one core at a time to the largest predicted marginal gain, equal
+ *     gains to the lowest job id.
+ *
+ * Conventions
+ *   - Every function returns an int status: 0 = SLAQ_OK, < 0 error, > 0 warning.
+ *     Nothing throws or aborts.  slaq_last_error() gives a message for the last
+ *     non-zero status of a handle.
+ *   - "host" pointers are ordinary host memory, "device" pointers are memory of the
+ *     GPU that was current when the handle was created.  The caller owns every pointer
+ *     it passes and may release it when the call returns, unless stated otherwise.
+ *   - The handle owns all scheduler state on the device.  Calls on one handle must not
+ *     overlap; work is ordered on the handle's stream (slaq_set_stream).  Functions
+ *     that take or fill host buffers return after the stream has finished that work.
+ *   - Job ids are 0 .. max_jobs-1.  A job is active from its first loss until removed.
+ *   - The library needs a CUDA device: there is no CPU path.
+ */
+#ifndef SLAQ_H
+#define SLAQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct slaq_handle slaq_t;
+
+enum {
+    SLAQ_OK = 0,
+    SLAQ_E_ARG = -1,        /* null pointer, negative count, duplicate job id, bad key or value */
+    SLAQ_E_RANGE = -2,      /* job id outside 0 .. max_jobs-1, or a size beyond what the handle was created for */
+    SLAQ_E_NONFINITE = -3,  /* a loss or time that is NaN or infinite */
+    SLAQ_E_NOMEM = -4,      /* device or host allocation failed, or the given workspace is too small */
+    SLAQ_E_CUDA = -5,       /* a CUDA call failed; the message holds its error string */
+    SLAQ_E_TIMEOUT = -6,    /* a bounded device-side wait ran out */
+    SLAQ_W_OVERSUBSCRIBED = 1, /* fewer cores than active jobs: no one-core floor, cores go to the best first units */
+    SLAQ_W_UNDERFILLED = 2     /* more cores than active jobs x max_cores_per_job: every job is at its cap */
+};
+
+/* keys of slaq_set_param / slaq_get_param */
+enum {
+    SLAQ_P_GAMMA = 1,             /* weight base of the fit, point i of H weighs gamma^(H-1-i); default 0.9; (0, 1] */
+    SLAQ_P_LM_TRIALS = 2,         /* Levenberg-Marquardt trials per family; default 20; 0 .. 1000 */
+    SLAQ_P_MAX_CORES_PER_JOB = 3, /* cap on a_j; default 64; 1 .. what the handle was created for */
+    SLAQ_P_MIN_FIT_POINTS = 4     /* fewer stored points than this use linear extrapolation; default 4; >= 4 */
+};
+
+/* per-job status written by slaq_schedule (slaq_get_predictions, out_status) */
+enum {
+    SLAQ_JOB_INACTIVE = -1,  /* no loss reported */
+    SLAQ_JOB_FITTED = 0,     /* a curve family was fitted */
+    SLAQ_JOB_SHORT = 1,      /* two or three points: linear extrapolation of the normalised reduction */
+    SLAQ_JOB_NEW = 2,        /* one point: normalised loss 1, one unit per iteration */
+    SLAQ_JOB_FIT_FAILED = 3, /* both families failed numerically: linear extrapolation */
+    SLAQ_JOB_FLAT = 4,       /* the loss never fell: no predicted gain */
+    SLAQ_JOB_NONFINITE = 5,  /* a stored value is not finite: no predicted gain */
+    SLAQ_JOB_NO_TIME = 6     /* no iteration-time model yet: no predicted gain */
+};
+
+/* Timings and counts of the last slaq_schedule / slaq_schedule_device call. */
+typedef struct slaq_stats {
+    float ms_total;        /* device time of the whole epoch */
+    float ms_fit;          /* normalise + fit kernel */
+    float ms_gain;         /* marginal-gain kernel (with the first selection histogram) */
+    float ms_alloc;        /* threshold selection, per-job counts, allocation */
+    int32_t launches;      /* kernels launched by the call */
+    int32_t active_jobs;
+    int64_t cores_handed_out;
+    int64_t points;        /* loss values read by the fit kernel */
+    int64_t model_sweeps;  /* sum over fitted jobs and families of (history length x sweeps over it) */
+    int64_t tie_units;     /* units taken at exactly the threshold gain */
+    double threshold;      /* smallest gain that received a core beyond the floor (0 if none) */
+    int32_t fitted_jobs;
+    int32_t sublinear_wins;
+    int32_t exponential_wins;
+    int32_t fallback_jobs;
+} slaq_stats;
+
+/*
+ * Create a scheduler for job ids 0..max_jobs-1, each keeping a window of its newest
+ * max_hist losses (4 <= max_hist <= 6000) - the "history loss values" the fit uses.
+ * Allocates all device state with cudaMalloc on the current device:
+ * slaq_workspace_bytes(max_jobs, max_hist, 64) bytes; up to 64 cores per job.
+ * *out receives the handle.  Errors: SLAQ_E_ARG, SLAQ_E_NOMEM, SLAQ_E_CUDA.
+ */
+int slaq_create(int32_t max_jobs, int32_t max_hist, slaq_t** out);
+
+/*
+ * Same with an explicit cap on cores per job (1..1024).  dev_ws == NULL: the library
+ * allocates.  Otherwise the state lives inside device memory the caller owns (for
+ * instance a torch tensor): dev_ws must be 256-byte aligned, hold at least
+ * slaq_workspace_bytes(max_jobs, max_hist, max_cores_per_job) bytes and outlive the
+ * handle.  The library never frees it.
+ */
+int slaq_create_in(void* dev_ws, size_t bytes, int32_t max_jobs, int32_t max_hist, int32_t max_cores_per_job,
+                   slaq_t** out);
+size_t slaq_workspace_bytes(int32_t max_jobs, int32_t max_hist, int32_t max_cores_per_job);
+
+/* Release the handle and the device memory it allocated itself.  NULL is accepted. */
+int slaq_destroy(slaq_t* h);
+
+/* Message for the last non-zero status of h (handle-owned storage; valid until the next call on h). */
+const char* slaq_last_error(const slaq_t* h);
+
+/* cuda_stream is a cudaStream_t (NULL = default stream).  All later work of h runs on it. */
+int slaq_set_stream(slaq_t* h, void* cuda_stream);
+
+int slaq_set_param(slaq_t* h, int key, double value);
+int slaq_get_param(const slaq_t* h, int key, double* out_value);
+
+/*
+ * One new iteration for each listed job: losses[i] is the loss job_ids[i] reports,
+ * iter_times[i] the wall seconds that iteration took.  A job id may appear at most once
+ * per call.  The first loss activates the job (iteration index 0).  The call updates the
+ * job's window (the oldest point is dropped once max_hist are stored), its iteration
+ * index, the largest reduction l_{k-1} - l_k it has shown so far ("the largest change we
+ * have seen so far", "Normalizing Quality Metrics"), and the sums of its iteration-time
+ * law t(n) = s + w/n, the iteration being booked at the job's current core count: its
+ * allocation from the last slaq_schedule, 1 before any.  iter_times may be NULL (no time
+ * sample).  All pointers are host pointers, n entries each.
+ * Errors: SLAQ_E_ARG (n < 0, null, duplicate id), SLAQ_E_RANGE, SLAQ_E_NONFINITE
+ * (nothing is applied when an error is returned).
+ */
+int slaq_append_losses(slaq_t* h, int32_t n, const int32_t* job_ids, const double* losses,
+                       const double* iter_times);
+/* Same with the core count of each sample given explicitly (cores_used[i] >= 1). */
+int slaq_append_losses_ex(slaq_t* h, int32_t n, const int32_t* job_ids, const double* losses,
+                          const double* iter_times, const int32_t* cores_used);
+
+/*
+ * Bulk load: replace the stored window of n_jobs jobs.  Histories are ragged, in CSR
+ * form: job job_ids[i] owns losses[offsets[i] .. offsets[i+1]), oldest first; k_last[i]
+ * is the iteration index of its newest loss; m_seen[i] (array may be NULL) the largest
+ * one-step reduction of its earlier life, joined at scheduling time with the window's
+ * own.  If a history is longer than max_hist only its newest max_hist points are kept.
+ * Time sums and time models are left as they are.  Host pointers.
+ * slaq_load_histories stores each job in its own max_hist-long ring, so later appends
+ * extend the window up to max_hist.  slaq_load_histories_packed keeps the rows packed
+ * back to back on the device exactly as given (one cudaMalloc of the total size, which
+ * replaces any earlier packed load - jobs of an earlier packed load must be reloaded or
+ * removed first): a job loaded this way keeps a window of the length it was loaded with,
+ * later appends overwrite its oldest point.
+ * Errors: SLAQ_E_ARG, SLAQ_E_RANGE, SLAQ_E_NONFINITE, SLAQ_E_NOMEM, SLAQ_E_CUDA.
+ */
+int slaq_load_histories(slaq_t* h, int32_t n_jobs, const int32_t* job_ids, const int64_t* offsets,
+                        const double* losses, const int64_t* k_last, const double* m_seen);
+int slaq_load_histories_packed(slaq_t* h, int32_t n_jobs, const int32_t* job_ids, const int64_t* offsets,
+                               const double* losses, const int64_t* k_last, const double* m_seen);
+
+/*
+ * Fix the iteration-time law t(n) = s[i] + w[i]/n of the listed jobs (s >= 0 seconds,
+ * w > 0 core-seconds), overriding the estimate from iter_times.  The paper leaves the
+ * map from cores to progress open ("predict how much progress the job would achieve if
+ * it was granted a certain amount of resources"); this law is the library's.  Host pointers.
+ */
+int slaq_set_time_model(slaq_t* h, int32_t n, const int32_t* job_ids, const double* s, const double* w);
+
+/* Deactivate jobs and forget their state.  Host pointer. */
+int slaq_remove_jobs(slaq_t* h, int32_t n, const int32_t* job_ids);
+
+/*
+ * One scheduling epoch (Design: normalise, predict, allocate): epoch_seconds = T,
+ * total_cores = C.  out_alloc (host, max_jobs entries) receives a_j: 0 for inactive
+ * ids, otherwise 1..max_cores_per_job with sum = min(C, active x max_cores_per_job)
+ * (0..max when C < active jobs).  Stored histories are not modified: the call can be
+ * repeated.  The allocation is remembered as each job's current core count.
+ * Returns SLAQ_OK, SLAQ_W_OVERSUBSCRIBED, SLAQ_W_UNDERFILLED, or an error
+ * (SLAQ_E_ARG for T <= 0, C < 0 or null; SLAQ_E_CUDA).
+ */
+int slaq_schedule(slaq_t* h, double epoch_seconds, int64_t total_cores, int32_t* out_alloc);
+/* Same, asynchronous on the handle's stream; d_out_alloc is a device pointer or NULL (result kept in the handle). */
+int slaq_schedule_device(slaq_t* h, double epoch_seconds, int64_t total_cores, int32_t* d_out_alloc);
+
+/*
+ * Results of the last epoch, host pointers, any may be NULL; sizes in entries:
+ * out_reduction [max_jobs]: predicted normalised loss reduction at the allocation,
+ * Loss_j(a_j, t) - Loss_j(a_j, t+T) in units of the largest reduction seen;
+ * out_gain [max_jobs x max_cores_per_job], row-major, gain of the n-th core at [j][n-1];
+ * out_family [max_jobs]: 0 = 1/(a x^2 + b x + c) + d, 1 = exp(alpha - beta x) + c, -1 none;
+ * out_params [max_jobs x 4]: (a, b, c, d) or (alpha, beta, c, 0) in window coordinates
+ * (x = 0 at the newest point, -1 at the oldest, y = loss / out_largest);
+ * out_residual [max_jobs x 2]: final weighted residual of each family;
+ * out_status [max_jobs]: SLAQ_JOB_*; out_sweeps [max_jobs x 2]: sweeps over the history
+ * spent on each family; out_largest [max_jobs]: largest reduction seen.
+ */
+int slaq_get_predictions(slaq_t* h, double* out_reduction, double* out_gain, int8_t* out_family,
+                         double* out_params, double* out_residual, int32_t* out_status, int32_t* out_sweeps,
+                         double* out_largest);
+
+/*
+ * Normalisation alone, for inspection: for each listed job, oldest first and packed
+ * back to back in the order given, the normalised changes (l_{i-1} - l_i) / M (0 for a
+ * job's first stored point) and the normalised levels l_i / M; out_offsets [n+1] receives
+ * where each job's values start, out_largest [n] the M used.  capacity = entries available
+ * in out_changes / out_levels (SLAQ_E_RANGE if too small).  Host pointers; any output may be NULL.
+ */
+int slaq_get_normalised(slaq_t* h, int32_t n, const int32_t* job_ids, int64_t capacity, int64_t* out_offsets,
+                        double* out_changes, double* out_levels, double* out_largest);
+
+/* Iteration-time law in use for every job (NaN where none yet).  Host pointers [max_jobs]. */
+int slaq_get_time_model(slaq_t* h, double* out_s, double* out_w);
+
+/*
+ * Test hook for the allocation step alone: overwrite the gain rows (host,
+ * max_jobs x max_cores_per_job, rows non-increasing, values >= +0) and allocate from
+ * them with slaq_allocate_only, which runs only the greedy-equivalent selection.
+ */
+int slaq_set_gains(slaq_t* h, const double* gain);
+int slaq_allocate_only(slaq_t* h, int64_t total_cores, int32_t* out_alloc);
+
+int slaq_get_stats(slaq_t* h, slaq_stats* out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLAQ_H */

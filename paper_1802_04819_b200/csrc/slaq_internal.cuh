@@ -1,0 +1,123 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "slaq.h"
+
+namespace slaq {
+
+constexpr int kMaxHistLimit = 6000;   // one warp stages a whole window in shared memory
+constexpr int kMaxCoresLimit = 1024;
+constexpr int kRadixBits = 11;
+constexpr int kRadixBins = 1 << kRadixBits;
+constexpr int kRadixPasses = 6;       // 11 + 11 + 11 + 11 + 11 + 9 bits, most significant first
+
+// Device-side state of one job, structure of arrays (index = job id).
+struct JobArrays {
+    double** row;        // start of the job's window storage (ring of `cap` slots)
+    int32_t* cap;        // slots in the ring
+    int32_t* head;       // slot the next loss goes to
+    int32_t* count;      // stored losses, 0 = inactive
+    int64_t* k_last;     // iteration index of the newest loss
+    double* m_seen;      // largest one-step reduction seen so far (-inf: none)
+    double* tm;          // [8][max_jobs]: count, sum u, sum u^2, sum t, sum u t, sum t n, min u, max u (u = 1/cores)
+    double* s_set;       // fixed time law (NaN: use the estimate)
+    double* w_set;
+    int32_t* last_alloc; // core count of the last epoch (1 before any)
+};
+
+// What the fit leaves for the later stages, one entry per job.
+struct FitArrays {
+    int32_t* status;     // SLAQ_JOB_*
+    int8_t* family;      // 0, 1 or -1
+    double* params;      // [max_jobs][4]; linear-extrapolation kinds keep (rho, r_cap) in slots 0, 1
+    double* residual;    // [max_jobs][2]
+    int32_t* sweeps;     // [max_jobs][2]
+    double* largest;     // M
+    double* span;        // max(H-1, 1)
+};
+
+// Running state of the radix select.
+struct SelectState {
+    unsigned long long prefix;       // bits of the threshold key found so far
+    long long want;                  // units still to take inside the current candidate set
+    int done;                        // nothing is wanted: the threshold lies above every gain
+};
+
+// Scratch of one epoch; [hist, hist + zero_bytes) is cleared at the start of every epoch.
+struct Scratch {
+    unsigned long long* hist;        // [kRadixPasses][kRadixBins]
+    unsigned int* ticket;            // [8]: job queue head, then one block-completion counter per pass
+    SelectState* sel;
+    long long* counters;             // [16] statistics accumulated by kernels
+    size_t zero_bytes;
+    int32_t* gt;                     // per job: candidate gains strictly above the threshold
+    int32_t* eq;                     // per job: candidate gains equal to it
+    long long* block_eq;             // per block of the count kernel: sum of eq
+    int32_t* order;                  // job ids, longest history first (fit kernel work list)
+    int32_t* bucket;                 // counting-sort buckets by history length
+};
+
+struct Staging {
+    int32_t* ids;
+    double* losses;
+    double* times;
+    int32_t* cores;
+    int64_t* offsets;
+    int64_t* k_last;
+    double* m_seen;
+};
+
+}  // namespace slaq
+
+struct slaq_handle {
+    int device = 0;
+    int32_t max_jobs = 0, max_hist = 0, cap_alloc = 0;   // cap_alloc: gain columns the buffers were sized for
+    int32_t max_cores = 64;
+    double gamma = 0.9;
+    int32_t lm_trials = 20, min_fit_points = 4;
+    cudaStream_t stream = nullptr;
+    bool owns_ws = false;
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    double* ring_pool = nullptr;      // [max_jobs][max_hist]
+    double* packed_pool = nullptr;    // separate allocation made by slaq_load_histories_packed
+    size_t packed_len = 0;
+    double* wtab = nullptr;           // gamma^m, m = 0..max_hist-1
+    double wtab_gamma = -1.0;
+    slaq::JobArrays job;
+    slaq::FitArrays fit;
+    slaq::Scratch scratch;
+    slaq::Staging stage;
+    double* gain = nullptr;           // [max_jobs][max_cores]
+    int32_t* alloc = nullptr;
+    double* reduction = nullptr;
+    int32_t* err_word = nullptr;      // device error flags set by kernels
+    cudaEvent_t ev[4] = {};
+    bool have_epoch = false;
+    int32_t last_launches = 0;
+    int64_t last_cores = 0;
+    int sm_count = 148;
+    std::vector<uint8_t> active;      // host mirror: job has at least one loss
+    std::vector<uint32_t> stamp;      // host: duplicate detection
+    uint32_t stamp_epoch = 0;
+    int32_t n_active = 0;
+    std::string err;
+};
+
+namespace slaq {
+
+// kernel launchers: each returns the number of kernels it launched, or -1 after setting h->err
+int launch_fit(slaq_handle* h);
+int launch_gain(slaq_handle* h, double epoch_seconds, int first_unit);
+int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_ready, int32_t* d_out_alloc);
+int launch_normalise_export(slaq_handle* h, int32_t n, const int64_t* d_offsets, double* d_changes,
+                            double* d_levels, double* d_largest);
+int launch_time_model(slaq_handle* h, double* d_s, double* d_w);
+
+}  // namespace slaq
