@@ -1,0 +1,315 @@
+// Allocation: the greedy loop of "Scheduling Based on Quality Improvements" as a global
+// top-C selection.
+//
+// The paper starts every job at one core and then gives one core at a time to the job
+// whose next core has the largest predicted gain.  Gain rows are non-increasing in n, so
+// that loop hands out exactly the `want` largest gains beyond the floor, and among equal
+// gains it serves (job id ascending, n ascending).  Here: a most-significant-digit-first
+// radix select over the 64-bit patterns of the gains (all >= +0, so the IEEE pattern
+// orders like the value) finds the threshold tau and how many gains equal to tau are
+// still wanted; then per job  a_j = floor + #{g > tau} + clamp(wanted - P_j, 0, #{g = tau})
+// with P_j the number of gains equal to tau in jobs with a lower id.
+#include <math_constants.h>
+
+#include "slaq_internal.cuh"
+
+namespace slaq {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kSelectThreads = 256;
+constexpr int kJobsPerBlock = 256;   // count / finalise kernels: 8 warps x 32 jobs
+
+__host__ __device__ inline int pass_shift(int pass) {
+    return pass < kRadixPasses - 1 ? 64 - kRadixBits * (pass + 1) : 0;
+}
+__host__ __device__ inline int pass_bits(int pass) {
+    return pass < kRadixPasses - 1 ? kRadixBits : 64 - kRadixBits * (kRadixPasses - 1);
+}
+
+// After the histogram of `pass` is complete: walk the bins from the top until `want`
+// units are covered, extend the threshold prefix by that bin and keep what is still
+// wanted inside it.  Called by every thread of one block of kSelectThreads threads;
+// sh holds kSelectThreads + 1 entries.
+__device__ void pick_bin(const unsigned long long* hist, int pass, SelectState* sel, unsigned long long* sh) {
+    const int t = threadIdx.x;
+    const int nbins = 1 << pass_bits(pass);
+    const int per = (kRadixBins + kSelectThreads - 1) / kSelectThreads;   // bins per thread, from the top down
+    unsigned long long mine = 0;
+    for (int k = 0; k < per; ++k) {
+        const int b = nbins - 1 - (t * per + k);
+        if (b >= 0) mine += __ldcg(&hist[b]);
+    }
+    sh[t] = mine;
+    __syncthreads();
+    if (t == 0) {   // exclusive prefix over threads
+        unsigned long long run = 0;
+        for (int i = 0; i < kSelectThreads; ++i) {
+            const unsigned long long v = sh[i];
+            sh[i] = run;
+            run += v;
+        }
+        sh[kSelectThreads] = run;
+    }
+    __syncthreads();
+    const long long want = sel->want;
+    const bool done = sel->done != 0;
+    __syncthreads();
+    if (done) return;
+    unsigned long long above = sh[t];
+    for (int k = 0; k < per; ++k) {
+        const int b = nbins - 1 - (t * per + k);
+        if (b < 0) break;
+        const unsigned long long c = __ldcg(&hist[b]);
+        if (above < (unsigned long long)want && (unsigned long long)want <= above + c) {
+            sel->prefix |= (unsigned long long)b << pass_shift(pass);   // exactly one thread gets here
+            sel->want = want - (long long)above;
+        }
+        above += c;
+    }
+}
+
+// Histogram of one digit over the candidates that match the prefix found so far; the
+// last block to finish picks the bin.
+__global__ void __launch_bounds__(kSelectThreads)
+select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap,
+                   int first_unit, int pass, unsigned long long* __restrict__ hist_all, SelectState* sel,
+                   unsigned int* ticket) {
+    __shared__ unsigned int sh_hist[kRadixBins];
+    __shared__ unsigned long long sh_scan[kSelectThreads + 1];
+    __shared__ bool is_last;
+    unsigned long long* hist = hist_all + (size_t)pass * kRadixBins;
+    if (sel->done) return;   // uniform over the grid: nothing is wanted
+    for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) sh_hist[i] = 0;
+    __syncthreads();
+    const unsigned long long prefix = sel->prefix;
+    const int shift = pass_shift(pass), bits = pass_bits(pass);
+    const int hi_shift = shift + bits;                     // bits from here up are already fixed
+    const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(gain);
+    const int lane = threadIdx.x & 31;
+    const int warps_total = gridDim.x * (kSelectThreads / 32);
+    for (int j = blockIdx.x * (kSelectThreads / 32) + (threadIdx.x >> 5); j < max_jobs; j += warps_total) {
+        if (count[j] <= 0) continue;
+        for (int n = first_unit + lane; n <= cap; n += 32) {
+            const unsigned long long key = keys[(size_t)j * cap + (n - 1)];
+            if ((key >> hi_shift) == (prefix >> hi_shift))
+                atomicAdd(&sh_hist[(unsigned)(key >> shift) & ((1u << bits) - 1u)], 1u);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) {
+        const unsigned v = sh_hist[i];
+        if (v) atomicAdd(&hist[i], (unsigned long long)v);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(&ticket[1 + pass], 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (is_last) {
+        __threadfence();
+        pick_bin(hist, pass, sel, sh_scan);
+    }
+}
+
+// The first histogram is complete when this starts (it was filled by an earlier kernel).
+__global__ void __launch_bounds__(kSelectThreads) pick_first_kernel(unsigned long long* hist_all, SelectState* sel) {
+    __shared__ unsigned long long sh_scan[kSelectThreads + 1];
+    pick_bin(hist_all, 0, sel, sh_scan);
+}
+
+__global__ void init_select_kernel(SelectState* sel, long long want) {
+    sel->prefix = want > 0 ? 0ull : ~0ull;   // nothing wanted: a threshold above every gain
+    sel->want = want > 0 ? want : 0;
+    sel->done = want > 0 ? 0 : 1;
+}
+
+// Histogram of the first digit when the gain rows were not written by the gain kernel.
+__global__ void __launch_bounds__(kSelectThreads)
+first_hist_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap,
+                  int first_unit, unsigned long long* __restrict__ hist0) {
+    __shared__ unsigned int sh_hist[kRadixBins];
+    for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) sh_hist[i] = 0;
+    __syncthreads();
+    const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(gain);
+    const int lane = threadIdx.x & 31;
+    const int warps_total = gridDim.x * (kSelectThreads / 32);
+    for (int j = blockIdx.x * (kSelectThreads / 32) + (threadIdx.x >> 5); j < max_jobs; j += warps_total) {
+        if (count[j] <= 0) continue;
+        for (int n = first_unit + lane; n <= cap; n += 32)
+            atomicAdd(&sh_hist[(unsigned)(keys[(size_t)j * cap + (n - 1)] >> (64 - kRadixBits))], 1u);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) {
+        const unsigned v = sh_hist[i];
+        if (v) atomicAdd(&hist0[i], (unsigned long long)v);
+    }
+}
+
+// Per job: how many candidate gains lie above the threshold and how many equal it.
+__global__ void __launch_bounds__(256)
+count_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap, int first_unit,
+             const SelectState* __restrict__ sel, int32_t* __restrict__ gt, int32_t* __restrict__ eq,
+             long long* __restrict__ block_eq) {
+    __shared__ int sh_eq[8];
+    const unsigned long long tau = sel->prefix;
+    const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(gain);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int eq_sum = 0;
+    for (int i = 0; i < 32; ++i) {
+        const int j = blockIdx.x * kJobsPerBlock + warp * 32 + i;
+        if (j >= max_jobs) break;
+        int n_gt = 0, n_eq = 0;
+        if (count[j] > 0) {
+            for (int base = first_unit; base <= cap; base += 32) {
+                const int n = base + lane;
+                unsigned long long key = 0;
+                const bool in = n <= cap;
+                if (in) key = keys[(size_t)j * cap + (n - 1)];
+                n_gt += __popc(__ballot_sync(kFull, in && key > tau));
+                n_eq += __popc(__ballot_sync(kFull, in && key == tau));
+            }
+        }
+        if (lane == 0) {
+            gt[j] = n_gt;
+            eq[j] = n_eq;
+        }
+        eq_sum += n_eq;
+    }
+    if (lane == 0) sh_eq[warp] = eq_sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long total = 0;
+        for (int w = 0; w < 8; ++w) total += sh_eq[w];
+        block_eq[blockIdx.x] = total;
+    }
+}
+
+// Exclusive prefix sum of block_eq[0..n), one block of 1024 threads.
+__global__ void __launch_bounds__(1024) scan_blocks_kernel(long long* block_eq, int n) {
+    __shared__ long long sh[1024];
+    const int t = threadIdx.x;
+    const int per = (n + 1023) / 1024;
+    const int lo = min(t * per, n), hi = min(lo + per, n);
+    long long sum = 0;
+    for (int i = lo; i < hi; ++i) sum += block_eq[i];
+    sh[t] = sum;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {   // inclusive scan
+        const long long v = t >= o ? sh[t - o] : 0;
+        __syncthreads();
+        sh[t] += v;
+        __syncthreads();
+    }
+    long long run = sh[t] - sum;
+    for (int i = lo; i < hi; ++i) {
+        const long long v = block_eq[i];
+        block_eq[i] = run;
+        run += v;
+    }
+}
+
+// a_j from the counts, the predicted reduction at a_j, and the allocation becomes the job's core count.
+__global__ void __launch_bounds__(256)
+finalise_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap, int floor_units,
+                const SelectState* __restrict__ sel, const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
+                const long long* __restrict__ block_prefix, int32_t* __restrict__ alloc, double* __restrict__ reduction,
+                int32_t* __restrict__ last_alloc, int32_t* __restrict__ out_alloc, long long* counters) {
+    __shared__ long long sh_pre[kJobsPerBlock];
+    __shared__ int sh_alloc[kJobsPerBlock];
+    const int t = threadIdx.x;
+    const int j0 = blockIdx.x * kJobsPerBlock;
+    const int jt = j0 + t;
+    const int my_eq = jt < max_jobs ? eq[jt] : 0;
+    sh_pre[t] = my_eq;
+    __syncthreads();
+    for (int o = 1; o < kJobsPerBlock; o <<= 1) {
+        const long long v = t >= o ? sh_pre[t - o] : 0;
+        __syncthreads();
+        sh_pre[t] += v;
+        __syncthreads();
+    }
+    const long long before = block_prefix[blockIdx.x] + sh_pre[t] - my_eq;   // ties in jobs with a lower id
+    int a = 0;
+    long long ties_taken = 0;
+    if (jt < max_jobs && count[jt] > 0) {
+        long long take = sel->want - before;
+        take = take < 0 ? 0 : (take > my_eq ? my_eq : take);
+        a = floor_units + gt[jt] + (int)take;
+        ties_taken = take;
+    }
+    sh_alloc[t] = a;
+    if (jt < max_jobs) {
+        alloc[jt] = a;
+        if (out_alloc) out_alloc[jt] = a;
+        if (count[jt] > 0) last_alloc[jt] = a;
+    }
+    // block totals for the statistics: cores handed out and ties taken, both at most 1024 per job
+    __syncthreads();
+    sh_pre[t] = ((long long)a << 20) | ties_taken;
+    __syncthreads();
+    for (int o = kJobsPerBlock / 2; o > 0; o >>= 1) {
+        if (t < o) sh_pre[t] += sh_pre[t + o];
+        __syncthreads();
+    }
+    if (t == 0) {
+        atomicAdd((unsigned long long*)&counters[6], (unsigned long long)(sh_pre[0] >> 20));
+        atomicAdd((unsigned long long*)&counters[7], (unsigned long long)(sh_pre[0] & ((1ll << 20) - 1)));
+    }
+    // predicted reduction at the allocation: the job's first a_j gains, one warp per job
+    const int warp = t >> 5, lane = t & 31;
+    for (int i = 0; i < 32; ++i) {
+        const int local = warp * 32 + i;
+        const int j = j0 + local;
+        if (j >= max_jobs) break;
+        const int aj = sh_alloc[local];
+        double R = 0.0;
+        for (int n = lane; n < aj; n += 32) R += gain[(size_t)j * cap + n];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) R += __shfl_xor_sync(kFull, R, o);
+        if (lane == 0) reduction[j] = R;
+    }
+}
+
+}  // namespace
+
+// Selection + counts + allocation on the gain rows held by the handle.  `want` = units to
+// hand out beyond the floor among gains n >= first_unit.  hist0_ready: the first histogram
+// was already accumulated (by the gain kernel).
+int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_ready, int32_t* d_out_alloc) {
+    int launches = 0;
+    const int J = h->max_jobs, cap = h->max_cores;
+    cudaStream_t st = h->stream;
+    int grid = h->sm_count * 8;
+    const int needed = (J + (kSelectThreads / 32) - 1) / (kSelectThreads / 32);
+    if (grid > needed) grid = needed;
+    init_select_kernel<<<1, 1, 0, st>>>(h->scratch.sel, want);
+    ++launches;
+    if (!hist0_ready) {
+        first_hist_kernel<<<grid, kSelectThreads, 0, st>>>(h->gain, h->job.count, J, cap, first_unit, h->scratch.hist);
+        ++launches;
+    }
+    pick_first_kernel<<<1, kSelectThreads, 0, st>>>(h->scratch.hist, h->scratch.sel);
+    ++launches;
+    for (int pass = 1; pass < kRadixPasses; ++pass) {
+        select_pass_kernel<<<grid, kSelectThreads, 0, st>>>(h->gain, h->job.count, J, cap, first_unit, pass,
+                                                           h->scratch.hist, h->scratch.sel, h->scratch.ticket);
+        ++launches;
+    }
+    const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
+    count_kernel<<<blocks, 256, 0, st>>>(h->gain, h->job.count, J, cap, first_unit, h->scratch.sel, h->scratch.gt,
+                                         h->scratch.eq, h->scratch.block_eq);
+    scan_blocks_kernel<<<1, 1024, 0, st>>>(h->scratch.block_eq, blocks);
+    finalise_kernel<<<blocks, 256, 0, st>>>(h->gain, h->job.count, J, cap, first_unit - 1, h->scratch.sel, h->scratch.gt,
+                                            h->scratch.eq, h->scratch.block_eq, h->alloc, h->reduction,
+                                            h->job.last_alloc, d_out_alloc, h->scratch.counters);
+    launches += 3;
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        h->err = std::string("allocation kernels launch: ") + cudaGetErrorString(e);
+        return -1;
+    }
+    return launches;
+}
+
+}  // namespace slaq

@@ -1,0 +1,190 @@
+// Marginal gains: expand every job's fitted curve into the predicted loss reduction of its
+// n-th core, n = 1..max_cores_per_job (the objective Loss_j(a_j, t) - Loss_j(a_j, t+T) of
+// "Scheduling Based on Quality Improvements", differenced in a_j).
+//
+// An iteration on n cores takes t(n) = s + w/n seconds, so an epoch of T seconds runs
+// m(n) = T n / (s n + w) iterations; in window coordinates that is X_n = m(n) / span ahead
+// of the newest point, and R(n) = f(0) - f(X_n).  g(n) = R(n) - R(n-1) is evaluated without
+// cancellation, clamped to +0 where it is not a positive finite number, and made
+// non-increasing in n by a running minimum.  One warp per job; the row is written once,
+// coalesced, and its keys feed the first histogram of the threshold selection.
+#include <math_constants.h>
+
+#include "slaq_internal.cuh"
+
+namespace slaq {
+
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ bool finite_d(double v) { return fabs(v) <= 1.7976931348623157e308; }
+
+// Iteration-time law of job j: the fixed one if set, else ordinary least squares of the
+// sampled seconds on u = 1/cores from the running sums.  s and w are left untouched if the
+// job has neither; returns whether the law can be used (s >= 0, w > 0, finite).
+__device__ bool time_law(const JobArrays& job, int j, int max_jobs, double& s, double& w) {
+    const double s_fix = job.s_set[j], w_fix = job.w_set[j];
+    if (finite_d(s_fix) && finite_d(w_fix)) {
+        s = s_fix;
+        w = w_fix;
+    } else {
+        const double* tm = job.tm + j;
+        const size_t J = (size_t)max_jobs;
+        const double cnt = tm[0], su = tm[J], suu = tm[2 * J], st = tm[3 * J], sut = tm[4 * J], stn = tm[5 * J];
+        const double umin = tm[6 * J], umax = tm[7 * J];
+        if (!(cnt > 0.0)) return false;
+        bool fitted = false;
+        if (umax > umin) {
+            const double den = __dsub_rn(__dmul_rn(cnt, suu), __dmul_rn(su, su));
+            const double ww = __ddiv_rn(__dsub_rn(__dmul_rn(cnt, sut), __dmul_rn(su, st)), den);
+            const double ss = __ddiv_rn(__dsub_rn(st, __dmul_rn(ww, su)), cnt);
+            if (den > 0.0 && finite_d(ww) && finite_d(ss) && ss >= 0.0 && ww > 0.0) {
+                s = ss;
+                w = ww;
+                fitted = true;
+            }
+        }
+        if (!fitted) {   // one core count only, or an unphysical fit: all time is parallel work
+            s = 0.0;
+            w = __ddiv_rn(stn, cnt);
+        }
+    }
+    return finite_d(s) && finite_d(w) && w > 0.0 && s >= 0.0;
+}
+
+struct Curve {
+    int kind;        // 0 family I, 1 family II, 2 linear extrapolation, 3 no gain
+    double p0, p1, p2;
+    double span, s, w, T;
+};
+
+// after an epoch on n cores: s n + w, iterations completed, and the same in window coordinates
+__device__ __forceinline__ void ahead(const Curve& c, int n, double& X, double& den, double& m) {
+    den = __dadd_rn(__dmul_rn(c.s, (double)n), c.w);
+    m = __ddiv_rn(__dmul_rn(c.T, (double)n), den);
+    X = __ddiv_rn(m, c.span);
+}
+
+__device__ double raw_gain(const Curve& c, int n) {
+    double X, den, m, Xp = 0.0, denp = c.w, mp = 0.0;
+    ahead(c, n, X, den, m);
+    if (n > 1) ahead(c, n - 1, Xp, denp, mp);
+    double gain;
+    if (c.kind == 0) {
+        // 1/q(Xp) - 1/q(X) = (q(X) - q(Xp)) / (q(X) q(Xp)), q(X) - q(Xp) = (X - Xp)(a (X + Xp) + b)
+        const double dX = __ddiv_rn(__dmul_rn(c.T, c.w), __dmul_rn(__dmul_rn(c.span, den), denp));
+        const double q_now = __dadd_rn(__dadd_rn(__dmul_rn(__dmul_rn(c.p0, X), X), __dmul_rn(c.p1, X)), c.p2);
+        const double q_prev = __dadd_rn(__dadd_rn(__dmul_rn(__dmul_rn(c.p0, Xp), Xp), __dmul_rn(c.p1, Xp)), c.p2);
+        const double dq = __dmul_rn(dX, __dadd_rn(__dmul_rn(c.p0, __dadd_rn(X, Xp)), c.p1));
+        gain = __ddiv_rn(dq, __dmul_rn(q_now, q_prev));
+    } else if (c.kind == 1) {
+        // e^(alpha - beta Xp) - e^(alpha - beta X) = e^(alpha - beta Xp) (1 - e^(-beta (X - Xp)))
+        const double dX = __ddiv_rn(__dmul_rn(c.T, c.w), __dmul_rn(__dmul_rn(c.span, den), denp));
+        gain = exp(__dsub_rn(c.p0, __dmul_rn(c.p1, Xp))) * (-expm1(-__dmul_rn(c.p1, dX)));
+    } else {
+        const double R = fmin(__dmul_rn(c.p0, m), c.p1);
+        const double Rp = n > 1 ? fmin(__dmul_rn(c.p0, mp), c.p1) : 0.0;
+        gain = __dsub_rn(R, Rp);
+    }
+    return (finite_d(gain) && gain > 0.0) ? gain : 0.0;
+}
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int first_unit, double* __restrict__ gain,
+            unsigned long long* __restrict__ hist0) {
+    __shared__ unsigned int sh_hist[kRadixBins];
+    for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) sh_hist[i] = 0;
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warps_total = gridDim.x * kWarpsPerBlock;
+    for (int j = blockIdx.x * kWarpsPerBlock + warp; j < max_jobs; j += warps_total) {
+        int status = fit.status[j];
+        const bool active = job.count[j] > 0;
+        Curve c;
+        c.kind = 3;
+        c.T = T;
+        c.span = fit.span[j];
+        c.s = c.w = c.p0 = c.p1 = c.p2 = 0.0;
+        const bool predicts = status == SLAQ_JOB_FITTED || status == SLAQ_JOB_SHORT || status == SLAQ_JOB_NEW ||
+                              status == SLAQ_JOB_FIT_FAILED;
+        if (active && status != SLAQ_JOB_NONFINITE && status != SLAQ_JOB_FLAT) {
+            if (!time_law(job, j, max_jobs, c.s, c.w)) {
+                status = SLAQ_JOB_NO_TIME;
+                if (lane == 0) fit.status[j] = status;
+            } else if (predicts) {
+                c.p0 = fit.params[4 * (size_t)j];
+                c.p1 = fit.params[4 * (size_t)j + 1];
+                c.p2 = fit.params[4 * (size_t)j + 2];
+                c.kind = status == SLAQ_JOB_FITTED ? (int)fit.family[j] : 2;
+            }
+        }
+        double carry = CUDART_INF;   // running minimum of the gains before this chunk
+        for (int base = 0; base < cap; base += 32) {
+            const int n = base + lane + 1;
+            double g = CUDART_INF;
+            if (n <= cap) g = c.kind == 3 ? 0.0 : raw_gain(c, n);
+            // inclusive running minimum over n
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double up = __shfl_up_sync(kFull, g, o);
+                if (lane >= o) g = fmin(g, up);
+            }
+            g = fmin(g, carry);
+            carry = __shfl_sync(kFull, g, 31);
+            const bool counted = active && n <= cap && n >= first_unit;
+            if (n <= cap) gain[(size_t)j * cap + (n - 1)] = g;
+            const unsigned digit = (unsigned)((unsigned long long)__double_as_longlong(g) >> (64 - kRadixBits));
+            // lanes with the same digit add once: a row is nearly constant in its top bits
+            const unsigned live = __ballot_sync(kFull, counted);
+            if (counted) {
+                const unsigned peers = __match_any_sync(live, digit);
+                if ((int)(__ffs(peers) - 1) == lane) atomicAdd(&sh_hist[digit], (unsigned)__popc(peers));
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) {
+        const unsigned v = sh_hist[i];
+        if (v) atomicAdd(&hist0[i], (unsigned long long)v);
+    }
+}
+
+__global__ void time_model_kernel(JobArrays job, int max_jobs, double* out_s, double* out_w) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= max_jobs) return;
+    double s = CUDART_NAN, w = CUDART_NAN;
+    (void)time_law(job, j, max_jobs, s, w);   // leaves NaN where the job has neither a fixed law nor samples
+    out_s[j] = s;
+    out_w[j] = w;
+}
+
+}  // namespace
+
+int launch_gain(slaq_handle* h, double epoch_seconds, int first_unit) {
+    int blocks = h->sm_count * 4;
+    const int needed = (h->max_jobs + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (blocks > needed) blocks = needed;
+    gain_kernel<<<blocks, kWarpsPerBlock * 32, 0, h->stream>>>(h->job, h->fit, h->max_jobs, h->max_cores, epoch_seconds,
+                                                              first_unit, h->gain, h->scratch.hist);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        h->err = std::string("gain kernel launch: ") + cudaGetErrorString(e);
+        return -1;
+    }
+    return 1;
+}
+
+int launch_time_model(slaq_handle* h, double* d_s, double* d_w) {
+    const int threads = 256, blocks = (h->max_jobs + threads - 1) / threads;
+    time_model_kernel<<<blocks, threads, 0, h->stream>>>(h->job, h->max_jobs, d_s, d_w);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        h->err = std::string("time model kernel launch: ") + cudaGetErrorString(e);
+        return -1;
+    }
+    return 1;
+}
+
+}  // namespace slaq
