@@ -155,8 +155,8 @@ int slaq_append_losses_ex(slaq_t* h, int32_t n, const int32_t* job_ids, const do
  * slaq_load_histories stores each job in its own max_hist-long ring, so later appends
  * extend the window up to max_hist.  slaq_load_histories_packed keeps the rows packed
  * back to back on the device exactly as given (one cudaMalloc of the total size, which
- * replaces any earlier packed load - jobs of an earlier packed load must be reloaded or
- * removed first): a job loaded this way keeps a window of the length it was loaded with,
+ * replaces any earlier packed load - jobs of an earlier packed load that are not listed
+ * again become inactive): a job loaded this way keeps a window of the length it was loaded with,
  * later appends overwrite its oldest point.
  * Errors: SLAQ_E_ARG, SLAQ_E_RANGE, SLAQ_E_NONFINITE, SLAQ_E_NOMEM, SLAQ_E_CUDA.
  */

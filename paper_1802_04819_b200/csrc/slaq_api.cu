@@ -1,0 +1,762 @@
+// C ABI of the library: handle, state updates (append / bulk load / time law / removal),
+// the scheduling epoch, and read-back of results.  The contract is in include/slaq.h.
+#include <math_constants.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "slaq_internal.cuh"
+
+using namespace slaq;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+
+struct Bump {
+    char* base;
+    size_t off = 0;
+    template <class T>
+    T* take(size_t n) {
+        off = (off + kAlign - 1) / kAlign * kAlign;
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+// Lay every device array out inside one workspace; with base == nullptr only the size is computed.
+size_t layout(slaq_handle* h, char* base, int32_t J, int32_t Hmax, int32_t cap) {
+    Bump b{base};
+    const size_t Js = (size_t)J;
+    double* ring = b.take<double>(Js * Hmax);
+    double* wtab = b.take<double>(Hmax);
+    JobArrays job;
+    job.row = b.take<double*>(Js);
+    job.cap = b.take<int32_t>(Js);
+    job.head = b.take<int32_t>(Js);
+    job.count = b.take<int32_t>(Js);
+    job.k_last = b.take<int64_t>(Js);
+    job.m_seen = b.take<double>(Js);
+    job.tm = b.take<double>(8 * Js);
+    job.s_set = b.take<double>(Js);
+    job.w_set = b.take<double>(Js);
+    job.last_alloc = b.take<int32_t>(Js);
+    FitArrays fit;
+    fit.status = b.take<int32_t>(Js);
+    fit.family = b.take<int8_t>(Js);
+    fit.params = b.take<double>(4 * Js);
+    fit.residual = b.take<double>(2 * Js);
+    fit.sweeps = b.take<int32_t>(2 * Js);
+    fit.largest = b.take<double>(Js);
+    fit.span = b.take<double>(Js);
+    Scratch sc;
+    sc.hist = b.take<unsigned long long>((size_t)kRadixPasses * kRadixBins);
+    const size_t zero_from = b.off - sizeof(unsigned long long) * (size_t)kRadixPasses * kRadixBins;
+    sc.ticket = b.take<unsigned int>(8);
+    sc.sel = b.take<SelectState>(1);
+    sc.counters = b.take<long long>(16);
+    sc.zero_bytes = b.off - zero_from;
+    sc.gt = b.take<int32_t>(Js);
+    sc.eq = b.take<int32_t>(Js);
+    sc.block_eq = b.take<long long>(Js / 256 + 2);
+    sc.order = b.take<int32_t>(Js);
+    sc.bucket = b.take<int32_t>((size_t)Hmax + 2);
+    Staging st;
+    st.ids = b.take<int32_t>(Js);
+    st.losses = b.take<double>(Js);
+    st.times = b.take<double>(Js);
+    st.cores = b.take<int32_t>(Js);
+    st.offsets = b.take<int64_t>(Js + 1);
+    st.k_last = b.take<int64_t>(Js);
+    st.m_seen = b.take<double>(Js);
+    double* gain = b.take<double>(Js * cap);
+    int32_t* alloc = b.take<int32_t>(Js);
+    double* reduction = b.take<double>(Js);
+    int32_t* err_word = b.take<int32_t>(4);
+    if (h && base) {
+        h->ring_pool = ring;
+        h->wtab = wtab;
+        h->job = job;
+        h->fit = fit;
+        h->scratch = sc;
+        h->stage = st;
+        h->gain = gain;
+        h->alloc = alloc;
+        h->reduction = reduction;
+        h->err_word = err_word;
+    }
+    return (b.off + kAlign - 1) / kAlign * kAlign;
+}
+
+int fail(slaq_handle* h, int code, const std::string& msg) {
+    if (h) h->err = msg;
+    return code;
+}
+
+int cuda_fail(slaq_handle* h, cudaError_t e, const char* what) {
+    return fail(h, SLAQ_E_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+#define CK(call, what)                                            \
+    do {                                                          \
+        const cudaError_t e_ = (call);                            \
+        if (e_ != cudaSuccess) return cuda_fail(h, e_, what);     \
+    } while (0)
+
+// (Re)initialise jobs: all of them (ids == nullptr) or the listed ones.
+__global__ void init_jobs_kernel(JobArrays job, FitArrays fit, double* ring, int max_jobs, int max_hist,
+                                 const int32_t* ids, int n, int32_t* alloc, double* reduction) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int j = ids ? ids[i] : i;
+    if (j < 0 || j >= max_jobs) return;
+    job.row[j] = ring + (size_t)j * max_hist;
+    job.cap[j] = max_hist;
+    job.head[j] = 0;
+    job.count[j] = 0;
+    job.k_last[j] = -1;
+    job.m_seen[j] = -CUDART_INF;
+    const size_t J = (size_t)max_jobs;
+    for (int k = 0; k < 6; ++k) job.tm[k * J + j] = 0.0;
+    job.tm[6 * J + j] = CUDART_INF;
+    job.tm[7 * J + j] = -CUDART_INF;
+    job.s_set[j] = CUDART_NAN;
+    job.w_set[j] = CUDART_NAN;
+    job.last_alloc[j] = 1;
+    fit.status[j] = SLAQ_JOB_INACTIVE;
+    fit.family[j] = -1;
+    for (int k = 0; k < 4; ++k) fit.params[4 * (size_t)j + k] = CUDART_NAN;
+    fit.residual[2 * (size_t)j] = fit.residual[2 * (size_t)j + 1] = CUDART_INF;
+    fit.sweeps[2 * (size_t)j] = fit.sweeps[2 * (size_t)j + 1] = 0;
+    fit.largest[j] = CUDART_NAN;
+    fit.span[j] = 1.0;
+    alloc[j] = 0;
+    reduction[j] = 0.0;
+}
+
+// One new iteration per listed job: ring write, iteration index, largest reduction seen,
+// and the sums of the iteration-time law (booked at the given or the current core count).
+__global__ void append_kernel(JobArrays job, int max_jobs, int n, const int32_t* ids, const double* losses,
+                              const double* times, const int32_t* cores) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int j = ids[i];
+    if (j < 0 || j >= max_jobs) return;
+    const double loss = losses[i];
+    double* row = job.row[j];
+    const int cap = job.cap[j];
+    int head = job.head[j];
+    const int count = job.count[j];
+    if (count > 0) {
+        const double prev = row[head == 0 ? cap - 1 : head - 1];
+        const double seen = job.m_seen[j], drop = prev - loss;
+        job.m_seen[j] = drop > seen ? drop : seen;
+    }
+    row[head] = loss;
+    head = head + 1 == cap ? 0 : head + 1;
+    job.head[j] = head;
+    job.count[j] = count < cap ? count + 1 : cap;
+    job.k_last[j] += 1;
+    if (times) {
+        int nc = cores ? cores[i] : job.last_alloc[j];
+        if (nc < 1) nc = 1;
+        const double t = times[i], nn = (double)nc, u = __ddiv_rn(1.0, nn);
+        const size_t J = (size_t)max_jobs;
+        double* tm = job.tm + j;
+        tm[0] = __dadd_rn(tm[0], 1.0);
+        tm[J] = __dadd_rn(tm[J], u);
+        tm[2 * J] = __dadd_rn(tm[2 * J], __dmul_rn(u, u));
+        tm[3 * J] = __dadd_rn(tm[3 * J], t);
+        tm[4 * J] = __dadd_rn(tm[4 * J], __dmul_rn(u, t));
+        tm[5 * J] = __dadd_rn(tm[5 * J], __dmul_rn(t, nn));
+        tm[6 * J] = fmin(tm[6 * J], u);
+        tm[7 * J] = fmax(tm[7 * J], u);
+    }
+}
+
+// Bulk load: one warp per listed job copies (ring mode) or adopts (packed mode) its row.
+__global__ void load_kernel(JobArrays job, double* ring, int max_jobs, int max_hist, int n, const int32_t* ids,
+                            const int64_t* offsets, const double* src, const int64_t* k_last, const double* m_seen,
+                            int packed) {
+    const int slot = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (slot >= n) return;
+    const int j = ids[slot];
+    if (j < 0 || j >= max_jobs) return;
+    const int64_t lo = offsets[slot], hi = offsets[slot + 1];
+    int64_t H = hi - lo;
+    if (H > max_hist) H = max_hist;   // keep the newest points
+    const double* from = src + (hi - H);
+    double* row = ring + (size_t)j * max_hist;
+    int cap = max_hist;
+    if (packed && H > 0) {
+        row = const_cast<double*>(from);
+        cap = (int)H;
+    } else {
+        for (int i = lane; i < H; i += 32) row[i] = from[i];
+    }
+    if (lane == 0) {
+        job.row[j] = row;
+        job.cap[j] = cap;
+        job.head[j] = (int)(H % cap);
+        job.count[j] = (int)H;
+        job.k_last[j] = H > 0 ? k_last[slot] : -1;
+        job.m_seen[j] = m_seen ? m_seen[slot] : -CUDART_INF;
+    }
+}
+
+__global__ void set_time_kernel(JobArrays job, int max_jobs, int n, const int32_t* ids, const double* s,
+                                const double* w) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int j = ids[i];
+    if (j < 0 || j >= max_jobs) return;
+    job.s_set[j] = s[i];
+    job.w_set[j] = w[i];
+}
+
+int check_ids(slaq_handle* h, int32_t n, const int32_t* ids, bool forbid_dups) {
+    if (n < 0) return fail(h, SLAQ_E_ARG, "negative count");
+    if (n > 0 && !ids) return fail(h, SLAQ_E_ARG, "job_ids is null");
+    if (n > h->max_jobs) return fail(h, SLAQ_E_ARG, "more entries than job ids");
+    if (++h->stamp_epoch == 0) {
+        std::fill(h->stamp.begin(), h->stamp.end(), 0u);
+        h->stamp_epoch = 1;
+    }
+    for (int32_t i = 0; i < n; ++i) {
+        const int32_t j = ids[i];
+        if (j < 0 || j >= h->max_jobs) return fail(h, SLAQ_E_RANGE, "job id outside 0..max_jobs-1");
+        if (forbid_dups) {
+            if (h->stamp[j] == h->stamp_epoch) return fail(h, SLAQ_E_ARG, "a job id is listed twice in one call");
+            h->stamp[j] = h->stamp_epoch;
+        }
+    }
+    return SLAQ_OK;
+}
+
+int ensure_weights(slaq_handle* h) {
+    if (h->wtab_gamma == h->gamma) return SLAQ_OK;
+    std::vector<double> tab((size_t)h->max_hist);
+    for (int m = 0; m < h->max_hist; ++m) tab[m] = std::pow(h->gamma, (double)m);
+    CK(cudaMemcpyAsync(h->wtab, tab.data(), tab.size() * sizeof(double), cudaMemcpyHostToDevice, h->stream),
+       "upload weight table");
+    CK(cudaStreamSynchronize(h->stream), "upload weight table");
+    h->wtab_gamma = h->gamma;
+    return SLAQ_OK;
+}
+
+int check_device_errors(slaq_handle* h) {
+    int32_t word = 0;
+    CK(cudaMemcpyAsync(&word, h->err_word, sizeof word, cudaMemcpyDeviceToHost, h->stream), "read error word");
+    CK(cudaStreamSynchronize(h->stream), "read error word");
+    if (word != 0) return fail(h, SLAQ_E_CUDA, "a kernel found inconsistent job storage (window longer than its ring)");
+    return SLAQ_OK;
+}
+
+int create_common(slaq_handle* h, int32_t max_jobs, int32_t max_hist, int32_t cap, void* ws, size_t bytes) {
+    h->max_jobs = max_jobs;
+    h->max_hist = max_hist;
+    h->cap_alloc = cap;
+    h->max_cores = cap;
+    CK(cudaGetDevice(&h->device), "cudaGetDevice");
+    cudaDeviceProp prop;
+    CK(cudaGetDeviceProperties(&prop, h->device), "cudaGetDeviceProperties");
+    h->sm_count = prop.multiProcessorCount;
+    const size_t need = layout(nullptr, nullptr, max_jobs, max_hist, cap);
+    if (ws) {
+        if (bytes < need) return fail(h, SLAQ_E_NOMEM, "workspace smaller than slaq_workspace_bytes()");
+        if (reinterpret_cast<uintptr_t>(ws) % kAlign) return fail(h, SLAQ_E_ARG, "workspace is not 256-byte aligned");
+        h->ws = ws;
+        h->owns_ws = false;
+    } else {
+        const cudaError_t e = cudaMalloc(&h->ws, need);
+        if (e != cudaSuccess) {
+            h->ws = nullptr;
+            return fail(h, SLAQ_E_NOMEM, std::string("cudaMalloc of the workspace: ") + cudaGetErrorString(e));
+        }
+        h->owns_ws = true;
+    }
+    h->ws_bytes = need;
+    layout(h, static_cast<char*>(h->ws), max_jobs, max_hist, cap);
+    h->active.assign((size_t)max_jobs, 0);
+    h->stamp.assign((size_t)max_jobs, 0u);
+    h->in_packed.assign((size_t)max_jobs, 0);
+    for (auto& ev : h->ev) CK(cudaEventCreate(&ev), "cudaEventCreate");
+    CK(cudaMemsetAsync(h->scratch.hist, 0, h->scratch.zero_bytes, h->stream), "clear scratch");
+    CK(cudaMemsetAsync(h->err_word, 0, 16, h->stream), "clear error word");
+    const int threads = 256;
+    init_jobs_kernel<<<(max_jobs + threads - 1) / threads, threads, 0, h->stream>>>(
+        h->job, h->fit, h->ring_pool, max_jobs, max_hist, nullptr, max_jobs, h->alloc, h->reduction);
+    CK(cudaGetLastError(), "init kernel");
+    CK(cudaStreamSynchronize(h->stream), "init kernel");
+    return SLAQ_OK;
+}
+
+bool sizes_ok(int32_t max_jobs, int32_t max_hist, int32_t cap) {
+    return max_jobs >= 1 && max_hist >= 4 && max_hist <= kMaxHistLimit && cap >= 1 && cap <= kMaxCoresLimit;
+}
+
+int do_append(slaq_handle* h, int32_t n, const int32_t* ids, const double* losses, const double* times,
+              const int32_t* cores) {
+    if (!h) return SLAQ_E_ARG;
+    if (n > 0 && !losses) return fail(h, SLAQ_E_ARG, "losses is null");
+    const int rc = check_ids(h, n, ids, true);
+    if (rc) return rc;
+    for (int32_t i = 0; i < n; ++i) {
+        if (!std::isfinite(losses[i])) return fail(h, SLAQ_E_NONFINITE, "a loss is not finite");
+        if (times && !std::isfinite(times[i])) return fail(h, SLAQ_E_NONFINITE, "an iteration time is not finite");
+        if (cores && cores[i] < 1) return fail(h, SLAQ_E_ARG, "cores_used must be at least 1");
+    }
+    if (n == 0) return SLAQ_OK;
+    cudaStream_t st = h->stream;
+    CK(cudaMemcpyAsync(h->stage.ids, ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy job ids");
+    CK(cudaMemcpyAsync(h->stage.losses, losses, sizeof(double) * n, cudaMemcpyHostToDevice, st), "copy losses");
+    if (times) CK(cudaMemcpyAsync(h->stage.times, times, sizeof(double) * n, cudaMemcpyHostToDevice, st), "copy times");
+    if (times && cores)
+        CK(cudaMemcpyAsync(h->stage.cores, cores, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy cores");
+    const int threads = 256;
+    append_kernel<<<(n + threads - 1) / threads, threads, 0, st>>>(h->job, h->max_jobs, n, h->stage.ids, h->stage.losses,
+                                                                  times ? h->stage.times : nullptr,
+                                                                  (times && cores) ? h->stage.cores : nullptr);
+    CK(cudaGetLastError(), "append kernel");
+    CK(cudaStreamSynchronize(st), "append");   // the caller may reuse its buffers
+    for (int32_t i = 0; i < n; ++i) {
+        if (!h->active[ids[i]]) {
+            h->active[ids[i]] = 1;
+            h->n_active += 1;
+        }
+    }
+    return SLAQ_OK;
+}
+
+int do_load(slaq_handle* h, int32_t n, const int32_t* ids, const int64_t* offsets, const double* losses,
+            const int64_t* k_last, const double* m_seen, bool packed) {
+    if (!h) return SLAQ_E_ARG;
+    if (n > 0 && (!offsets || !losses || !k_last)) return fail(h, SLAQ_E_ARG, "offsets, losses or k_last is null");
+    const int rc = check_ids(h, n, ids, true);
+    if (rc) return rc;
+    if (n == 0) return SLAQ_OK;
+    if (offsets[0] < 0) return fail(h, SLAQ_E_ARG, "offsets must start at or above 0");
+    for (int32_t i = 0; i < n; ++i)
+        if (offsets[i + 1] < offsets[i]) return fail(h, SLAQ_E_ARG, "offsets must not decrease");
+    const int64_t lo = offsets[0], total = offsets[n] - lo;
+    for (int64_t i = 0; i < total; ++i)
+        if (!std::isfinite(losses[lo + i])) return fail(h, SLAQ_E_NONFINITE, "a loss is not finite");
+    if (m_seen)
+        for (int32_t i = 0; i < n; ++i)
+            if (std::isnan(m_seen[i]) || m_seen[i] == INFINITY)
+                return fail(h, SLAQ_E_NONFINITE, "m_seen must be a number below +infinity");
+    cudaStream_t st = h->stream;
+    double* d_src = nullptr;
+    if (packed) {
+        if (h->packed_pool) {
+            // jobs still stored in the old pool lose their storage with it: deactivate them first
+            std::vector<int32_t> stale;
+            for (int32_t j = 0; j < h->max_jobs; ++j)
+                if (h->in_packed[j]) stale.push_back(j);
+            const int32_t m = (int32_t)stale.size();
+            if (m > 0) {
+                CK(cudaMemcpyAsync(h->stage.ids, stale.data(), sizeof(int32_t) * m, cudaMemcpyHostToDevice, st),
+                   "copy job ids");
+                init_jobs_kernel<<<(m + 255) / 256, 256, 0, st>>>(h->job, h->fit, h->ring_pool, h->max_jobs, h->max_hist,
+                                                                  h->stage.ids, m, h->alloc, h->reduction);
+                CK(cudaGetLastError(), "release kernel");
+            }
+            CK(cudaStreamSynchronize(st), "sync before releasing the packed pool");
+            for (int32_t j : stale) {
+                h->in_packed[j] = 0;
+                if (h->active[j]) {
+                    h->active[j] = 0;
+                    h->n_active -= 1;
+                }
+            }
+            CK(cudaFree(h->packed_pool), "cudaFree packed pool");
+            h->packed_pool = nullptr;
+            h->packed_len = 0;
+        }
+        if (total > 0) {
+            const cudaError_t e = cudaMalloc(&h->packed_pool, sizeof(double) * (size_t)total);
+            if (e != cudaSuccess) {
+                h->packed_pool = nullptr;
+                return fail(h, SLAQ_E_NOMEM, std::string("cudaMalloc of the packed pool: ") + cudaGetErrorString(e));
+            }
+            h->packed_len = (size_t)total;
+        }
+        d_src = h->packed_pool;
+    } else if (total > 0) {
+        const cudaError_t e = cudaMalloc(&d_src, sizeof(double) * (size_t)total);
+        if (e != cudaSuccess)
+            return fail(h, SLAQ_E_NOMEM, std::string("cudaMalloc of the load buffer: ") + cudaGetErrorString(e));
+    }
+    int status = SLAQ_OK;
+    {
+        cudaError_t e = cudaSuccess;
+        if (total > 0) e = cudaMemcpyAsync(d_src, losses + lo, sizeof(double) * (size_t)total, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage.ids, ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st);
+        std::vector<int64_t> rel((size_t)n + 1);
+        for (int32_t i = 0; i <= n; ++i) rel[i] = offsets[i] - lo;
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(h->stage.offsets, rel.data(), sizeof(int64_t) * (n + 1), cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage.k_last, k_last, sizeof(int64_t) * n, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess && m_seen)
+            e = cudaMemcpyAsync(h->stage.m_seen, m_seen, sizeof(double) * n, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) {
+            const int threads = 256, warps = threads / 32;
+            load_kernel<<<(n + warps - 1) / warps, threads, 0, st>>>(h->job, h->ring_pool, h->max_jobs, h->max_hist, n,
+                                                                    h->stage.ids, h->stage.offsets, d_src, h->stage.k_last,
+                                                                    m_seen ? h->stage.m_seen : nullptr, packed ? 1 : 0);
+            e = cudaGetLastError();
+        }
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // `rel` and the caller's buffers are free again
+        if (e != cudaSuccess) status = cuda_fail(h, e, "bulk load");
+    }
+    if (!packed && d_src) cudaFree(d_src);
+    if (status) return status;
+    for (int32_t i = 0; i < n; ++i) {
+        const bool now = offsets[i + 1] > offsets[i];
+        h->in_packed[ids[i]] = (packed && now) ? 1 : 0;
+        if (now != (h->active[ids[i]] != 0)) {
+            h->active[ids[i]] = now ? 1 : 0;
+            h->n_active += now ? 1 : -1;
+        }
+    }
+    return SLAQ_OK;
+}
+
+int run_epoch(slaq_handle* h, double T, int64_t C, int32_t* d_out, bool only_allocate) {
+    if (!only_allocate && !(T > 0.0 && std::isfinite(T))) return fail(h, SLAQ_E_ARG, "epoch_seconds must be positive");
+    if (C < 0) return fail(h, SLAQ_E_ARG, "total_cores must not be negative");
+    const int rc = ensure_weights(h);
+    if (rc) return rc;
+    const int64_t active = h->n_active, cap = h->max_cores;
+    const int floor_units = C >= active ? 1 : 0;
+    const int64_t usable = std::min<int64_t>(C, active * cap);
+    const int64_t want = usable - active * floor_units;
+    cudaStream_t st = h->stream;
+    int launches = 0, k;
+    CK(cudaMemsetAsync(h->scratch.hist, 0, h->scratch.zero_bytes, st), "clear scratch");
+    CK(cudaEventRecord(h->ev[0], st), "event");
+    if (!only_allocate) {
+        if ((k = launch_fit(h)) < 0) return SLAQ_E_CUDA;
+        launches += k;
+    }
+    CK(cudaEventRecord(h->ev[1], st), "event");
+    if (!only_allocate) {
+        if ((k = launch_gain(h, T, floor_units + 1)) < 0) return SLAQ_E_CUDA;
+        launches += k;
+    }
+    CK(cudaEventRecord(h->ev[2], st), "event");
+    if ((k = launch_allocate(h, want, floor_units + 1, !only_allocate, d_out)) < 0) return SLAQ_E_CUDA;
+    launches += k;
+    CK(cudaEventRecord(h->ev[3], st), "event");
+    h->have_epoch = true;
+    h->last_launches = launches;
+    h->last_cores = usable;
+    if (active > 0 && C < active) return SLAQ_W_OVERSUBSCRIBED;
+    if (C > active * cap) return SLAQ_W_UNDERFILLED;
+    return SLAQ_OK;
+}
+
+template <class T>
+int fetch(slaq_handle* h, T* host, const T* dev, size_t n, const char* what) {
+    if (!host) return SLAQ_OK;
+    CK(cudaMemcpyAsync(host, dev, sizeof(T) * n, cudaMemcpyDeviceToHost, h->stream), what);
+    return SLAQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t slaq_workspace_bytes(int32_t max_jobs, int32_t max_hist, int32_t max_cores_per_job) {
+    if (!sizes_ok(max_jobs, max_hist, max_cores_per_job)) return 0;
+    return layout(nullptr, nullptr, max_jobs, max_hist, max_cores_per_job);
+}
+
+int slaq_create_in(void* dev_ws, size_t bytes, int32_t max_jobs, int32_t max_hist, int32_t max_cores_per_job,
+                   slaq_t** out) {
+    if (!out) return SLAQ_E_ARG;
+    *out = nullptr;
+    if (!sizes_ok(max_jobs, max_hist, max_cores_per_job)) return SLAQ_E_ARG;
+    slaq_handle* h = new (std::nothrow) slaq_handle();
+    if (!h) return SLAQ_E_NOMEM;
+    const int rc = create_common(h, max_jobs, max_hist, max_cores_per_job, dev_ws, bytes);
+    if (rc < 0) {
+        slaq_destroy(h);
+        return rc;
+    }
+    *out = h;
+    return SLAQ_OK;
+}
+
+int slaq_create(int32_t max_jobs, int32_t max_hist, slaq_t** out) {
+    return slaq_create_in(nullptr, 0, max_jobs, max_hist, 64, out);
+}
+
+int slaq_destroy(slaq_t* h) {
+    if (!h) return SLAQ_OK;
+    if (h->ws) cudaStreamSynchronize(h->stream);
+    for (auto& ev : h->ev)
+        if (ev) cudaEventDestroy(ev);
+    if (h->packed_pool) cudaFree(h->packed_pool);
+    if (h->owns_ws && h->ws) cudaFree(h->ws);
+    delete h;
+    return SLAQ_OK;
+}
+
+const char* slaq_last_error(const slaq_t* h) { return h ? h->err.c_str() : "null handle"; }
+
+int slaq_set_stream(slaq_t* h, void* cuda_stream) {
+    if (!h) return SLAQ_E_ARG;
+    CK(cudaStreamSynchronize(h->stream), "sync old stream");
+    h->stream = static_cast<cudaStream_t>(cuda_stream);
+    return SLAQ_OK;
+}
+
+int slaq_set_param(slaq_t* h, int key, double value) {
+    if (!h) return SLAQ_E_ARG;
+    switch (key) {
+        case SLAQ_P_GAMMA:
+            if (!(value > 0.0 && value <= 1.0)) return fail(h, SLAQ_E_ARG, "gamma must lie in (0, 1]");
+            h->gamma = value;
+            return SLAQ_OK;
+        case SLAQ_P_LM_TRIALS:
+            if (!(value >= 0 && value <= 1000)) return fail(h, SLAQ_E_ARG, "trials must lie in 0..1000");
+            h->lm_trials = (int32_t)value;
+            return SLAQ_OK;
+        case SLAQ_P_MAX_CORES_PER_JOB:
+            if (!(value >= 1 && value <= kMaxCoresLimit)) return fail(h, SLAQ_E_ARG, "max cores per job must lie in 1..1024");
+            if ((int32_t)value > h->cap_alloc)
+                return fail(h, SLAQ_E_RANGE, "max cores per job beyond what the handle was created for");
+            h->max_cores = (int32_t)value;
+            return SLAQ_OK;
+        case SLAQ_P_MIN_FIT_POINTS:
+            if (!(value >= 4 && value <= kMaxHistLimit)) return fail(h, SLAQ_E_ARG, "min fit points must be at least 4");
+            h->min_fit_points = (int32_t)value;
+            return SLAQ_OK;
+        default:
+            return fail(h, SLAQ_E_ARG, "unknown parameter key");
+    }
+}
+
+int slaq_get_param(const slaq_t* h, int key, double* out_value) {
+    if (!h || !out_value) return SLAQ_E_ARG;
+    switch (key) {
+        case SLAQ_P_GAMMA: *out_value = h->gamma; return SLAQ_OK;
+        case SLAQ_P_LM_TRIALS: *out_value = h->lm_trials; return SLAQ_OK;
+        case SLAQ_P_MAX_CORES_PER_JOB: *out_value = h->max_cores; return SLAQ_OK;
+        case SLAQ_P_MIN_FIT_POINTS: *out_value = h->min_fit_points; return SLAQ_OK;
+        default: return SLAQ_E_ARG;
+    }
+}
+
+int slaq_append_losses(slaq_t* h, int32_t n, const int32_t* job_ids, const double* losses, const double* iter_times) {
+    return do_append(h, n, job_ids, losses, iter_times, nullptr);
+}
+
+int slaq_append_losses_ex(slaq_t* h, int32_t n, const int32_t* job_ids, const double* losses, const double* iter_times,
+                          const int32_t* cores_used) {
+    return do_append(h, n, job_ids, losses, iter_times, cores_used);
+}
+
+int slaq_load_histories(slaq_t* h, int32_t n_jobs, const int32_t* job_ids, const int64_t* offsets, const double* losses,
+                        const int64_t* k_last, const double* m_seen) {
+    return do_load(h, n_jobs, job_ids, offsets, losses, k_last, m_seen, false);
+}
+
+int slaq_load_histories_packed(slaq_t* h, int32_t n_jobs, const int32_t* job_ids, const int64_t* offsets,
+                               const double* losses, const int64_t* k_last, const double* m_seen) {
+    return do_load(h, n_jobs, job_ids, offsets, losses, k_last, m_seen, true);
+}
+
+int slaq_set_time_model(slaq_t* h, int32_t n, const int32_t* job_ids, const double* s, const double* w) {
+    if (!h) return SLAQ_E_ARG;
+    if (n > 0 && (!s || !w)) return fail(h, SLAQ_E_ARG, "s or w is null");
+    const int rc = check_ids(h, n, job_ids, true);
+    if (rc) return rc;
+    for (int32_t i = 0; i < n; ++i)
+        if (!(std::isfinite(s[i]) && std::isfinite(w[i]) && s[i] >= 0.0 && w[i] > 0.0))
+            return fail(h, SLAQ_E_ARG, "time law needs finite s >= 0 and w > 0");
+    if (n == 0) return SLAQ_OK;
+    cudaStream_t st = h->stream;
+    CK(cudaMemcpyAsync(h->stage.ids, job_ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy job ids");
+    CK(cudaMemcpyAsync(h->stage.losses, s, sizeof(double) * n, cudaMemcpyHostToDevice, st), "copy s");
+    CK(cudaMemcpyAsync(h->stage.times, w, sizeof(double) * n, cudaMemcpyHostToDevice, st), "copy w");
+    const int threads = 256;
+    set_time_kernel<<<(n + threads - 1) / threads, threads, 0, st>>>(h->job, h->max_jobs, n, h->stage.ids, h->stage.losses,
+                                                                    h->stage.times);
+    CK(cudaGetLastError(), "time law kernel");
+    CK(cudaStreamSynchronize(st), "time law");
+    return SLAQ_OK;
+}
+
+int slaq_remove_jobs(slaq_t* h, int32_t n, const int32_t* job_ids) {
+    if (!h) return SLAQ_E_ARG;
+    const int rc = check_ids(h, n, job_ids, false);
+    if (rc) return rc;
+    if (n == 0) return SLAQ_OK;
+    cudaStream_t st = h->stream;
+    CK(cudaMemcpyAsync(h->stage.ids, job_ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy job ids");
+    const int threads = 256;
+    init_jobs_kernel<<<(n + threads - 1) / threads, threads, 0, st>>>(h->job, h->fit, h->ring_pool, h->max_jobs,
+                                                                     h->max_hist, h->stage.ids, n, h->alloc, h->reduction);
+    CK(cudaGetLastError(), "remove kernel");
+    CK(cudaStreamSynchronize(st), "remove");
+    for (int32_t i = 0; i < n; ++i) {
+        h->in_packed[job_ids[i]] = 0;
+        if (h->active[job_ids[i]]) {
+            h->active[job_ids[i]] = 0;
+            h->n_active -= 1;
+        }
+    }
+    return SLAQ_OK;
+}
+
+int slaq_schedule_device(slaq_t* h, double epoch_seconds, int64_t total_cores, int32_t* d_out_alloc) {
+    if (!h) return SLAQ_E_ARG;
+    return run_epoch(h, epoch_seconds, total_cores, d_out_alloc, false);
+}
+
+int slaq_schedule(slaq_t* h, double epoch_seconds, int64_t total_cores, int32_t* out_alloc) {
+    if (!h) return SLAQ_E_ARG;
+    if (!out_alloc) return fail(h, SLAQ_E_ARG, "out_alloc is null");
+    const int rc = run_epoch(h, epoch_seconds, total_cores, nullptr, false);
+    if (rc < 0) return rc;
+    CK(cudaMemcpyAsync(out_alloc, h->alloc, sizeof(int32_t) * (size_t)h->max_jobs, cudaMemcpyDeviceToHost, h->stream),
+       "copy allocation");
+    const int ec = check_device_errors(h);
+    return ec ? ec : rc;
+}
+
+int slaq_set_gains(slaq_t* h, const double* gain) {
+    if (!h || !gain) return SLAQ_E_ARG;
+    CK(cudaMemcpyAsync(h->gain, gain, sizeof(double) * (size_t)h->max_jobs * h->max_cores, cudaMemcpyHostToDevice,
+                       h->stream),
+       "copy gains");
+    CK(cudaStreamSynchronize(h->stream), "copy gains");
+    return SLAQ_OK;
+}
+
+int slaq_allocate_only(slaq_t* h, int64_t total_cores, int32_t* out_alloc) {
+    if (!h) return SLAQ_E_ARG;
+    if (!out_alloc) return fail(h, SLAQ_E_ARG, "out_alloc is null");
+    const int rc = run_epoch(h, 1.0, total_cores, nullptr, true);
+    if (rc < 0) return rc;
+    CK(cudaMemcpyAsync(out_alloc, h->alloc, sizeof(int32_t) * (size_t)h->max_jobs, cudaMemcpyDeviceToHost, h->stream),
+       "copy allocation");
+    CK(cudaStreamSynchronize(h->stream), "copy allocation");
+    return rc;
+}
+
+int slaq_get_predictions(slaq_t* h, double* out_reduction, double* out_gain, int8_t* out_family, double* out_params,
+                         double* out_residual, int32_t* out_status, int32_t* out_sweeps, double* out_largest) {
+    if (!h) return SLAQ_E_ARG;
+    if (!h->have_epoch) return fail(h, SLAQ_E_ARG, "no epoch has been scheduled yet");
+    const size_t J = (size_t)h->max_jobs;
+    int rc = 0;
+    if ((rc = fetch(h, out_reduction, h->reduction, J, "copy reductions"))) return rc;
+    if ((rc = fetch(h, out_gain, h->gain, J * h->max_cores, "copy gains"))) return rc;
+    if ((rc = fetch(h, out_family, h->fit.family, J, "copy families"))) return rc;
+    if ((rc = fetch(h, out_params, h->fit.params, 4 * J, "copy parameters"))) return rc;
+    if ((rc = fetch(h, out_residual, h->fit.residual, 2 * J, "copy residuals"))) return rc;
+    if ((rc = fetch(h, out_status, h->fit.status, J, "copy status"))) return rc;
+    if ((rc = fetch(h, out_sweeps, h->fit.sweeps, 2 * J, "copy sweeps"))) return rc;
+    if ((rc = fetch(h, out_largest, h->fit.largest, J, "copy largest reductions"))) return rc;
+    CK(cudaStreamSynchronize(h->stream), "copy predictions");
+    return SLAQ_OK;
+}
+
+int slaq_get_normalised(slaq_t* h, int32_t n, const int32_t* job_ids, int64_t capacity, int64_t* out_offsets,
+                        double* out_changes, double* out_levels, double* out_largest) {
+    if (!h) return SLAQ_E_ARG;
+    int rc = check_ids(h, n, job_ids, false);
+    if (rc) return rc;
+    if ((rc = ensure_weights(h))) return rc;
+    if (n == 0) {
+        if (out_offsets) out_offsets[0] = 0;
+        return SLAQ_OK;
+    }
+    cudaStream_t st = h->stream;
+    std::vector<int32_t> counts((size_t)h->max_jobs);
+    CK(cudaMemcpyAsync(counts.data(), h->job.count, sizeof(int32_t) * counts.size(), cudaMemcpyDeviceToHost, st),
+       "read window lengths");
+    CK(cudaStreamSynchronize(st), "read window lengths");
+    std::vector<int64_t> offs((size_t)n + 1, 0);
+    for (int32_t i = 0; i < n; ++i) offs[i + 1] = offs[i] + counts[job_ids[i]];
+    const int64_t total = offs[n];
+    if ((out_changes || out_levels) && total > capacity) return fail(h, SLAQ_E_RANGE, "output capacity too small");
+    if (out_offsets) std::memcpy(out_offsets, offs.data(), sizeof(int64_t) * (n + 1));
+    double *d_changes = nullptr, *d_levels = nullptr, *d_largest = nullptr;
+    int status = SLAQ_OK;
+    cudaError_t e = cudaMalloc(&d_largest, sizeof(double) * n);
+    if (e == cudaSuccess && total > 0) e = cudaMalloc(&d_changes, sizeof(double) * (size_t)total);
+    if (e == cudaSuccess && total > 0) e = cudaMalloc(&d_levels, sizeof(double) * (size_t)total);
+    if (e != cudaSuccess) {
+        status = fail(h, SLAQ_E_NOMEM, std::string("cudaMalloc of the export buffers: ") + cudaGetErrorString(e));
+    } else {
+        e = cudaMemcpyAsync(h->stage.ids, job_ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(h->stage.offsets, offs.data(), sizeof(int64_t) * (n + 1), cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess && launch_normalise_export(h, n, h->stage.offsets, d_changes, d_levels, d_largest) < 0)
+            status = SLAQ_E_CUDA;
+        if (e == cudaSuccess && status == SLAQ_OK) {
+            if (out_changes && total > 0)
+                e = cudaMemcpyAsync(out_changes, d_changes, sizeof(double) * (size_t)total, cudaMemcpyDeviceToHost, st);
+            if (e == cudaSuccess && out_levels && total > 0)
+                e = cudaMemcpyAsync(out_levels, d_levels, sizeof(double) * (size_t)total, cudaMemcpyDeviceToHost, st);
+            if (e == cudaSuccess && out_largest)
+                e = cudaMemcpyAsync(out_largest, d_largest, sizeof(double) * n, cudaMemcpyDeviceToHost, st);
+        }
+        const cudaError_t e2 = cudaStreamSynchronize(st);
+        if (e == cudaSuccess) e = e2;
+        if (e != cudaSuccess) status = cuda_fail(h, e, "normalised export");
+    }
+    cudaFree(d_changes);
+    cudaFree(d_levels);
+    cudaFree(d_largest);
+    return status;
+}
+
+int slaq_get_time_model(slaq_t* h, double* out_s, double* out_w) {
+    if (!h || !out_s || !out_w) return SLAQ_E_ARG;
+    // the staging arrays hold one double per job each: they serve as the kernel's output
+    if (launch_time_model(h, h->stage.losses, h->stage.times) < 0) return SLAQ_E_CUDA;
+    const size_t J = (size_t)h->max_jobs;
+    CK(cudaMemcpyAsync(out_s, h->stage.losses, sizeof(double) * J, cudaMemcpyDeviceToHost, h->stream), "copy s");
+    CK(cudaMemcpyAsync(out_w, h->stage.times, sizeof(double) * J, cudaMemcpyDeviceToHost, h->stream), "copy w");
+    CK(cudaStreamSynchronize(h->stream), "copy time law");
+    return SLAQ_OK;
+}
+
+int slaq_get_stats(slaq_t* h, slaq_stats* out) {
+    if (!h || !out) return SLAQ_E_ARG;
+    if (!h->have_epoch) return fail(h, SLAQ_E_ARG, "no epoch has been scheduled yet");
+    std::memset(out, 0, sizeof *out);
+    long long counters[16];
+    SelectState sel;
+    CK(cudaMemcpyAsync(counters, h->scratch.counters, sizeof counters, cudaMemcpyDeviceToHost, h->stream), "copy counters");
+    CK(cudaMemcpyAsync(&sel, h->scratch.sel, sizeof sel, cudaMemcpyDeviceToHost, h->stream), "copy selection state");
+    CK(cudaStreamSynchronize(h->stream), "copy statistics");
+    CK(cudaEventElapsedTime(&out->ms_total, h->ev[0], h->ev[3]), "event time");
+    CK(cudaEventElapsedTime(&out->ms_fit, h->ev[0], h->ev[1]), "event time");
+    CK(cudaEventElapsedTime(&out->ms_gain, h->ev[1], h->ev[2]), "event time");
+    CK(cudaEventElapsedTime(&out->ms_alloc, h->ev[2], h->ev[3]), "event time");
+    out->launches = h->last_launches;
+    out->active_jobs = h->n_active;
+    out->points = counters[0];
+    out->model_sweeps = counters[1];
+    out->fitted_jobs = (int32_t)counters[2];
+    out->sublinear_wins = (int32_t)counters[3];
+    out->exponential_wins = (int32_t)counters[4];
+    out->fallback_jobs = (int32_t)counters[5];
+    out->cores_handed_out = counters[6];
+    out->tie_units = counters[7];
+    double tau = 0.0;
+    if (sel.prefix != ~0ull) std::memcpy(&tau, &sel.prefix, sizeof tau);
+    out->threshold = tau;
+    return SLAQ_OK;
+}
+
+}  // extern "C"

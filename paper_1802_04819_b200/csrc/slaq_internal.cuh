@@ -105,6 +105,7 @@ struct slaq_handle {
     int sm_count = 148;
     std::vector<uint8_t> active;      // host mirror: job has at least one loss
     std::vector<uint32_t> stamp;      // host: duplicate detection
+    std::vector<uint8_t> in_packed;   // host: job's row lives in the packed pool
     uint32_t stamp_epoch = 0;
     int32_t n_active = 0;
     std::string err;
