@@ -1,0 +1,229 @@
+"""ctypes binding of libslaq.so: same names as the C ABI, argument marshalling only."""
+
+from __future__ import annotations
+
+import ctypes
+from ctypes import POINTER, c_double, c_float, c_int, c_int8, c_int32, c_int64, c_size_t, c_void_p, c_char_p
+
+import numpy as np
+
+from .build import LIB
+
+JOB_INACTIVE, JOB_FITTED, JOB_SHORT, JOB_NEW, JOB_FIT_FAILED, JOB_FLAT, JOB_NONFINITE, JOB_NO_TIME = -1, 0, 1, 2, 3, 4, 5, 6
+P_GAMMA, P_LM_TRIALS, P_MAX_CORES_PER_JOB, P_MIN_FIT_POINTS = 1, 2, 3, 4
+W_OVERSUBSCRIBED, W_UNDERFILLED = 1, 2
+
+EXPORTED_SYMBOLS = [
+    "slaq_create", "slaq_create_in", "slaq_workspace_bytes", "slaq_destroy", "slaq_last_error", "slaq_set_stream",
+    "slaq_set_param", "slaq_get_param", "slaq_append_losses", "slaq_append_losses_ex", "slaq_load_histories",
+    "slaq_load_histories_packed", "slaq_set_time_model", "slaq_remove_jobs", "slaq_schedule", "slaq_schedule_device",
+    "slaq_get_predictions", "slaq_get_normalised", "slaq_get_time_model", "slaq_set_gains", "slaq_allocate_only",
+    "slaq_get_stats",
+]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [
+        ("ms_total", c_float), ("ms_fit", c_float), ("ms_gain", c_float), ("ms_alloc", c_float),
+        ("launches", c_int32), ("active_jobs", c_int32), ("cores_handed_out", c_int64), ("points", c_int64),
+        ("model_sweeps", c_int64), ("tie_units", c_int64), ("threshold", c_double), ("fitted_jobs", c_int32),
+        ("sublinear_wins", c_int32), ("exponential_wins", c_int32), ("fallback_jobs", c_int32),
+    ]
+
+    def as_dict(self):
+        return {name: getattr(self, name) for name, _ in self._fields_}
+
+
+class SlaqError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"slaq error {code}: {message}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library():
+    """Load libslaq.so (must have been built: ``python -m paper_1802_04819_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not LIB.exists():
+        raise FileNotFoundError(f"{LIB} is missing: build the CUDA library first (paper_1802_04819_b200.build())")
+    lib = ctypes.CDLL(str(LIB))
+    vp = c_void_p
+    sig = {
+        "slaq_create": (c_int, [c_int32, c_int32, POINTER(vp)]),
+        "slaq_create_in": (c_int, [vp, c_size_t, c_int32, c_int32, c_int32, POINTER(vp)]),
+        "slaq_workspace_bytes": (c_size_t, [c_int32, c_int32, c_int32]),
+        "slaq_destroy": (c_int, [vp]),
+        "slaq_last_error": (c_char_p, [vp]),
+        "slaq_set_stream": (c_int, [vp, vp]),
+        "slaq_set_param": (c_int, [vp, c_int, c_double]),
+        "slaq_get_param": (c_int, [vp, c_int, POINTER(c_double)]),
+        "slaq_append_losses": (c_int, [vp, c_int32, vp, vp, vp]),
+        "slaq_append_losses_ex": (c_int, [vp, c_int32, vp, vp, vp, vp]),
+        "slaq_load_histories": (c_int, [vp, c_int32, vp, vp, vp, vp, vp]),
+        "slaq_load_histories_packed": (c_int, [vp, c_int32, vp, vp, vp, vp, vp]),
+        "slaq_set_time_model": (c_int, [vp, c_int32, vp, vp, vp]),
+        "slaq_remove_jobs": (c_int, [vp, c_int32, vp]),
+        "slaq_schedule": (c_int, [vp, c_double, c_int64, vp]),
+        "slaq_schedule_device": (c_int, [vp, c_double, c_int64, vp]),
+        "slaq_get_predictions": (c_int, [vp] * 9),
+        "slaq_get_normalised": (c_int, [vp, c_int32, vp, c_int64, vp, vp, vp, vp]),
+        "slaq_get_time_model": (c_int, [vp, vp, vp]),
+        "slaq_set_gains": (c_int, [vp, vp]),
+        "slaq_allocate_only": (c_int, [vp, c_int64, vp]),
+        "slaq_get_stats": (c_int, [vp, POINTER(Stats)]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def workspace_bytes(max_jobs: int, max_hist: int, max_cores_per_job: int) -> int:
+    return int(load_library().slaq_workspace_bytes(max_jobs, max_hist, max_cores_per_job))
+
+
+def _arr(a, dtype):
+    return None if a is None else np.ascontiguousarray(a, dtype=dtype)
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(c_void_p)
+
+
+class Scheduler:
+    """One scheduler handle.  Methods mirror the C calls of the same name (without ``slaq_``)."""
+
+    def __init__(self, max_jobs: int, max_hist: int, max_cores_per_job: int = 64, workspace=None, stream=None):
+        """``workspace``: optional torch uint8 CUDA tensor of at least ``workspace_bytes(...)`` bytes
+        (device memory owned by the caller); ``stream``: optional ``torch.cuda.Stream``."""
+        self._lib = load_library()
+        self._h = c_void_p()
+        self.max_jobs, self.max_hist, self.max_cores_per_job = int(max_jobs), int(max_hist), int(max_cores_per_job)
+        self._workspace = workspace
+        if workspace is not None:
+            rc = self._lib.slaq_create_in(c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size(),
+                                          max_jobs, max_hist, max_cores_per_job, ctypes.byref(self._h))
+        else:
+            rc = self._lib.slaq_create_in(None, 0, max_jobs, max_hist, max_cores_per_job, ctypes.byref(self._h))
+        if rc < 0 or not self._h:
+            raise SlaqError(rc, "slaq_create failed (is a CUDA device present?)")
+        if stream is not None:
+            self.set_stream(stream)
+
+    # -- plumbing --
+    def _check(self, rc: int) -> int:
+        if rc < 0:
+            raise SlaqError(rc, self._lib.slaq_last_error(self._h).decode())
+        return rc
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.slaq_destroy(self._h)
+            self._h = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # -- the C calls --
+    def set_stream(self, stream):
+        raw = getattr(stream, "cuda_stream", stream)
+        return self._check(self._lib.slaq_set_stream(self._h, c_void_p(raw)))
+
+    def set_param(self, key: int, value: float):
+        rc = self._check(self._lib.slaq_set_param(self._h, key, float(value)))
+        if key == P_MAX_CORES_PER_JOB:
+            self.max_cores_per_job = int(value)
+        return rc
+
+    def get_param(self, key: int) -> float:
+        out = c_double()
+        self._check(self._lib.slaq_get_param(self._h, key, ctypes.byref(out)))
+        return out.value
+
+    def append_losses(self, job_ids, losses, iter_times=None, cores_used=None):
+        ids, ls = _arr(job_ids, np.int32), _arr(losses, np.float64)
+        ts, cs = _arr(iter_times, np.float64), _arr(cores_used, np.int32)
+        if cs is None:
+            return self._check(self._lib.slaq_append_losses(self._h, ids.size, _ptr(ids), _ptr(ls), _ptr(ts)))
+        return self._check(self._lib.slaq_append_losses_ex(self._h, ids.size, _ptr(ids), _ptr(ls), _ptr(ts), _ptr(cs)))
+
+    def load_histories(self, job_ids, offsets, losses, k_last, m_seen=None, packed=False):
+        ids, off = _arr(job_ids, np.int32), _arr(offsets, np.int64)
+        ls, kl, ms = _arr(losses, np.float64), _arr(k_last, np.int64), _arr(m_seen, np.float64)
+        fn = self._lib.slaq_load_histories_packed if packed else self._lib.slaq_load_histories
+        return self._check(fn(self._h, ids.size, _ptr(ids), _ptr(off), _ptr(ls), _ptr(kl), _ptr(ms)))
+
+    def set_time_model(self, job_ids, s, w):
+        ids, s, w = _arr(job_ids, np.int32), _arr(s, np.float64), _arr(w, np.float64)
+        return self._check(self._lib.slaq_set_time_model(self._h, ids.size, _ptr(ids), _ptr(s), _ptr(w)))
+
+    def remove_jobs(self, job_ids):
+        ids = _arr(job_ids, np.int32)
+        return self._check(self._lib.slaq_remove_jobs(self._h, ids.size, _ptr(ids)))
+
+    def schedule(self, epoch_seconds: float, total_cores: int, out_alloc=None):
+        """Returns (alloc int32 [max_jobs], status) with status 0 or a warning code."""
+        out = np.empty(self.max_jobs, np.int32) if out_alloc is None else out_alloc
+        rc = self._check(self._lib.slaq_schedule(self._h, float(epoch_seconds), int(total_cores), _ptr(out)))
+        return out, rc
+
+    def schedule_device(self, epoch_seconds: float, total_cores: int, d_out_alloc=None):
+        """Asynchronous epoch; ``d_out_alloc``: optional torch int32 CUDA tensor [max_jobs]."""
+        ptr = None if d_out_alloc is None else c_void_p(d_out_alloc.data_ptr())
+        return self._check(self._lib.slaq_schedule_device(self._h, float(epoch_seconds), int(total_cores), ptr))
+
+    def get_predictions(self, want_gain=True):
+        J, cap = self.max_jobs, self.max_cores_per_job
+        out = dict(
+            R=np.empty(J), gain=np.empty((J, cap)) if want_gain else None, family=np.empty(J, np.int8),
+            params=np.empty((J, 4)), S=np.empty((J, 2)), status=np.empty(J, np.int32),
+            evals=np.empty((J, 2), np.int32), M=np.empty(J),
+        )
+        self._check(self._lib.slaq_get_predictions(
+            self._h, _ptr(out["R"]), _ptr(out["gain"]), _ptr(out["family"]), _ptr(out["params"]), _ptr(out["S"]),
+            _ptr(out["status"]), _ptr(out["evals"]), _ptr(out["M"])))
+        return out
+
+    def get_normalised(self, job_ids, capacity=None):
+        ids = _arr(job_ids, np.int32)
+        cap = int(capacity if capacity is not None else ids.size * self.max_hist)
+        offsets = np.empty(ids.size + 1, np.int64)
+        changes, levels, largest = np.empty(cap), np.empty(cap), np.empty(ids.size)
+        self._check(self._lib.slaq_get_normalised(self._h, ids.size, _ptr(ids), cap, _ptr(offsets), _ptr(changes),
+                                                  _ptr(levels), _ptr(largest)))
+        total = int(offsets[-1])
+        return offsets, changes[:total], levels[:total], largest
+
+    def get_time_model(self):
+        s, w = np.empty(self.max_jobs), np.empty(self.max_jobs)
+        self._check(self._lib.slaq_get_time_model(self._h, _ptr(s), _ptr(w)))
+        return s, w
+
+    def set_gains(self, gain):
+        g = _arr(gain, np.float64)
+        assert g.shape == (self.max_jobs, self.max_cores_per_job)
+        return self._check(self._lib.slaq_set_gains(self._h, _ptr(g)))
+
+    def allocate_only(self, total_cores: int):
+        out = np.empty(self.max_jobs, np.int32)
+        rc = self._check(self._lib.slaq_allocate_only(self._h, int(total_cores), _ptr(out)))
+        return out, rc
+
+    def get_stats(self) -> Stats:
+        st = Stats()
+        self._check(self._lib.slaq_get_stats(self._h, ctypes.byref(st)))
+        return st

@@ -1,0 +1,281 @@
+"""GPU-vs-oracle parity, element by element, through the C ABI."""
+
+import numpy as np
+import pytest
+
+from workloads import make_workload, make_time_samples
+from gpu_common import compare_epoch, make_scheduler, oracle_epoch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def slaq():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    import paper_1802_04819_b200 as mod
+    mod.build()
+    return mod
+
+
+# ---------------------------------------------------------------- normalisation: bit-exact
+@pytest.mark.parametrize("cfg,n_jobs,packed", [(1, None, False), (2, None, True), (4, 3000, False)])
+def test_normalisation_is_bit_exact(slaq, oracle_mod, cfg, n_jobs, packed):
+    wl = make_workload(cfg, n_jobs=n_jobs)
+    sched = make_scheduler(wl, packed=packed)
+    ids = np.arange(wl.n_jobs)
+    offsets, changes, levels, largest = sched.get_normalised(ids, capacity=int(wl.offsets[-1]))
+    M, dn, y = oracle_mod.normalise(wl.offsets, wl.losses, wl.m_seen)
+    np.testing.assert_array_equal(offsets, wl.offsets)
+    np.testing.assert_array_equal(largest, M)
+    usable = np.repeat(M > 0, wl.hist_len)
+    np.testing.assert_array_equal(changes[usable], dn[usable])
+    np.testing.assert_array_equal(levels[usable], y[usable])
+    assert np.isnan(levels[~usable]).all()
+    # the paper's property: normalised changes never exceed 1
+    assert (changes[usable] <= 1.0).all()
+
+
+# ---------------------------------------------------------------- allocation alone: bit-exact
+def _alloc_case(slaq, oracle_mod, gain, active, C):
+    J, cap = gain.shape
+    sched = slaq.Scheduler(J, 8, cap)
+    live = np.nonzero(active)[0].astype(np.int32)
+    if live.size:
+        sched.append_losses(live, np.ones(live.size))
+    sched.set_gains(gain)
+    got, rc = sched.allocate_only(C)
+    want = oracle_mod.allocate(gain, active, C)
+    np.testing.assert_array_equal(got, want)
+    n_act = int(active.sum())
+    if n_act and C < n_act:
+        assert rc == 1
+    elif C > n_act * cap:
+        assert rc == 2
+    return got
+
+
+def test_allocation_matches_greedy_on_oracle_gains(slaq, oracle_mod):
+    for cfg, n in ((1, None), (2, None), (4, 6000)):
+        wl = make_workload(cfg, n_jobs=n)
+        ref = oracle_mod.predict(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds,
+                                 wl.max_cores_per_job)
+        active = np.ones(wl.n_jobs, np.uint8)
+        for C in (wl.total_cores, wl.n_jobs, wl.n_jobs + 1, 2 * wl.n_jobs + 7, wl.n_jobs * wl.max_cores_per_job - 3):
+            _alloc_case(slaq, oracle_mod, ref["gain"], active, C)
+
+
+def test_allocation_degenerate_gain_tables(slaq, oracle_mod):
+    rng = np.random.default_rng(4)
+    J, cap = 700, 12
+    active = np.ones(J, np.uint8)
+    zero = np.zeros((J, cap))
+    equal = np.full((J, cap), 0.125)
+    few = -np.sort(-rng.integers(0, 4, (J, cap)).astype(float) / 8.0, axis=1)   # many exact ties at 4 levels
+    for gain in (zero, equal, few):
+        for C in (0, 1, J - 1, J, J + 1, 3 * J, J * cap - 1, J * cap, J * cap + 5):
+            _alloc_case(slaq, oracle_mod, gain, active, C)
+    # inactive rows never receive cores, even with the largest gains
+    some = (rng.random(J) < 0.6).astype(np.uint8)
+    raw = -np.sort(-rng.uniform(0, 1, (J, cap)), axis=1)
+    for C in (int(some.sum()) - 3, int(some.sum()), 2 * J, J * cap):
+        got = _alloc_case(slaq, oracle_mod, raw, some, C)
+        assert (got[some == 0] == 0).all()
+    # tiny and huge magnitudes, denormals included, order like their bit patterns
+    wide = -np.sort(-(10.0 ** rng.uniform(-320, 300, (J, cap))), axis=1)
+    for C in (J + 5, 4 * J):
+        _alloc_case(slaq, oracle_mod, wide, active, C)
+
+
+# ---------------------------------------------------------------- whole epoch
+@pytest.mark.parametrize("cfg,n_jobs,packed", [(0, None, False), (1, None, False), (2, None, True),
+                                               (3, 3000, True), (4, 20000, False)])
+def test_epoch_matches_oracle(slaq, oracle_mod, cfg, n_jobs, packed):
+    wl = make_workload(cfg, n_jobs=n_jobs)
+    sched = make_scheduler(wl, packed=packed)
+    alloc, rc = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    assert rc == 0
+    pred = sched.get_predictions()
+    ref = oracle_epoch(oracle_mod, wl)
+    info = compare_epoch(alloc, pred, ref, wl.total_cores, wl.max_cores_per_job)
+    assert alloc.sum() == wl.total_cores
+    assert alloc.min() >= 1 and alloc.max() <= wl.max_cores_per_job
+    g = pred["gain"]
+    assert (g >= 0).all() and (np.diff(g, axis=1) <= 0).all()
+    stats = sched.get_stats()
+    assert stats.cores_handed_out == wl.total_cores
+    assert stats.points == wl.offsets[-1]
+    assert stats.fitted_jobs == info["fitted"]
+    sweeps = (ref["evals"].sum(axis=1) * wl.hist_len)[ref["status"] == 0].sum()
+    assert abs(stats.model_sweeps - sweeps) <= 0.02 * sweeps      # same algorithm, same number of sweeps
+    if cfg == 0:
+        import json
+        from pathlib import Path
+        doc = json.loads((Path(__file__).parent / "golden" / "config0_oracle.json").read_text())
+        assert alloc.tolist() == doc["alloc"]
+
+
+def test_epoch_is_deterministic_and_repeatable(slaq):
+    wl = make_workload(2)
+    sched = make_scheduler(wl, packed=True)
+    a1, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    p1 = sched.get_predictions()
+    a2, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    p2 = sched.get_predictions()
+    np.testing.assert_array_equal(a1, a2)
+    for key in ("gain", "params", "S", "R"):
+        np.testing.assert_array_equal(p1[key], p2[key])
+    # and a second handle in ring layout gives the same bits as the packed one
+    other = make_scheduler(wl, packed=False)
+    a3, _ = other.schedule(wl.epoch_seconds, wl.total_cores)
+    np.testing.assert_array_equal(a1, a3)
+    np.testing.assert_array_equal(p1["gain"], other.get_predictions()["gain"])
+
+
+def test_clones_get_identical_gains_and_ordered_ties(slaq, oracle_mod):
+    wl = make_workload(4, n_jobs=30000)
+    sched = make_scheduler(wl)
+    alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    gain = sched.get_predictions()["gain"]
+    dst = np.nonzero(wl.clone_of >= 0)[0]
+    src = wl.clone_of[dst]
+    np.testing.assert_array_equal(gain[dst], gain[src])
+    lo, hi = np.minimum(src, dst), np.maximum(src, dst)
+    assert (alloc[lo] >= alloc[hi]).all()
+
+
+# ---------------------------------------------------------------- state: append path, ring, time law
+def test_append_path_matches_oracle_scheduler(slaq, oracle_mod):
+    wl = make_workload(1)
+    J, max_hist, cap = wl.n_jobs, 16, wl.max_cores_per_job     # ring shorter than many histories: it wraps
+    sched = slaq.Scheduler(J, max_hist, cap)
+    ref = oracle_mod.OracleScheduler(J, max_hist, cap)
+    H = wl.hist_len
+    cores, secs = make_time_samples(wl, int(H.max()))
+    for step in range(int(H.max())):
+        live = np.nonzero(step < H)[0]
+        losses = wl.losses[wl.offsets[live] + step]
+        sched.append_losses(live, losses, secs[step, live], cores[step, live])
+        ref.append_losses(live, losses, secs[step, live], cores[step, live])
+        if step in (0, 1, 2, 5, 17, int(H.max()) - 1):
+            alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+            out = ref.schedule(wl.epoch_seconds, wl.total_cores)
+            compare_epoch(alloc, sched.get_predictions(), out, wl.total_cores, cap)
+    s, w = sched.get_time_model()
+    rs, rw = ref.time_model()
+    np.testing.assert_array_equal(s, rs)
+    np.testing.assert_array_equal(w, rw)
+    np.testing.assert_allclose(s, wl.s, rtol=1e-9)
+    # default core count of a sample = the last allocation
+    last = alloc.copy()
+    t = wl.s + wl.w / last
+    ids = np.arange(J)
+    newest = wl.losses[wl.offsets[1:] - 1] * 0.97
+    sched.append_losses(ids, newest, t)
+    ref.append_losses(ids, newest, t)
+    s2, w2 = sched.get_time_model()
+    r2s, r2w = ref.time_model()
+    np.testing.assert_array_equal(s2, r2s)
+    np.testing.assert_array_equal(w2, r2w)
+
+
+def test_short_flat_new_and_removed_jobs(slaq, oracle_mod):
+    J, max_hist, cap = 12, 8, 6
+    sched = slaq.Scheduler(J, max_hist, cap)
+    ref = oracle_mod.OracleScheduler(J, max_hist, cap)
+    histories = {
+        0: [5.0],                                  # one point
+        1: [5.0, 4.0],                             # two
+        2: [5.0, 4.0, 3.5],                        # three
+        3: [1.0, 2.0, 3.0, 4.0, 5.0],              # never fell
+        4: [3.0, 3.0, 3.0, 3.0],                   # constant
+        5: [9.0, 6.0, 4.5, 3.6, 3.0, 2.6, 2.3],    # ordinary
+        6: [9.0, 6.0, 4.5, 3.6, 3.0, 2.6, 2.3, 2.1, 1.95, 1.85],   # longer than the ring
+        7: [2.0, 1.0, 1.5, 0.7],                   # a rebound
+    }
+    for step in range(10):
+        ids = [j for j, h in histories.items() if step < len(h)]
+        vals = [histories[j][step] for j in ids]
+        times = [1.0 + 0.1 * j for j in ids]
+        cs = [1 + (step + j) % 3 for j in ids]
+        sched.append_losses(ids, vals, times, cs)
+        ref.append_losses(ids, vals, times, cs)
+    for C in (3, 8, 20, 200):
+        alloc, rc = sched.schedule(2.0, C)
+        out = ref.schedule(2.0, C)
+        compare_epoch(alloc, sched.get_predictions(), out, C, cap)
+        assert (alloc[8:] == 0).all()
+    status = sched.get_predictions()["status"]
+    assert status[0] == slaq.JOB_NEW and status[1] == slaq.JOB_SHORT and status[3] == slaq.JOB_FLAT
+    assert status[4] == slaq.JOB_FLAT and status[5] == slaq.JOB_FITTED and status[9] == slaq.JOB_INACTIVE
+    sched.remove_jobs([5, 6])
+    ref.remove_jobs([5, 6])
+    alloc, _ = sched.schedule(2.0, 20)
+    out = ref.schedule(2.0, 20)
+    compare_epoch(alloc, sched.get_predictions(), out, 20, cap)
+    assert alloc[5] == 0 and alloc[6] == 0
+    # a job without any time sample predicts nothing
+    sched.append_losses([10], [4.0])
+    sched.append_losses([10], [3.0])
+    ref.append_losses([10], [4.0])
+    ref.append_losses([10], [3.0])
+    alloc, _ = sched.schedule(2.0, 20)
+    compare_epoch(alloc, sched.get_predictions(), ref.schedule(2.0, 20), 20, cap)
+    assert sched.get_predictions()["status"][10] == slaq.JOB_NO_TIME
+
+
+def test_empty_scheduler_and_argument_errors(slaq):
+    sched = slaq.Scheduler(16, 8, 4)
+    alloc, rc = sched.schedule(1.0, 10)
+    assert (alloc == 0).all() and rc == 2
+    with pytest.raises(slaq.SlaqError) as e:
+        sched.append_losses([16], [1.0])
+    assert e.value.code == -2
+    with pytest.raises(slaq.SlaqError) as e:
+        sched.append_losses([1, 1], [1.0, 2.0])
+    assert e.value.code == -1
+    with pytest.raises(slaq.SlaqError) as e:
+        sched.append_losses([1], [float("nan")])
+    assert e.value.code == -3
+    with pytest.raises(slaq.SlaqError):
+        sched.schedule(0.0, 10)
+    with pytest.raises(slaq.SlaqError):
+        sched.schedule(1.0, -1)
+    with pytest.raises(slaq.SlaqError):
+        sched.set_param(3, 5)                       # beyond the 4 cores per job the handle was made for
+    with pytest.raises(slaq.SlaqError):
+        sched.set_time_model([0], [0.1], [0.0])
+    # nothing was applied by the failed calls
+    alloc, _ = sched.schedule(1.0, 10)
+    assert (alloc == 0).all()
+    with pytest.raises(slaq.SlaqError):
+        slaq.Scheduler(4, 100000, 4)                # window too long for one warp's shared memory
+
+
+def test_caller_owned_workspace_and_stream(slaq, oracle_mod):
+    import torch
+    wl = make_workload(1)
+    need = slaq.workspace_bytes(wl.n_jobs, wl.max_hist, wl.max_cores_per_job)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    sched = make_scheduler(wl, workspace=ws)
+    sched.set_stream(stream)
+    d_alloc = torch.zeros(wl.n_jobs, dtype=torch.int32, device="cuda")
+    sched.schedule_device(wl.epoch_seconds, wl.total_cores, d_alloc)
+    stream.synchronize()
+    ref = oracle_epoch(oracle_mod, wl)
+    compare_epoch(d_alloc.cpu().numpy(), sched.get_predictions(), ref, wl.total_cores, wl.max_cores_per_job)
+    with pytest.raises(slaq.SlaqError):
+        slaq.Scheduler(wl.n_jobs, wl.max_hist, wl.max_cores_per_job, workspace=ws[: need // 2])
+
+
+def test_parameters_change_the_fit(slaq, oracle_mod):
+    wl = make_workload(1)
+    sched = make_scheduler(wl)
+    sched.set_param(1, 0.8)      # gamma
+    sched.set_param(2, 7)        # trials
+    sched.set_param(3, 16)       # cores per job
+    alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    ref = oracle_mod.schedule(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, wl.total_cores, 16,
+                              gamma=0.8, lm_trials=7)
+    compare_epoch(alloc, sched.get_predictions(), ref, wl.total_cores, 16)
