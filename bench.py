@@ -1,0 +1,285 @@
+"""Benchmark of the per-epoch scheduling path: jobs scheduled per second at 100,000 jobs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one whole scheduling epoch (normalise, fit, predict, allocate) over the
+100,000-job synthetic workload (config 3: ragged histories of 3..1000 losses stored
+packed with a CSR offsets array, 400,000 cores, at most 64 per job, T = 1 s).
+Prints one JSON line.  With N > 1 (under torchrun) every rank schedules its own
+100,000-job cluster partition; there is no exchange on the data path.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from workloads import make_workload, true_curve  # noqa: E402
+
+CFG = 3
+METRIC = "jobs_scheduled_per_second"
+UNIT = "jobs/s"
+# algorithmic fp64 work of the fit, per stored point: one sweep of family I, one of family II, set-up
+FLOP_SWEEP_I, FLOP_SWEEP_II, FLOP_SETUP = 40.0, 25.0, 40.0
+FP64_LANES_PER_SM = 64          # fp64 FMA lanes per SM on B200
+
+
+def rank_info():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in self.rows:
+            if len(row) < 7:
+                continue
+            try:
+                sm.append(float(row[0]))
+                mx.append(float(row[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, row[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def next_losses(wl, step: int, rng):
+    """The loss each job would report `step + 1` iterations after its stored window (same generator law)."""
+    k = (wl.k_last + 1 + step).astype(np.float64)
+    clean = true_curve(wl.family, wl.params, k)
+    return clean * np.exp(wl.sigma * rng.standard_normal(wl.n_jobs))
+
+
+def measured_peaks():
+    path = ROOT / "MEASURED_PEAKS.json"
+    if path.exists():
+        return json.loads(path.read_text()), "measured"
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank, _, world = rank_info()
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    sample_jobs = 20_000
+    wl = make_workload(CFG, n_jobs=sample_jobs)
+    cores = oracle.max_threads()
+
+    def step():
+        return oracle.schedule(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, wl.total_cores,
+                               wl.max_cores_per_job, threads=cores)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = sample_jobs / dt
+    sample = f"first {sample_jobs} jobs of the config-3 generator ({int(wl.offsets[-1])} stored losses), one epoch per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config3_100k_jobs_400k_cores_cap64_hist3-1000_csr", "sample_jobs": sample_jobs},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_gpu(args):
+    import torch
+    rank, local_rank, world = rank_info()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    import paper_1802_04819_b200 as slaq
+    slaq.build()
+
+    wl = make_workload(CFG, seed_offset=rank)          # every rank: its own 100,000-job partition
+    J, cap = wl.n_jobs, wl.max_cores_per_job
+    ids = np.arange(J, dtype=np.int32)
+    stream = torch.cuda.current_stream()
+    sched = slaq.Scheduler(J, wl.max_hist, cap, stream=stream)
+    sched.load_histories(ids, wl.offsets, wl.losses, wl.k_last, wl.m_seen, packed=True)
+    sched.set_time_model(ids, wl.s, wl.w)
+    d_alloc = torch.zeros(J, dtype=torch.int32, device="cuda")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident throughput ----
+    for _ in range(args.warmup):
+        sched.schedule_device(wl.epoch_seconds, wl.total_cores, d_alloc)
+    torch.cuda.synchronize()
+    pred = sched.get_predictions(want_gain=False)
+    fitted = pred["status"] == 0
+    H = wl.hist_len.astype(np.float64)
+    fit_flops = float((H[fitted] * (FLOP_SWEEP_I * pred["evals"][fitted, 0] + FLOP_SWEEP_II * pred["evals"][fitted, 1]
+                                    + FLOP_SETUP)).sum())
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fit_ms, stage_ms, launches = [], [], 0
+    ev0.record(stream)
+    for _ in range(args.steps):
+        sched.schedule_device(wl.epoch_seconds, wl.total_cores, d_alloc)
+        st = sched.get_stats()                 # reads the library's own per-stage CUDA events (same stream)
+        fit_ms.append(st.ms_fit)
+        stage_ms.append((st.ms_fit, st.ms_gain, st.ms_alloc))
+        launches += st.launches
+    ev1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_step = ev0.elapsed_time(ev1) / args.steps
+    alloc_dev = d_alloc.cpu().numpy()
+    assert int(alloc_dev.sum()) == wl.total_cores
+
+    # ---- end to end through the host-pointer calls: append one new loss per job, schedule, read the allocation ----
+    rng = np.random.default_rng(99 + rank)
+    pin = lambda n, dt: torch.empty(n, dtype=dt).pin_memory().numpy()   # noqa: E731
+    h_ids, h_loss, h_time = pin(J, torch.int32), pin(J, torch.float64), pin(J, torch.float64)
+    h_alloc = pin(J, torch.int32)
+    h_ids[:] = ids
+    e2e_steps = max(1, min(args.steps, 10))
+    feeds = [next_losses(wl, s, rng) for s in range(args.warmup + e2e_steps)]
+    last = alloc_dev.astype(np.float64)
+
+    def e2e_step(k):
+        h_loss[:] = feeds[k]
+        h_time[:] = wl.s + wl.w / np.maximum(last, 1.0)
+        sched.append_losses(h_ids, h_loss, h_time)
+        sched.schedule(wl.epoch_seconds, wl.total_cores, out_alloc=h_alloc)
+
+    for k in range(args.warmup):
+        e2e_step(k)
+    barrier()
+    t0 = time.perf_counter()
+    for k in range(e2e_steps):
+        e2e_step(args.warmup + k)
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    assert int(h_alloc.sum()) == wl.total_cores
+
+    times = torch.tensor([ms_step, e2e_s * 1e3], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_step, e2e_ms = float(times[0]), float(times[1])
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        sm_max = float(peaks.get("sm_max_mhz", 1965.0))
+        sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        peak_tflops = sm_count * FP64_LANES_PER_SM * 2 * sm_max * 1e6 / 1e12
+        fit_ms_avg = float(np.mean(fit_ms))
+        achieved = fit_flops / (fit_ms_avg * 1e-3) / 1e12
+        stage = np.mean(np.array(stage_ms), axis=0)
+        line = {
+            "metric": METRIC, "value": world * J / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "config3_100k_jobs_400k_cores_cap64_hist3-1000_csr", "jobs_per_gpu": J,
+                       "stored_losses_per_gpu": int(wl.offsets[-1]), "total_cores_per_gpu": wl.total_cores,
+                       "max_cores_per_job": cap, "epoch_seconds": wl.epoch_seconds,
+                       "l2": "inputs larger than L2 (401 MB of losses read per step)",
+                       "parallelism": f"{world} independent cluster partition(s), one per GPU"},
+            "clocks": clocks,
+            "e2e": {"value": world * J / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": int(J * (4 + 8 + 8)), "d2h_bytes_per_step": int(J * 4 + 4),
+                    "steps": e2e_steps,
+                    "what": "slaq_append_losses (host arrays, one new loss per job) + slaq_schedule (host out_alloc)"},
+            "gpu_launches": launches,
+            "stage_ms": {"fit": float(stage[0]), "gain": float(stage[1]), "alloc": float(stage[2])},
+            "roofline": {"bound": "alu", "kernel": "fit_kernel", "achieved": achieved, "peak": peak_tflops,
+                         "unit": "TFLOP/s", "frac": achieved / peak_tflops, "traffic": None,
+                         "algorithmic_flops_per_launch": fit_flops, "ms_per_launch": fit_ms_avg,
+                         "peak_is": f"{sm_count} SMs x {FP64_LANES_PER_SM} fp64 FMA lanes x 2 x {sm_max:.0f} MHz "
+                                    f"(clock from MEASURED_PEAKS.json: {peak_kind})"},
+        }
+        if args.cpu_baseline:
+            import oracle
+            oracle.build()
+            cores = oracle.max_threads()
+            t0 = time.perf_counter()
+            oracle.schedule(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, wl.total_cores, cap,
+                            threads=cores)
+            dt = time.perf_counter() - t0
+            line["cpu_baseline"] = {"value": J / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": "the whole config-3 workload, one epoch, run once", "seconds": dt}
+        print(json.dumps(line), flush=True)
+    sched.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
