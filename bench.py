@@ -147,7 +147,7 @@ def run_gpu(args):
     import paper_1802_04819_b200 as slaq
     slaq.build()
 
-    wl = make_workload(CFG, seed_offset=rank)          # every rank: its own 100,000-job partition
+    wl = make_workload(CFG, n_jobs=args.jobs, seed_offset=rank)   # every rank: its own 100,000-job partition
     J, cap = wl.n_jobs, wl.max_cores_per_job
     ids = np.arange(J, dtype=np.int32)
     stream = torch.cuda.current_stream()
@@ -232,7 +232,8 @@ def run_gpu(args):
             "metric": METRIC, "value": world * J / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "config3_100k_jobs_400k_cores_cap64_hist3-1000_csr", "jobs_per_gpu": J,
+            "config": {"workload": "config3_100k_jobs_400k_cores_cap64_hist3-1000_csr" if args.jobs is None
+                       else f"config3 generator cut to {J} jobs (profiling run, not the benchmark)", "jobs_per_gpu": J,
                        "stored_losses_per_gpu": int(wl.offsets[-1]), "total_cores_per_gpu": wl.total_cores,
                        "max_cores_per_job": cap, "epoch_seconds": wl.epoch_seconds,
                        "l2": "inputs larger than L2 (401 MB of losses read per step)",
@@ -273,6 +274,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--jobs", type=int, default=None,
+                    help="profiling aid: a smaller cut of the same generator (the reported line is then not the benchmark)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
