@@ -60,9 +60,10 @@ class ClockSampler:
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
 
-    def stop(self):
+    def stop(self, t_from=0.0, t_to=float("inf")):
+        """Summary of the samples that arrived within [t_from, t_to] (perf_counter seconds)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -72,8 +73,8 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for row in self.rows:
-            if len(row) < 7:
+        for stamp, row in self.rows:
+            if len(row) < 7 or not (t_from <= stamp <= t_to + 0.15):
                 continue
             try:
                 sm.append(float(row[0]))
@@ -162,6 +163,8 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     # ---- device-resident throughput ----
+    sampler = ClockSampler(local_rank)
+    sampler.start()                      # nvidia-smi needs a moment to start: the warm-up covers it
     for _ in range(args.warmup):
         sched.schedule_device(wl.epoch_seconds, wl.total_cores, d_alloc)
     torch.cuda.synchronize()
@@ -170,11 +173,10 @@ def run_gpu(args):
     H = wl.hist_len.astype(np.float64)
     fit_flops = float((H[fitted] * (FLOP_SWEEP_I * pred["evals"][fitted, 0] + FLOP_SWEEP_II * pred["evals"][fitted, 1]
                                     + FLOP_SETUP)).sum())
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     fit_ms, stage_ms, launches = [], [], 0
+    t_from = time.perf_counter()
     ev0.record(stream)
     for _ in range(args.steps):
         sched.schedule_device(wl.epoch_seconds, wl.total_cores, d_alloc)
@@ -184,7 +186,7 @@ def run_gpu(args):
         launches += st.launches
     ev1.record(stream)
     barrier()
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_from, time.perf_counter())
     ms_step = ev0.elapsed_time(ev1) / args.steps
     alloc_dev = d_alloc.cpu().numpy()
     assert int(alloc_dev.sum()) == wl.total_cores
@@ -270,7 +272,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
