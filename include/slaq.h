@@ -228,6 +228,41 @@ int slaq_allocate_only(slaq_t* h, int64_t total_cores, int32_t* out_alloc);
 
 int slaq_get_stats(slaq_t* h, slaq_stats* out);
 
+/*
+ * The allocation step for callers that must not allocate device memory.  (The paper has
+ * no counterpart: it is the selection of slaq_allocate_only, packaged so that it touches
+ * the allocator nowhere.)
+ *
+ * Who needs it: a scheduler loop that runs beside other GPU work and cannot afford the
+ * device-wide synchronisation that cudaMalloc and cudaFree imply; a plug-in that was
+ * handed a fixed memory budget and a stream by its host and is not allowed to grow it;
+ * code that runs after start-up in a process whose policy is "no allocation after
+ * initialisation".  Such a caller has no handle (creating one allocates), so there is no
+ * handle here: inputs and outputs are the caller's device buffers, and the scratch the
+ * kernels need (histograms of the threshold search, per-job counts) lives in an array
+ * that is part of the library image, about 0.6 MB on every GPU that loads the library,
+ * until the process ends.
+ *
+ * d_gain [n_jobs x max_cores_per_job], row-major device memory: gain of the n-th core of
+ * row j at [j][n-1], every row non-increasing, values >= +0; every row is an active job.
+ * d_out_alloc [n_jobs] receives a_j (1..max_cores_per_job, sum = min(total_cores,
+ * n_jobs x max_cores_per_job); 0..max when total_cores < n_jobs), d_out_reduction
+ * [n_jobs] the sum of the row's first a_j gains.  cuda_stream: cudaStream_t or NULL.
+ * The call is asynchronous on that stream.  Limits: n_jobs <= 32768,
+ * max_cores_per_job <= 1024; beyond them SLAQ_E_RANGE and nothing is launched.
+ * Other errors: SLAQ_E_ARG (null pointer, n_jobs < 1, total_cores < 0), SLAQ_E_CUDA.
+ * Warnings as slaq_schedule.  No cudaMalloc, cudaFree or other allocating call is made.
+ *
+ * The first call on each device looks up the device address of the static array (the
+ * device that is current at the call); make that first call outside any stream capture.
+ * All calls on one device share the array: it still holds the previous call's values,
+ * the call clears the parts that must start at zero, and two calls whose kernels overlap
+ * on the GPU (different streams, or different host threads without ordering) race on it -
+ * run them one after the other.
+ */
+int slaq_allocate_static(const double* d_gain, int32_t n_jobs, int32_t max_cores_per_job, int64_t total_cores,
+                         int32_t* d_out_alloc, double* d_out_reduction, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

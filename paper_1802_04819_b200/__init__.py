@@ -7,6 +7,6 @@ arguments.  Importing this package does not need a GPU; creating a ``Scheduler``
 
 from .binding import (  # noqa: F401
     JOB_FIT_FAILED, JOB_FITTED, JOB_FLAT, JOB_INACTIVE, JOB_NEW, JOB_NO_TIME, JOB_NONFINITE, JOB_SHORT,
-    EXPORTED_SYMBOLS, Scheduler, SlaqError, Stats, load_library, workspace_bytes,
+    EXPORTED_SYMBOLS, STATIC_MAX_JOBS, Scheduler, SlaqError, Stats, allocate_static, load_library, workspace_bytes,
 )
 from .build import build  # noqa: F401

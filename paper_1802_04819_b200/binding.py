@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = [
     "slaq_set_param", "slaq_get_param", "slaq_append_losses", "slaq_append_losses_ex", "slaq_load_histories",
     "slaq_load_histories_packed", "slaq_set_time_model", "slaq_remove_jobs", "slaq_schedule", "slaq_schedule_device",
     "slaq_get_predictions", "slaq_get_normalised", "slaq_get_time_model", "slaq_set_gains", "slaq_allocate_only",
-    "slaq_get_stats",
+    "slaq_get_stats", "slaq_allocate_static",
 ]
 
 
@@ -75,6 +75,7 @@ def load_library():
         "slaq_set_gains": (c_int, [vp, vp]),
         "slaq_allocate_only": (c_int, [vp, c_int64, vp]),
         "slaq_get_stats": (c_int, [vp, POINTER(Stats)]),
+        "slaq_allocate_static": (c_int, [vp, c_int32, c_int32, c_int64, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -85,6 +86,29 @@ def load_library():
 
 def workspace_bytes(max_jobs: int, max_hist: int, max_cores_per_job: int) -> int:
     return int(load_library().slaq_workspace_bytes(max_jobs, max_hist, max_cores_per_job))
+
+
+STATIC_MAX_JOBS = 32768
+
+
+def allocate_static(d_gain, total_cores: int, d_out_alloc, d_out_reduction, stream=None) -> int:
+    """slaq_allocate_static on torch CUDA tensors: gain float64 [n_jobs, cap], outputs int32 / float64 [n_jobs].
+
+    Allocates nothing on the device; asynchronous on ``stream`` (a torch stream, a raw
+    cudaStream_t or None).  Returns 0 or a warning code; raises SlaqError on an error code.
+    """
+    lib = load_library()
+    n_jobs, cap = d_gain.shape
+    assert d_gain.is_contiguous() and d_out_alloc.is_contiguous() and d_out_reduction.is_contiguous()
+    raw = getattr(stream, "cuda_stream", stream)
+    rc = lib.slaq_allocate_static(c_void_p(d_gain.data_ptr()), n_jobs, cap, int(total_cores),
+                                  c_void_p(d_out_alloc.data_ptr()), c_void_p(d_out_reduction.data_ptr()),
+                                  c_void_p(raw))
+    if rc < 0:
+        messages = {-1: "bad argument", -2: f"size beyond the static scratch (n_jobs <= {STATIC_MAX_JOBS}, cap <= 1024)",
+                    -5: "a CUDA call failed"}
+        raise SlaqError(rc, messages.get(rc, "error"))
+    return rc
 
 
 def _arr(a, dtype):

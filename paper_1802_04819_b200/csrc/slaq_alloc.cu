@@ -312,4 +312,100 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
     return launches;
 }
 
+// ---------------------------------------------------------------------------------
+// Allocation without any device allocation: the same kernels, their scratch in a static
+// device array that ships with the library image.
+// ---------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxJobs = 32768;
+constexpr int kStaticBlocks = kStaticMaxJobs / kJobsPerBlock;
+
+// Everything the selection and the per-job counts write besides the caller's outputs.
+struct StaticScratch {
+    unsigned long long hist[kRadixPasses * kRadixBins];   // cleared every call
+    unsigned int ticket[8];                               // cleared every call
+    SelectState sel;                                      // rewritten every call
+    long long counters[16];                               // cleared every call
+    long long block_eq[kStaticBlocks + 2];                // fully rewritten before it is read
+    int32_t gt[kStaticMaxJobs];                           // fully rewritten before it is read
+    int32_t eq[kStaticMaxJobs];
+    int32_t every_row_active[kStaticMaxJobs];             // set to 1 every call
+    int32_t cores_now[kStaticMaxJobs];                    // sink for the "current core count" the kernels keep
+};
+
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+__global__ void fill_ones_kernel(int32_t* v, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) v[i] = 1;
+}
+
+// Device address of g_static_scratch on the current device, looked up once per device.
+// In host code the array's name only stands for the symbol; kernels need this address.
+int static_scratch_for_current_device(StaticScratch** out) {
+    constexpr int kMaxDevices = 64;
+    static StaticScratch* cache[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SLAQ_E_CUDA;
+    StaticScratch* p = __atomic_load_n(&cache[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        void* addr = nullptr;
+        if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return SLAQ_E_CUDA;
+        p = static_cast<StaticScratch*>(addr);
+        __atomic_store_n(&cache[dev], p, __ATOMIC_RELEASE);   // every thread finds the same address
+    }
+    *out = p;
+    return SLAQ_OK;
+}
+
+}  // namespace
+
 }  // namespace slaq
+
+extern "C" int slaq_allocate_static(const double* d_gain, int32_t n_jobs, int32_t max_cores_per_job,
+                                    int64_t total_cores, int32_t* d_out_alloc, double* d_out_reduction,
+                                    void* cuda_stream) {
+    using namespace slaq;
+    if (!d_gain || !d_out_alloc || !d_out_reduction || n_jobs < 1 || max_cores_per_job < 1 || total_cores < 0)
+        return SLAQ_E_ARG;
+    if (n_jobs > kStaticMaxJobs || max_cores_per_job > kMaxCoresLimit) return SLAQ_E_RANGE;
+    StaticScratch* sc = nullptr;
+    const int rc = static_scratch_for_current_device(&sc);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int J = n_jobs, cap = max_cores_per_job;
+    const int floor_units = total_cores >= J ? 1 : 0, first_unit = floor_units + 1;
+    const long long usable = total_cores < (long long)J * cap ? total_cores : (long long)J * cap;
+    const long long want = usable - (long long)J * floor_units;
+
+    // the array keeps the previous call's contents: clear what the kernels accumulate into
+    if (cudaMemsetAsync(sc->hist, 0, sizeof sc->hist, st) != cudaSuccess) return SLAQ_E_CUDA;
+    if (cudaMemsetAsync(sc->ticket, 0, sizeof sc->ticket, st) != cudaSuccess) return SLAQ_E_CUDA;
+    if (cudaMemsetAsync(sc->counters, 0, sizeof sc->counters, st) != cudaSuccess) return SLAQ_E_CUDA;
+    fill_ones_kernel<<<(J + 255) / 256, 256, 0, st>>>(sc->every_row_active, J);
+    init_select_kernel<<<1, 1, 0, st>>>(&sc->sel, want);
+
+    int sm_count = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    int grid = sm_count * 8;
+    const int needed = (J + (kSelectThreads / 32) - 1) / (kSelectThreads / 32);
+    if (grid > needed) grid = needed;
+    first_hist_kernel<<<grid, kSelectThreads, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, sc->hist);
+    pick_first_kernel<<<1, kSelectThreads, 0, st>>>(sc->hist, &sc->sel);
+    for (int pass = 1; pass < kRadixPasses; ++pass)
+        select_pass_kernel<<<grid, kSelectThreads, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, pass,
+                                                           sc->hist, &sc->sel, sc->ticket);
+    const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
+    count_kernel<<<blocks, 256, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, &sc->sel, sc->gt, sc->eq,
+                                         sc->block_eq);
+    scan_blocks_kernel<<<1, 1024, 0, st>>>(sc->block_eq, blocks);
+    finalise_kernel<<<blocks, 256, 0, st>>>(d_gain, sc->every_row_active, J, cap, floor_units, &sc->sel, sc->gt, sc->eq,
+                                            sc->block_eq, d_out_alloc, d_out_reduction, sc->cores_now, nullptr,
+                                            sc->counters);
+    if (cudaGetLastError() != cudaSuccess) return SLAQ_E_CUDA;
+    if (total_cores < J) return SLAQ_W_OVERSUBSCRIBED;
+    if (total_cores > (long long)J * cap) return SLAQ_W_UNDERFILLED;
+    return SLAQ_OK;
+}
