@@ -60,7 +60,9 @@ enum {
     SLAQ_P_GAMMA = 1,             /* weight base of the fit, point i of H weighs gamma^(H-1-i); default 0.9; (0, 1] */
     SLAQ_P_LM_TRIALS = 2,         /* Levenberg-Marquardt trials per family; default 20; 0 .. 1000 */
     SLAQ_P_MAX_CORES_PER_JOB = 3, /* cap on a_j; default 64; 1 .. what the handle was created for */
-    SLAQ_P_MIN_FIT_POINTS = 4     /* fewer stored points than this use linear extrapolation; default 4; >= 4 */
+    SLAQ_P_MIN_FIT_POINTS = 4,    /* fewer stored points than this use linear extrapolation; default 4; >= 4 */
+    SLAQ_P_FIT_SLICE_BYTES = 5    /* tuning: shared memory one warp of the fit kernel may use (8 KB..200 KB);
+                                     decides how many lanes share a job; results stay within rounding */
 };
 
 /* per-job status written by slaq_schedule (slaq_get_predictions, out_status) */

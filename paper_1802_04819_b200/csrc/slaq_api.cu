@@ -55,15 +55,17 @@ size_t layout(slaq_handle* h, char* base, int32_t J, int32_t Hmax, int32_t cap) 
     Scratch sc;
     sc.hist = b.take<unsigned long long>((size_t)kRadixPasses * kRadixBins);
     const size_t zero_from = b.off - sizeof(unsigned long long) * (size_t)kRadixPasses * kRadixBins;
-    sc.ticket = b.take<unsigned int>(8);
+    sc.ticket = b.take<unsigned int>(kTickets);
     sc.sel = b.take<SelectState>(1);
     sc.counters = b.take<long long>(16);
+    sc.bucket = b.take<int32_t>((size_t)Hmax + 1);
     sc.zero_bytes = b.off - zero_from;
     sc.gt = b.take<int32_t>(Js);
     sc.eq = b.take<int32_t>(Js);
     sc.block_eq = b.take<long long>(Js / 256 + 2);
     sc.order = b.take<int32_t>(Js);
-    sc.bucket = b.take<int32_t>((size_t)Hmax + 2);
+    sc.start = b.take<int32_t>((size_t)Hmax + 1);
+    sc.cursor = b.take<int32_t>((size_t)Hmax + 1);
     Staging st;
     st.ids = b.take<int32_t>(Js);
     st.losses = b.take<double>(Js);
@@ -536,6 +538,10 @@ int slaq_set_param(slaq_t* h, int key, double value) {
             if (!(value >= 4 && value <= kMaxHistLimit)) return fail(h, SLAQ_E_ARG, "min fit points must be at least 4");
             h->min_fit_points = (int32_t)value;
             return SLAQ_OK;
+        case SLAQ_P_FIT_SLICE_BYTES:
+            if (!(value >= 8192 && value <= 200 * 1024)) return fail(h, SLAQ_E_ARG, "fit slice must lie in 8 KB..200 KB");
+            h->fit_slice_bytes = (size_t)value;
+            return SLAQ_OK;
         default:
             return fail(h, SLAQ_E_ARG, "unknown parameter key");
     }
@@ -548,6 +554,7 @@ int slaq_get_param(const slaq_t* h, int key, double* out_value) {
         case SLAQ_P_LM_TRIALS: *out_value = h->lm_trials; return SLAQ_OK;
         case SLAQ_P_MAX_CORES_PER_JOB: *out_value = h->max_cores; return SLAQ_OK;
         case SLAQ_P_MIN_FIT_POINTS: *out_value = h->min_fit_points; return SLAQ_OK;
+        case SLAQ_P_FIT_SLICE_BYTES: *out_value = (double)h->fit_slice_bytes; return SLAQ_OK;
         default: return SLAQ_E_ARG;
     }
 }

@@ -1,13 +1,20 @@
-// Normalisation and curve fit: one warp per job.
+// Normalisation and curve fit.
 //
-// The warp stages the job's window of stored losses in shared memory, finds the largest
-// one-step reduction seen so far, scales the window by it ("Normalizing Quality Metrics"),
-// then fits both convergence families of "Predicting Quality Improvement",
+// For every active job: stage the window of stored losses in shared memory, find the largest
+// one-step reduction seen so far and scale the window by it ("Normalizing Quality Metrics"),
+// then fit both convergence families of "Predicting Quality Improvement",
 //     I : f(x) = 1 / (a x^2 + b x + c) + d          II : f(x) = exp(alpha - beta x) + c,
 // by exponentially weighted least squares with Levenberg-Marquardt, in window coordinates
-// (newest point x = 0, oldest x = -1).  Lanes stride over the points, the normal equations
-// are reduced with warp shuffles, every lane then solves the same 4x4 system.  The family
-// with the lower weighted residual wins.
+// (newest point x = 0, oldest x = -1); the family with the lower weighted residual wins.
+//
+// Work split.  Jobs are sorted by window length (counting sort, longest first) and cut into
+// length classes; one launch per class.  Inside a launch a group of L lanes (L = 1, 2, .. 32,
+// chosen per class so that a warp's windows fit its shared-memory slice) owns one job, so a
+// warp carries 32/L jobs.  A lane walks its job's points m = l, l + L, l + 2L, ... counted
+// from the newest one; both families are evaluated in the same sweep over the window; the
+// partial sums of the normal equations are reduced over the L lanes with shuffles; every
+// lane of a group then runs the same small solve for its job.  All per-job control flow is
+// per lane, so the jobs of a warp may be in different phases of the solver.
 #include <math_constants.h>
 
 #include "slaq_internal.cuh"
@@ -16,47 +23,83 @@ namespace slaq {
 
 namespace {
 
-constexpr int kMaxWarpsPerBlock = 8;
+constexpr int kMaxWarpsPerBlock = 4;
 constexpr size_t kSmemLimit = 227 * 1024;   // shared memory one block may use on sm_100
 constexpr unsigned kFull = 0xffffffffu;
 constexpr double kLambda0 = 1e-3, kLambdaMin = 1e-5, kLambdaMax = 1e12;
+constexpr int kParked = 20;                 // doubles per lane kept in shared memory between sweeps
 
-__device__ __forceinline__ double warp_sum(double v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
-    return v;
-}
-__device__ __forceinline__ double warp_max(double v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(kFull, v, o));
-    return v;
-}
-__device__ __forceinline__ double warp_min(double v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmin(v, __shfl_xor_sync(kFull, v, o));
-    return v;
-}
 __device__ __forceinline__ bool finite_d(double v) { return fabs(v) <= 1.7976931348623157e308; }
 
-// Copy the job's window, oldest first, into sm[0..H).  Ring storage: the newest loss sits
-// just before `head`.  Returns H, or 0 after flagging storage that cannot be right.
-__device__ int stage_window(const JobArrays& job, int j, int max_hist, double* sm, int lane, int32_t* err_word) {
+// Reciprocal to about one ulp: hardware seed and two Newton steps (no special-case paths;
+// a zero, subnormal or non-finite argument gives a non-finite or zero result, which the
+// callers treat as "not usable").
+__device__ __forceinline__ double fast_rcp(double q) {
+    double x;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(x) : "d"(q));
+    double e = fma(-q, x, 1.0);
+    x = fma(x, e, x);
+    e = fma(-q, x, 1.0);
+    return fma(x, e, x);
+}
+
+// Reductions over the L lanes of a group (L a power of two); every lane of the warp takes part.
+__device__ __forceinline__ double group_sum(double v, int L) {
+    for (int o = L >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+__device__ __forceinline__ double group_max(double v, int L) {
+    for (int o = L >> 1; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(kFull, v, o));
+    return v;
+}
+__device__ __forceinline__ double group_min(double v, int L) {
+    for (int o = L >> 1; o > 0; o >>= 1) v = fmin(v, __shfl_xor_sync(kFull, v, o));
+    return v;
+}
+__device__ __forceinline__ int group_and(int v, int L) {
+    for (int o = L >> 1; o > 0; o >>= 1) v &= __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+__device__ __forceinline__ int warp_max_int(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(kFull, v, o));
+    return v;
+}
+
+// Shared-memory view of one warp.  Point m of a lane's job (m = distance from the newest
+// point, m = l + L k for the lane with index l in its group) sits at y[k * 32 + lane]:
+// every access of the sweeps is lane-private and free of bank conflicts.
+struct Lanes {
+    double* y;         // [k_cap + 1][32]
+    double* park;      // [kParked][32]
+    const double* wtab;
+    int lane, L, l;
+};
+
+// The window value at distance m + 1 from the newest point, seen from the lane that owns m.
+__device__ __forceinline__ double older_neighbour(const Lanes& S, int k) {
+    return S.l + 1 < S.L ? S.y[k * 32 + S.lane + 1] : S.y[(k + 1) * 32 + S.lane - (S.L - 1)];
+}
+
+// Copy the job's window into the lane columns (ring storage: the newest loss sits just before
+// `head`).  Returns H, or 0 after flagging storage that cannot be right.
+__device__ int stage_window(const JobArrays& job, int j, int h_cap, const Lanes& S, int32_t* err_word) {
+    if (j < 0) return 0;
     const double* row = job.row[j];
     const int cap = job.cap[j];
     const int H = job.count[j];
-    if (H == 0) return 0;
-    if (H > cap || cap > max_hist || H < 0 || row == nullptr) {   // never expected: record and skip the job
-        if (lane == 0) atomicOr(err_word, 1);
+    if (H <= 0) return 0;
+    if (H > cap || H > h_cap || row == nullptr) {   // never expected: record and skip the job
+        if (S.l == 0) atomicOr(err_word, 1);
         return 0;
     }
-    int start = job.head[j] - H;
-    if (start < 0) start += cap;
-    for (int i = lane; i < H; i += 32) {
-        int s = start + i;
-        if (s >= cap) s -= cap;
-        sm[i] = row[s];
+    int newest = job.head[j] - 1;
+    if (newest < 0) newest += cap;
+    for (int m = S.l, k = 0; m < H; m += S.L, ++k) {
+        int pos = newest - m;
+        if (pos < 0) pos += cap;
+        S.y[k * 32 + S.lane] = row[pos];
     }
-    __syncwarp();
     return H;
 }
 
@@ -64,401 +107,454 @@ struct Normalised {
     double M;        // largest reduction seen so far
     int status;      // SLAQ_JOB_FITTED here means "usable": M > 0 and everything finite
     double rho;      // weighted mean normalised reduction per iteration (linear extrapolation)
+    double ymin, ymax;
 };
 
 // Largest reduction over the window joined with what was seen before it; weighted mean
-// normalised change; then the window is scaled in place to levels y = l / M.
-// d_changes (optional, global) receives the normalised changes of the window.
-__device__ Normalised normalise_window(double* sm, int H, double m_seen, const double* wtab, int lane,
-                                       double* d_changes) {
+// normalised change; then the window is scaled in place to levels y = l / M.  k_all: uniform
+// trip count of the warp.  changes_out (optional, global, indexed oldest first) receives the
+// normalised changes.
+__device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double m_seen, double* changes_out) {
     Normalised out;
     out.M = CUDART_NAN;
     out.rho = 0.0;
-    bool fin = true;
+    int fin = 1;
     double dmax = -CUDART_INF;
-    for (int i = lane; i < H; i += 32) {
-        const double v = sm[i];
-        fin = fin && finite_d(v);
-        if (i > 0) dmax = fmax(dmax, sm[i - 1] - v);
-    }
-    fin = __all_sync(kFull, fin) && !(m_seen != m_seen) && !(m_seen == CUDART_INF);
-    if (!fin) {
-        out.status = SLAQ_JOB_NONFINITE;
-        return out;
-    }
-    if (H == 1) {
-        out.status = SLAQ_JOB_NEW;
-        return out;
-    }
-    dmax = warp_max(dmax);
-    const double M = fmax(m_seen, dmax);
-    out.M = M;
-    if (!(M > 0.0) || !finite_d(M)) {
-        out.status = SLAQ_JOB_FLAT;
-        return out;
-    }
-    double num = 0.0, den = 0.0;
-    for (int i = lane; i < H; i += 32) {
-        if (i > 0) {
-            const double change = __ddiv_rn(sm[i - 1] - sm[i], M);
-            const double w = wtab[H - 1 - i];
-            num = fma(w, change, num);
-            den += w;
-            if (d_changes) d_changes[i] = change;
-        } else if (d_changes) {
-            d_changes[0] = 0.0;
+    for (int k = 0; k < k_all; ++k) {
+        const int m = S.l + S.L * k;
+        if (m < H) {
+            const double v = S.y[k * 32 + S.lane];
+            fin &= finite_d(v) ? 1 : 0;
+            if (m + 1 < H) dmax = fmax(dmax, older_neighbour(S, k) - v);
         }
     }
-    num = warp_sum(num);
-    den = warp_sum(den);
+    fin = group_and(fin, S.L);
+    dmax = group_max(dmax, S.L);
+    if (H <= 0) {
+        out.status = SLAQ_JOB_INACTIVE;
+    } else if (!fin || m_seen != m_seen || m_seen == CUDART_INF) {
+        out.status = SLAQ_JOB_NONFINITE;
+    } else if (H == 1) {
+        out.status = SLAQ_JOB_NEW;
+    } else {
+        out.M = fmax(m_seen, dmax);
+        out.status = (out.M > 0.0 && finite_d(out.M)) ? SLAQ_JOB_FITTED : SLAQ_JOB_FLAT;
+    }
+    const bool usable = out.status == SLAQ_JOB_FITTED;
+    const double M = out.M;
+    double num = 0.0, den = 0.0;
+    for (int k = 0; k < k_all; ++k) {
+        const int m = S.l + S.L * k;
+        if (usable && m + 1 < H) {
+            const double change = __ddiv_rn(older_neighbour(S, k) - S.y[k * 32 + S.lane], M);
+            const double w = S.wtab[m];
+            num = fma(w, change, num);
+            den += w;
+            if (changes_out) changes_out[H - 1 - m] = change;
+        }
+    }
+    if (changes_out && usable && S.l == 0) changes_out[0] = 0.0;
+    num = group_sum(num, S.L);
+    den = group_sum(den, S.L);
     out.rho = fmax(num / den, 0.0);
+    __syncwarp();   // all neighbour reads are done before the window is overwritten
+    double lo = CUDART_INF, hi = -CUDART_INF;
+    for (int k = 0; k < k_all; ++k) {
+        const int m = S.l + S.L * k;
+        if (usable && m < H) {
+            const double y = __ddiv_rn(S.y[k * 32 + S.lane], M);
+            S.y[k * 32 + S.lane] = y;
+            lo = fmin(lo, y);
+            hi = fmax(hi, y);
+        }
+    }
+    out.ymin = group_min(lo, S.L);
+    out.ymax = group_max(hi, S.L);
     __syncwarp();
-    for (int i = lane; i < H; i += 32) sm[i] = __ddiv_rn(sm[i], M);
-    __syncwarp();
-    out.status = SLAQ_JOB_FITTED;
     return out;
 }
 
-// ---- small dense algebra, every lane does the same work on the same numbers ----
+// ---- small dense algebra: every lane solves its own job's system ----
 
-// Solve B d = r for a symmetric positive definite N x N system (N = 3 or 4) by Cholesky.
-template <int N>
-__device__ bool chol_solve(const double (&B)[4][4], const double (&r)[4], double (&d)[4]) {
-    double L[4][4];
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-#pragma unroll
-        for (int j = 0; j <= i; ++j) {
-            double sum = B[i][j];
-#pragma unroll
-            for (int k = 0; k < j; ++k) sum = fma(-L[i][k], L[j][k], sum);
-            if (i == j) {
-                if (!(sum > 0.0) || !finite_d(sum)) return false;
-                L[i][i] = sqrt(sum);
-            } else {
-                L[i][j] = sum / L[j][j];
-            }
-        }
-    }
-    double z[4];
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-        double sum = r[i];
-#pragma unroll
-        for (int k = 0; k < i; ++k) sum = fma(-L[i][k], z[k], sum);
-        z[i] = sum / L[i][i];
-    }
-    bool ok = true;
-#pragma unroll
-    for (int i = N - 1; i >= 0; --i) {
-        double sum = z[i];
-#pragma unroll
-        for (int k = i + 1; k < N; ++k) sum = fma(-L[k][i], d[k], sum);
-        d[i] = sum / L[i][i];
-        ok = ok && finite_d(d[i]);
-    }
+struct Sym4 {   // symmetric 4x4, upper triangle
+    double a00, a01, a02, a03, a11, a12, a13, a22, a23, a33;
+};
+
+// Solve B x = r for symmetric positive definite B by the root-free Cholesky factorisation
+// B = L D L^T.  False if a pivot is not positive and finite or the solution is not finite.
+__device__ bool ldl_solve(const Sym4& B, const double (&r)[4], double (&x)[4]) {
+    const double d0 = B.a00;
+    const double i0 = 1.0 / d0;
+    const double l10 = B.a01 * i0, l20 = B.a02 * i0, l30 = B.a03 * i0;
+    const double d1 = fma(-l10, B.a01, B.a11);
+    const double i1 = 1.0 / d1;
+    const double t21 = fma(-l20, B.a01, B.a12), t31 = fma(-l30, B.a01, B.a13);
+    const double l21 = t21 * i1, l31 = t31 * i1;
+    const double d2 = fma(-l21, t21, fma(-l20, B.a02, B.a22));
+    const double i2 = 1.0 / d2;
+    const double t32 = fma(-l31, t21, fma(-l30, B.a02, B.a23));
+    const double l32 = t32 * i2;
+    const double d3 = fma(-l32, t32, fma(-l31, t31, fma(-l30, B.a03, B.a33)));
+    const double i3 = 1.0 / d3;
+    bool ok = d0 > 0.0 && d1 > 0.0 && d2 > 0.0 && d3 > 0.0 && finite_d(d0) && finite_d(d1) && finite_d(d2) &&
+              finite_d(d3);
+    const double z0 = r[0];
+    const double z1 = fma(-l10, z0, r[1]);
+    const double z2 = fma(-l21, z1, fma(-l20, z0, r[2]));
+    const double z3 = fma(-l32, z2, fma(-l31, z1, fma(-l30, z0, r[3])));
+    x[3] = z3 * i3;
+    x[2] = fma(-l32, x[3], z2 * i2);
+    x[1] = fma(-l31, x[3], fma(-l21, x[2], z1 * i1));
+    x[0] = fma(-l30, x[3], fma(-l20, x[2], fma(-l10, x[1], z0 * i0)));
+    ok = ok && finite_d(x[0]) && finite_d(x[1]) && finite_d(x[2]) && finite_d(x[3]);
     return ok;
 }
 
-struct Window {
-    const double* y;      // normalised levels in shared memory
-    const double* wtab;   // gamma^m in shared memory
-    int H;
-    int lane;
-    double inv_span;      // 1 / (H - 1)
-    double sw;            // sum of weights
+// Solver state of one family for one job (held by every lane of the job's group).
+struct Family {
+    double p[4];       // current parameters
+    double trial[4];   // trial point of the running sweep
+    double S;          // weighted residual at p
+    double lambda, nu;
+    double predicted;  // reduction the quadratic model promises for the trial step
+    unsigned was_frozen;
+    int sweeps;
+    bool ok;           // the starting point was usable
+    bool done;         // no further trials
+    bool has_trial;    // the running sweep evaluates `trial`
 };
 
-// Normal equations of one family at parameters p: S = sum w r^2, A = sum w J J^T,
-// g = sum w J r, r = y - f.  False when the model is undefined at a stored point or a
-// sum is not finite.
-struct Sublinear {
-    static constexpr int P = 4;
-    __device__ static double lower(int a) { return a == 3 ? -CUDART_INF : (a == 2 ? 1e-12 : 0.0); }
-    __device__ static bool normal_eq(const Window& W, const double (&p)[4], double (&A)[4][4], double (&g)[4],
-                                     double& S) {
-        // with u = 1/q^2: J = (-u x^2, -u x, -u, 1); A needs the moments of w u^2 and w u
-        double m0 = 0, m1 = 0, m2 = 0, m3 = 0, m4 = 0, n0 = 0, n1 = 0, n2 = 0;
-        double h0 = 0, h1 = 0, h2 = 0, gd = 0, acc = 0;
-        bool ok = true;
-        for (int i = W.lane; i < W.H; i += 32) {
-            const double x = (double)(i - (W.H - 1)) * W.inv_span;
-            const double w = W.wtab[W.H - 1 - i];
-            const double q = fma(fma(p[0], x, p[1]), x, p[2]);
-            ok = ok && (q > 0.0);
-            const double inv = 1.0 / q;
-            const double r = W.y[i] - (inv + p[3]);
-            const double u = inv * inv;
-            const double x2 = x * x;
-            const double wu = w * u, wuu = wu * u, wur = wu * r, wr = w * r;
-            const double t = wuu * x2;
-            m0 += wuu;
-            m1 = fma(wuu, x, m1);
-            m2 += t;
-            m3 = fma(t, x, m3);
-            m4 = fma(t, x2, m4);
-            n0 += wu;
-            n1 = fma(wu, x, n1);
-            n2 = fma(wu, x2, n2);
-            h0 += wur;
-            h1 = fma(wur, x, h1);
-            h2 = fma(wur, x2, h2);
-            gd += wr;
-            acc = fma(wr, r, acc);
-        }
-        ok = __all_sync(kFull, ok);
-        if (!ok) return false;
-        m0 = warp_sum(m0); m1 = warp_sum(m1); m2 = warp_sum(m2); m3 = warp_sum(m3); m4 = warp_sum(m4);
-        n0 = warp_sum(n0); n1 = warp_sum(n1); n2 = warp_sum(n2);
-        h0 = warp_sum(h0); h1 = warp_sum(h1); h2 = warp_sum(h2);
-        gd = warp_sum(gd);
-        S = warp_sum(acc);
-        A[0][0] = m4; A[0][1] = A[1][0] = m3; A[0][2] = A[2][0] = m2; A[1][1] = m2;
-        A[1][2] = A[2][1] = m1; A[2][2] = m0;
-        A[0][3] = A[3][0] = -n2; A[1][3] = A[3][1] = -n1; A[2][3] = A[3][2] = -n0; A[3][3] = W.sw;
-        g[0] = -h2; g[1] = -h1; g[2] = -h0; g[3] = gd;
-        const double chk = m0 + m1 + m2 + m3 + m4 + n0 + n1 + n2 + h0 + h1 + h2 + gd + S;
-        return finite_d(chk);
+template <int P>
+__device__ __forceinline__ double lower_bound_of(int a) {
+    if (P == 4) return a == 3 ? -CUDART_INF : (a == 2 ? 1e-12 : 0.0);   // a >= 0, b >= 0, c >= 1e-12
+    return a == 1 ? 0.0 : -CUDART_INF;                                   // beta >= 0
+}
+
+// One Levenberg-Marquardt trial up to the point where the model must be evaluated: freeze
+// parameters that sit on their bound while the descent direction or the solved step points
+// outside (and keep them frozen from then on), solve (A + lambda diag A) step = g over the
+// rest, clip the trial point to the bounds, and record the reduction the quadratic model
+// promises.  `busy` = this lane has a trial to prepare; the re-solve loop runs while any
+// lane of the warp needs another round.
+template <int P>
+__device__ void prepare_trial(Family& F, const Sym4& A, const double (&g)[4], bool busy, double sum_wy2) {
+    F.has_trial = false;
+    if (busy && F.S <= 1e-28 * sum_wy2) {   // residual is zero to rounding
+        F.done = true;
+        busy = false;
     }
-};
-
-struct Exponential {
-    static constexpr int P = 3;
-    __device__ static double lower(int a) { return a == 1 ? 0.0 : -CUDART_INF; }
-    __device__ static bool normal_eq(const Window& W, const double (&p)[4], double (&A)[4][4], double (&g)[4],
-                                     double& S) {
-        // J = (e, -x e, 1) with e = exp(alpha - beta x)
-        double e0 = 0, e1 = 0, e2 = 0, f0 = 0, f1 = 0, h0 = 0, h1 = 0, gc = 0, acc = 0;
-        for (int i = W.lane; i < W.H; i += 32) {
-            const double x = (double)(i - (W.H - 1)) * W.inv_span;
-            const double w = W.wtab[W.H - 1 - i];
-            const double e = exp(fma(-p[1], x, p[0]));
-            const double r = W.y[i] - (e + p[2]);
-            const double we = w * e, wee = we * e, wer = we * r, wr = w * r;
-            const double t = wee * x;
-            e0 += wee;
-            e1 += t;
-            e2 = fma(t, x, e2);
-            f0 += we;
-            f1 = fma(we, x, f1);
-            h0 += wer;
-            h1 = fma(wer, x, h1);
-            gc += wr;
-            acc = fma(wr, r, acc);
-        }
-        e0 = warp_sum(e0); e1 = warp_sum(e1); e2 = warp_sum(e2);
-        f0 = warp_sum(f0); f1 = warp_sum(f1);
-        h0 = warp_sum(h0); h1 = warp_sum(h1);
-        gc = warp_sum(gc);
-        S = warp_sum(acc);
-        A[0][0] = e0; A[0][1] = A[1][0] = -e1; A[1][1] = e2;
-        A[0][2] = A[2][0] = f0; A[1][2] = A[2][1] = -f1; A[2][2] = W.sw;
-        A[0][3] = A[3][0] = A[1][3] = A[3][1] = A[2][3] = A[3][2] = 0.0; A[3][3] = 1.0;
-        g[0] = h0; g[1] = -h1; g[2] = gc; g[3] = 0.0;
-        const double chk = e0 + e1 + e2 + f0 + f1 + h0 + h1 + gc + S;
-        return finite_d(chk);
-    }
-};
-
-struct LmResult {
-    bool ok;      // the starting point was usable
-    double S;     // final weighted residual
-    int sweeps;   // passes over the window: the start plus one per solved trial
-};
-
-// Levenberg-Marquardt with Marquardt's diagonal scaling and the gain-ratio damping update
-// (Madsen, Nielsen, Tingleff 2004).  Parameters on their lower bound are frozen while the
-// descent direction or the solved step points outside, and stay frozen from then on; the
-// trial point is clipped to the bounds; a trial is accepted only if the residual strictly falls.
-template <class F>
-__device__ LmResult levenberg_marquardt(const Window& W, double (&p)[4], int trials, double sum_wy2) {
-    constexpr int P = F::P;
-    LmResult out;
-    out.sweeps = 1;
-    out.S = CUDART_INF;
-    double A[4][4], g[4], S;
-    out.ok = F::normal_eq(W, p, A, g, S);
-    if (!out.ok) return out;
-    double lambda = kLambda0, nu = 2.0;
-    unsigned was_frozen = 0;
-    for (int t = 0; t < trials; ++t) {
-        if (S <= 1e-28 * sum_wy2) break;
-        unsigned frozen = 0;
+    unsigned frozen = 0;
 #pragma unroll
-        for (int a = 0; a < P; ++a)
-            if (p[a] <= F::lower(a) && (g[a] < 0.0 || ((was_frozen >> a) & 1u))) frozen |= 1u << a;
-        double step[4] = {0.0, 0.0, 0.0, 0.0};
-        bool solved = false;
-        for (int round = 0; round <= P; ++round) {
-            double B[4][4], rhs[4];
-#pragma unroll
-            for (int a = 0; a < 4; ++a) {
-                const bool fa = a >= P || ((frozen >> a) & 1u);
-#pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    const bool fb = b >= P || ((frozen >> b) & 1u);
-                    B[a][b] = (fa || fb) ? 0.0 : A[a][b];
-                }
-                B[a][a] = fa ? 1.0 : fma(lambda, fmax(A[a][a], 1e-300), A[a][a]);
-                rhs[a] = fa ? 0.0 : g[a];
-            }
-            solved = chol_solve<P>(B, rhs, step);
-            if (!solved) break;
+    for (int a = 0; a < P; ++a)
+        if (F.p[a] <= lower_bound_of<P>(a) && (g[a] < 0.0 || ((F.was_frozen >> a) & 1u))) frozen |= 1u << a;
+    double step[4] = {0.0, 0.0, 0.0, 0.0};
+    bool solved = false, again = busy;
+    for (int round = 0; round <= P; ++round) {
+        if (!__any_sync(kFull, again)) break;
+        if (again) {
+            const bool f0 = frozen & 1u, f1 = frozen & 2u, f2 = frozen & 4u, f3 = P < 4 || (frozen & 8u);
+            Sym4 B;
+            B.a00 = f0 ? 1.0 : fma(F.lambda, fmax(A.a00, 1e-300), A.a00);
+            B.a11 = f1 ? 1.0 : fma(F.lambda, fmax(A.a11, 1e-300), A.a11);
+            B.a22 = f2 ? 1.0 : fma(F.lambda, fmax(A.a22, 1e-300), A.a22);
+            B.a33 = f3 ? 1.0 : fma(F.lambda, fmax(A.a33, 1e-300), A.a33);
+            B.a01 = (f0 || f1) ? 0.0 : A.a01;
+            B.a02 = (f0 || f2) ? 0.0 : A.a02;
+            B.a03 = (f0 || f3) ? 0.0 : A.a03;
+            B.a12 = (f1 || f2) ? 0.0 : A.a12;
+            B.a13 = (f1 || f3) ? 0.0 : A.a13;
+            B.a23 = (f2 || f3) ? 0.0 : A.a23;
+            const double rhs[4] = {f0 ? 0.0 : g[0], f1 ? 0.0 : g[1], f2 ? 0.0 : g[2], f3 ? 0.0 : g[3]};
+            solved = ldl_solve(B, rhs, step);
             unsigned grow = 0;
+            if (solved) {
 #pragma unroll
-            for (int a = 0; a < P; ++a)
-                if (!((frozen >> a) & 1u) && p[a] <= F::lower(a) && step[a] < 0.0) grow |= 1u << a;
-            if (!grow) break;
+                for (int a = 0; a < P; ++a)
+                    if (!((frozen >> a) & 1u) && F.p[a] <= lower_bound_of<P>(a) && step[a] < 0.0) grow |= 1u << a;
+            }
             frozen |= grow;
-        }
-        was_frozen |= frozen;
-        bool accepted = false;
-        if (solved) {
-            double trial[4] = {0.0, 0.0, 0.0, 0.0}, d[4] = {0.0, 0.0, 0.0, 0.0};
-            bool fin = true;
-#pragma unroll
-            for (int a = 0; a < P; ++a) {
-                trial[a] = fmax(p[a] + step[a], F::lower(a));
-                d[a] = trial[a] - p[a];
-                fin = fin && finite_d(trial[a]);
-            }
-            double dg = 0.0, dAd = 0.0;
-#pragma unroll
-            for (int a = 0; a < P; ++a) {
-                dg = fma(d[a], g[a], dg);
-#pragma unroll
-                for (int b = 0; b < P; ++b) dAd = fma(d[a] * A[a][b], d[b], dAd);
-            }
-            const double predicted = 2.0 * dg - dAd;
-            double A2[4][4], g2[4], S2 = CUDART_INF;
-            bool ok2 = false;
-            out.sweeps += 1;   // every solved trial counts as one sweep over the window
-            if (fin) ok2 = F::normal_eq(W, trial, A2, g2, S2);
-            if (ok2 && S2 < S) {
-                accepted = true;
-                const double S_before = S;
-#pragma unroll
-                for (int a = 0; a < 4; ++a) {
-                    p[a] = trial[a];
-                    g[a] = g2[a];
-#pragma unroll
-                    for (int b = 0; b < 4; ++b) A[a][b] = A2[a][b];
-                }
-                S = S2;
-                const double rho = predicted > 0.0 ? (S_before - S) / predicted : 0.0;
-                const double c = 2.0 * rho - 1.0;
-                lambda *= fmax(1.0 / 3.0, 1.0 - c * c * c);
-                nu = 2.0;
-                lambda = fmin(fmax(lambda, kLambdaMin), kLambdaMax);
-                if (S_before - S <= 1e-14 * S_before) break;
-            }
-        }
-        if (!accepted) {
-            lambda = fmin(lambda * nu, kLambdaMax);
-            nu *= 2.0;
+            again = solved && grow != 0;
         }
     }
-    out.S = S;
-    return out;
+    if (!busy) return;
+    F.was_frozen |= frozen;
+    if (!solved) {   // no step: counts as a rejected trial
+        F.lambda = fmin(F.lambda * F.nu, kLambdaMax);
+        F.nu *= 2.0;
+        return;
+    }
+    double d[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll
+    for (int a = 0; a < P; ++a) {
+        F.trial[a] = fmax(F.p[a] + step[a], lower_bound_of<P>(a));
+        d[a] = F.trial[a] - F.p[a];
+    }
+    const double dg = fma(d[0], g[0], fma(d[1], g[1], fma(d[2], g[2], d[3] * g[3])));
+    const double Ad0 = fma(A.a00, d[0], fma(A.a01, d[1], fma(A.a02, d[2], A.a03 * d[3])));
+    const double Ad1 = fma(A.a01, d[0], fma(A.a11, d[1], fma(A.a12, d[2], A.a13 * d[3])));
+    const double Ad2 = fma(A.a02, d[0], fma(A.a12, d[1], fma(A.a22, d[2], A.a23 * d[3])));
+    const double Ad3 = fma(A.a03, d[0], fma(A.a13, d[1], fma(A.a23, d[2], A.a33 * d[3])));
+    const double dAd = fma(d[0], Ad0, fma(d[1], Ad1, fma(d[2], Ad2, d[3] * Ad3)));
+    F.predicted = 2.0 * dg - dAd;
+    F.has_trial = true;
+    F.sweeps += 1;   // every solved trial costs one sweep over the window
+}
+
+// After the sweep at the trial point: accept it only if the residual strictly fell, and move
+// the damping by the gain ratio (Madsen, Nielsen, Tingleff 2004).  Returns whether accepted.
+__device__ __forceinline__ bool finish_trial(Family& F, bool ok_trial, double S_trial) {
+    if (!F.has_trial) return false;
+    F.has_trial = false;
+    if (ok_trial && S_trial < F.S) {
+        const double S_before = F.S;
+#pragma unroll
+        for (int a = 0; a < 4; ++a) F.p[a] = F.trial[a];
+        F.S = S_trial;
+        const double rho = F.predicted > 0.0 ? (S_before - S_trial) / F.predicted : 0.0;
+        const double c = 2.0 * rho - 1.0;
+        F.lambda *= fmax(1.0 / 3.0, 1.0 - c * c * c);
+        F.nu = 2.0;
+        F.lambda = fmin(fmax(F.lambda, kLambdaMin), kLambdaMax);
+        if (S_before - S_trial <= 1e-14 * S_before) F.done = true;
+        return true;
+    }
+    F.lambda = fmin(F.lambda * F.nu, kLambdaMax);
+    F.nu *= 2.0;
+    return false;
+}
+
+// Sums of one sweep: family I needs the moments of w u^2 and w u (u = 1/q^2, J = (-u x^2, -u x, -u, 1)),
+// family II those of w e^2 and w e (J = (e, -x e, 1)).
+struct SweepSums {
+    double m0, m1, m2, m3, m4, n0, n1, n2, h0, h1, h2, gd, sI;   // family I
+    double e0, e1, e2, f0, f1, k0, k1, gc, sII;                  // family II
+    int feasible;                                                // family I: every denominator positive
+};
+
+// One sweep over the window: both families at once, each at its own point (pI, pII).
+// doI / doII: per lane, whether that family is evaluated.
+__device__ __forceinline__ void sweep(const Lanes& S, int H, int k_all, double inv_span, const double (&pI)[4],
+                                      bool doI, const double (&pII)[4], bool doII, SweepSums& out) {
+    double m0 = 0, m1 = 0, m2 = 0, m3 = 0, m4 = 0, n0 = 0, n1 = 0, n2 = 0, h0 = 0, h1 = 0, h2 = 0, gd = 0, sI = 0;
+    double e0 = 0, e1 = 0, e2 = 0, f0 = 0, f1 = 0, k0 = 0, k1 = 0, gc = 0, sII = 0;
+    int feasible = 1;
+    // e = exp(alpha - beta x) with x = -m / span grows geometrically with m: one exact value at
+    // the lane's newest point, then a constant ratio per step.  The rounding of the recurrence
+    // accumulates towards the old points, whose weights gamma^m have long vanished.
+    double e = 0.0, ratio = 1.0;
+    if (doII) {
+        e = exp(fma(pII[1], (double)S.l * inv_span, pII[0]));
+        ratio = exp(pII[1] * ((double)S.L * inv_span));
+    }
+    double md = (double)S.l;
+    const double dL = (double)S.L;
+    for (int k = 0; k < k_all; ++k, md += dL) {
+        const int m = S.l + S.L * k;
+        if (m < H) {
+            const double x = -md * inv_span;
+            const double w = S.wtab[m];
+            const double y = S.y[k * 32 + S.lane];
+            const double x2 = x * x;
+            if (doI) {
+                const double q = fma(fma(pI[0], x, pI[1]), x, pI[2]);
+                feasible &= q > 0.0 ? 1 : 0;
+                const double inv = fast_rcp(q);
+                const double r = y - (inv + pI[3]);
+                const double u = inv * inv;
+                const double wu = w * u, wuu = wu * u, wur = wu * r, wr = w * r;
+                const double t = wuu * x2;
+                m0 += wuu;
+                m1 = fma(wuu, x, m1);
+                m2 += t;
+                m3 = fma(t, x, m3);
+                m4 = fma(t, x2, m4);
+                n0 += wu;
+                n1 = fma(wu, x, n1);
+                n2 = fma(wu, x2, n2);
+                h0 += wur;
+                h1 = fma(wur, x, h1);
+                h2 = fma(wur, x2, h2);
+                gd += wr;
+                sI = fma(wr, r, sI);
+            }
+            if (doII) {
+                const double r = y - (e + pII[2]);
+                const double we = w * e, wee = we * e, wer = we * r, wr = w * r;
+                e0 += wee;
+                e1 = fma(wee, x, e1);
+                e2 = fma(wee, x2, e2);
+                f0 += we;
+                f1 = fma(we, x, f1);
+                k0 += wer;
+                k1 = fma(wer, x, k1);
+                gc += wr;
+                sII = fma(wr, r, sII);
+            }
+        }
+        e *= ratio;
+    }
+    for (int o = S.L >> 1; o > 0; o >>= 1) {
+        m0 += __shfl_xor_sync(kFull, m0, o); m1 += __shfl_xor_sync(kFull, m1, o);
+        m2 += __shfl_xor_sync(kFull, m2, o); m3 += __shfl_xor_sync(kFull, m3, o);
+        m4 += __shfl_xor_sync(kFull, m4, o); n0 += __shfl_xor_sync(kFull, n0, o);
+        n1 += __shfl_xor_sync(kFull, n1, o); n2 += __shfl_xor_sync(kFull, n2, o);
+        h0 += __shfl_xor_sync(kFull, h0, o); h1 += __shfl_xor_sync(kFull, h1, o);
+        h2 += __shfl_xor_sync(kFull, h2, o); gd += __shfl_xor_sync(kFull, gd, o);
+        sI += __shfl_xor_sync(kFull, sI, o);
+        e0 += __shfl_xor_sync(kFull, e0, o); e1 += __shfl_xor_sync(kFull, e1, o);
+        e2 += __shfl_xor_sync(kFull, e2, o); f0 += __shfl_xor_sync(kFull, f0, o);
+        f1 += __shfl_xor_sync(kFull, f1, o); k0 += __shfl_xor_sync(kFull, k0, o);
+        k1 += __shfl_xor_sync(kFull, k1, o); gc += __shfl_xor_sync(kFull, gc, o);
+        sII += __shfl_xor_sync(kFull, sII, o);
+        feasible &= __shfl_xor_sync(kFull, feasible, o);
+    }
+    out.m0 = m0; out.m1 = m1; out.m2 = m2; out.m3 = m3; out.m4 = m4; out.n0 = n0; out.n1 = n1; out.n2 = n2;
+    out.h0 = h0; out.h1 = h1; out.h2 = h2; out.gd = gd; out.sI = sI;
+    out.e0 = e0; out.e1 = e1; out.e2 = e2; out.f0 = f0; out.f1 = f1; out.k0 = k0; out.k1 = k1; out.gc = gc;
+    out.sII = sII;
+    out.feasible = feasible;
+}
+
+// The sums of the last accepted point live in the lane's shared-memory column between sweeps.
+__device__ __forceinline__ void park_I(const Lanes& S, const SweepSums& s) {
+    double* c = S.park + S.lane;
+    c[0 * 32] = s.m0; c[1 * 32] = s.m1; c[2 * 32] = s.m2; c[3 * 32] = s.m3; c[4 * 32] = s.m4;
+    c[5 * 32] = s.n0; c[6 * 32] = s.n1; c[7 * 32] = s.n2;
+    c[8 * 32] = s.h0; c[9 * 32] = s.h1; c[10 * 32] = s.h2; c[11 * 32] = s.gd;
+}
+__device__ __forceinline__ void park_II(const Lanes& S, const SweepSums& s) {
+    double* c = S.park + S.lane;
+    c[12 * 32] = s.e0; c[13 * 32] = s.e1; c[14 * 32] = s.e2; c[15 * 32] = s.f0; c[16 * 32] = s.f1;
+    c[17 * 32] = s.k0; c[18 * 32] = s.k1; c[19 * 32] = s.gc;
+}
+__device__ __forceinline__ void normal_eq_I(const Lanes& S, double sw, Sym4& A, double (&g)[4]) {
+    const double* c = S.park + S.lane;
+    A.a00 = c[4 * 32]; A.a01 = c[3 * 32]; A.a02 = c[2 * 32]; A.a11 = c[2 * 32]; A.a12 = c[1 * 32]; A.a22 = c[0 * 32];
+    A.a03 = -c[7 * 32]; A.a13 = -c[6 * 32]; A.a23 = -c[5 * 32]; A.a33 = sw;
+    g[0] = -c[10 * 32]; g[1] = -c[9 * 32]; g[2] = -c[8 * 32]; g[3] = c[11 * 32];
+}
+__device__ __forceinline__ void normal_eq_II(const Lanes& S, double sw, Sym4& A, double (&g)[4]) {
+    const double* c = S.park + S.lane;
+    A.a00 = c[12 * 32]; A.a01 = -c[13 * 32]; A.a11 = c[14 * 32]; A.a02 = c[15 * 32]; A.a12 = -c[16 * 32]; A.a22 = sw;
+    A.a03 = 0.0; A.a13 = 0.0; A.a23 = 0.0; A.a33 = 1.0;
+    g[0] = c[17 * 32]; g[1] = -c[18 * 32]; g[2] = c[19 * 32]; g[3] = 0.0;
+}
+__device__ __forceinline__ bool sums_finite_I(const SweepSums& s) {
+    return finite_d(s.m0 + s.m1 + s.m2 + s.m3 + s.m4 + s.n0 + s.n1 + s.n2 + s.h0 + s.h1 + s.h2 + s.gd + s.sI);
+}
+__device__ __forceinline__ bool sums_finite_II(const SweepSums& s) {
+    return finite_d(s.e0 + s.e1 + s.e2 + s.f0 + s.f1 + s.k0 + s.k1 + s.gc + s.sII);
 }
 
 struct Moments {
-    double sw, swx, swx2, swx3, swx4, swy2, ymin, ymax;
+    double sw, swy2;
 };
 
-__device__ Moments window_moments(const Window& W) {
-    Moments m = {0, 0, 0, 0, 0, 0, CUDART_INF, -CUDART_INF};
-    for (int i = W.lane; i < W.H; i += 32) {
-        const double x = (double)(i - (W.H - 1)) * W.inv_span;
-        const double w = W.wtab[W.H - 1 - i];
-        const double y = W.y[i];
-        const double wx = w * x, wx2 = wx * x;
-        m.sw += w;
-        m.swx += wx;
-        m.swx2 += wx2;
-        m.swx3 = fma(wx2, x, m.swx3);
-        m.swx4 = fma(wx2 * x, x, m.swx4);
-        m.swy2 = fma(w * y, y, m.swy2);
-        m.ymin = fmin(m.ymin, y);
-        m.ymax = fmax(m.ymax, y);
-    }
-    m.sw = warp_sum(m.sw); m.swx = warp_sum(m.swx); m.swx2 = warp_sum(m.swx2);
-    m.swx3 = warp_sum(m.swx3); m.swx4 = warp_sum(m.swx4); m.swy2 = warp_sum(m.swy2);
-    m.ymin = warp_min(m.ymin); m.ymax = warp_max(m.ymax);
-    return m;
-}
-
-// Offset below every level; both families are linearised around it for their first guess.
-__device__ double floor_guess(const Moments& m) {
-    if (m.ymax > m.ymin) return m.ymin - 0.1 * (m.ymax - m.ymin);
-    return m.ymin - 1e-3 * fmax(fabs(m.ymin), 1.0);
-}
-
-// Family I: with d fixed, 1/(y - d) is a quadratic in x: weighted linear least squares.
-__device__ void init_sublinear(const Window& W, const Moments& m, double (&p)[4]) {
-    const double d0 = floor_guess(m);
-    double r0 = 0, r1 = 0, r2 = 0;
-    for (int i = W.lane; i < W.H; i += 32) {
-        const double x = (double)(i - (W.H - 1)) * W.inv_span;
-        const double w = W.wtab[W.H - 1 - i];
-        const double wz = w / (W.y[i] - d0);
-        r2 += wz;
-        r1 = fma(wz, x, r1);
-        r0 = fma(wz * x, x, r0);
-    }
-    r0 = warp_sum(r0); r1 = warp_sum(r1); r2 = warp_sum(r2);
-    double B[4][4] = {{m.swx4, m.swx3, m.swx2, 0}, {m.swx3, m.swx2, m.swx, 0}, {m.swx2, m.swx, m.sw, 0}, {0, 0, 0, 1}};
-    double rhs[4] = {r0, r1, r2, 0}, sol[4] = {0, 0, 0, 0};
-    bool good = chol_solve<3>(B, rhs, sol) && sol[0] >= 0.0 && sol[1] >= 0.0;
-    if (good) {
-        bool pos = true;
-        for (int i = W.lane; i < W.H; i += 32) {
-            const double x = (double)(i - (W.H - 1)) * W.inv_span;
-            pos = pos && (fma(fma(sol[0], x, sol[1]), x, sol[2]) > 0.0);
+// First guesses.  d0 lies below every level; with the offset fixed at d0, 1/(y - d0) is a
+// quadratic in x (family I: weighted linear least squares, or the line through the oldest and
+// newest transformed points if that fit is not a decreasing curve with a positive denominator)
+// and log(y - d0) is a line in x (family II: weighted linear regression).
+__device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span, double ymin, double ymax, bool busy,
+                              Moments& mom, double (&pI)[4], double (&pII)[4]) {
+    const double d0 = ymax > ymin ? ymin - 0.1 * (ymax - ymin) : ymin - 1e-3 * fmax(fabs(ymin), 1.0);
+    double sw = 0, swx = 0, swx2 = 0, swx3 = 0, swx4 = 0, swy2 = 0, r0 = 0, r1 = 0, r2 = 0, su = 0, sxu = 0;
+    double md = (double)S.l;
+    for (int k = 0; k < k_all; ++k, md += (double)S.L) {
+        const int m = S.l + S.L * k;
+        if (busy && m < H) {
+            const double x = -md * inv_span;
+            const double w = S.wtab[m];
+            const double y = S.y[k * 32 + S.lane];
+            const double wx = w * x, wx2 = wx * x;
+            sw += w;
+            swx += wx;
+            swx2 += wx2;
+            swx3 = fma(wx2, x, swx3);
+            swx4 = fma(wx2 * x, x, swx4);
+            swy2 = fma(w * y, y, swy2);
+            const double wz = w / (y - d0);
+            r2 += wz;
+            r1 = fma(wz, x, r1);
+            r0 = fma(wz * x, x, r0);
+            const double wu = w * log(y - d0);
+            su += wu;
+            sxu = fma(wu, x, sxu);
         }
-        good = __all_sync(kFull, pos);
     }
+    for (int o = S.L >> 1; o > 0; o >>= 1) {
+        sw += __shfl_xor_sync(kFull, sw, o); swx += __shfl_xor_sync(kFull, swx, o);
+        swx2 += __shfl_xor_sync(kFull, swx2, o); swx3 += __shfl_xor_sync(kFull, swx3, o);
+        swx4 += __shfl_xor_sync(kFull, swx4, o); swy2 += __shfl_xor_sync(kFull, swy2, o);
+        r0 += __shfl_xor_sync(kFull, r0, o); r1 += __shfl_xor_sync(kFull, r1, o);
+        r2 += __shfl_xor_sync(kFull, r2, o); su += __shfl_xor_sync(kFull, su, o);
+        sxu += __shfl_xor_sync(kFull, sxu, o);
+    }
+    mom.sw = sw;
+    mom.swy2 = swy2;
+    // family I
+    Sym4 B;
+    B.a00 = swx4; B.a01 = swx3; B.a02 = swx2; B.a11 = swx2; B.a12 = swx; B.a22 = sw;
+    B.a03 = B.a13 = B.a23 = 0.0; B.a33 = 1.0;
+    const double rhs[4] = {r0, r1, r2, 0.0};
+    double sol[4] = {0.0, 0.0, 0.0, 0.0};
+    bool good = busy && ldl_solve(B, rhs, sol) && sol[0] >= 0.0 && sol[1] >= 0.0;
+    int pos = 1;
+    md = (double)S.l;
+    for (int k = 0; k < k_all; ++k, md += (double)S.L) {
+        const int m = S.l + S.L * k;
+        if (busy && m < H) {
+            const double x = -md * inv_span;
+            pos &= fma(fma(sol[0], x, sol[1]), x, sol[2]) > 0.0 ? 1 : 0;
+        }
+    }
+    pos = group_and(pos, S.L);
+    good = good && pos;
+    // the oldest point (m = H - 1) and the newest (m = 0), read from the lanes that own them
+    const int m_old = max(H - 1, 0);
+    const double y_old = S.y[(m_old / S.L) * 32 + (S.lane - S.l) + (m_old & (S.L - 1))];
+    const double y_new = S.y[S.lane - S.l];
     if (good) {
-        p[0] = sol[0]; p[1] = sol[1]; p[2] = sol[2];
-    } else {   // straight line through the oldest and newest transformed points
-        const double z_old = 1.0 / (W.y[0] - d0), z_new = 1.0 / (W.y[W.H - 1] - d0);
-        p[0] = 0.0;
-        p[1] = fmax(z_new - z_old, 0.0);
-        p[2] = z_new;
+        pI[0] = sol[0]; pI[1] = sol[1]; pI[2] = sol[2];
+    } else {
+        const double z_old = 1.0 / (y_old - d0), z_new = 1.0 / (y_new - d0);
+        pI[0] = 0.0;
+        pI[1] = fmax(z_new - z_old, 0.0);
+        pI[2] = z_new;
     }
-    p[3] = d0;
+    pI[3] = d0;
+    // family II
+    const double den = sw * swx2 - swx * swx;
+    const double slope = (sw * sxu - swx * su) / den;
+    pII[0] = (su - slope * swx) / sw;
+    pII[1] = fmax(-slope, 1e-8);
+    pII[2] = d0;
+    pII[3] = 0.0;
 }
 
-// Family II: with c fixed, log(y - c) is a line in x.
-__device__ void init_exponential(const Window& W, const Moments& m, double (&p)[4]) {
-    const double d0 = floor_guess(m);
-    double su = 0, sxu = 0;
-    for (int i = W.lane; i < W.H; i += 32) {
-        const double x = (double)(i - (W.H - 1)) * W.inv_span;
-        const double w = W.wtab[W.H - 1 - i];
-        const double wu = w * log(W.y[i] - d0);
-        su += wu;
-        sxu = fma(wu, x, sxu);
-    }
-    su = warp_sum(su); sxu = warp_sum(sxu);
-    const double den = m.sw * m.swx2 - m.swx * m.swx;
-    const double slope = (m.sw * sxu - m.swx * su) / den;
-    p[0] = (su - slope * m.swx) / m.sw;
-    p[1] = fmax(-slope, 1e-8);
-    p[2] = d0;
-    p[3] = 0.0;
-}
+struct ClassRange {
+    int h_lo, h_hi;     // jobs with h_lo < H <= h_hi
+    int L, k_cap;       // lanes per job, sweeps a lane makes at most (ceil(h_hi / L))
+};
 
-__global__ void __launch_bounds__(kMaxWarpsPerBlock * 32)
+__global__ void __launch_bounds__(kMaxWarpsPerBlock * 32, 4)
 fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, const int32_t* __restrict__ order,
-           int n_work, int max_hist, int lm_trials, int min_fit_points, unsigned int* queue, long long* counters,
-           int32_t* err_word) {
+           const int32_t* __restrict__ start, ClassRange cls, int lm_trials, int min_fit_points, unsigned int* queue,
+           long long* counters, int32_t* err_word) {
     extern __shared__ double smem[];
-    double* wtab = smem;                                   // [max_hist]
+    double* wtab = smem;                                   // [h_hi]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    double* win = smem + max_hist + (size_t)warp * max_hist;   // this warp's window
-    for (int i = threadIdx.x; i < max_hist; i += blockDim.x) wtab[i] = g_wtab[i];
+    const size_t per_warp = (size_t)(cls.k_cap + 1) * 32 + kParked * 32;   // one spare row for neighbour reads
+    Lanes S;
+    S.y = smem + cls.h_hi + warp * per_warp;
+    S.park = S.y + (size_t)(cls.k_cap + 1) * 32;
+    S.wtab = wtab;
+    S.lane = lane;
+    S.L = cls.L;
+    S.l = lane & (cls.L - 1);
+    for (int i = threadIdx.x; i < cls.h_hi; i += blockDim.x) wtab[i] = g_wtab[i];
     __syncthreads();
+    const int G = 32 / cls.L, g = lane / cls.L;
+    const int first = start[cls.h_hi], last = start[cls.h_lo];   // this class: order[first .. last)
 
     long long n_points = 0, n_sweep_points = 0;
     int n_fit = 0, n_sub = 0, n_exp = 0, n_fallback = 0;
@@ -466,84 +562,120 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         int slot = 0;
         if (lane == 0) slot = (int)atomicAdd(queue, 1u);
         slot = __shfl_sync(kFull, slot, 0);
-        if (slot >= n_work) break;
-        const int j = order ? order[slot] : slot;
-        const int H = stage_window(job, j, max_hist, win, lane, err_word);
+        const int base = first + slot * G;
+        if (base >= last) break;
+        const int idx = base + g;
+        const int j = idx < last ? order[idx] : -1;
+        __syncwarp();
+        const int H = stage_window(job, j, cls.h_hi, S, err_word);
+        const int k_all = warp_max_int((H + cls.L - 1) / cls.L);
+        __syncwarp();
+        const double m_seen = j >= 0 ? job.m_seen[j] : -CUDART_INF;
+        const Normalised nz = normalise_window(S, H, k_all, m_seen, nullptr);
 
-        int status = SLAQ_JOB_INACTIVE, family = -1;
+        int status = nz.status, family = -1;
         double p_out[4] = {CUDART_NAN, CUDART_NAN, CUDART_NAN, CUDART_NAN};
         double S_out[2] = {CUDART_INF, CUDART_INF};
-        int sweeps[2] = {0, 0};
-        double M = CUDART_NAN;
+        int sweeps_out[2] = {0, 0};
         const double span = (double)max(H - 1, 1);
-        if (H > 0) {
-            const Normalised nz = normalise_window(win, H, job.m_seen[j], wtab, lane, nullptr);
-            status = nz.status;
-            M = nz.M;
-            n_points += H;
-            if (status == SLAQ_JOB_NEW) {
-                p_out[0] = 1.0;   // one normalised unit per iteration
-                p_out[1] = 1.0;   // at most the whole normalised loss
-            } else if (status == SLAQ_JOB_FITTED) {
-                bool fitted = false;
-                if (H >= min_fit_points) {
-                    Window W = {win, wtab, H, lane, 1.0 / span, 0.0};
-                    const Moments mom = window_moments(W);
-                    W.sw = mom.sw;
-                    double pI[4], pII[4];
-                    init_sublinear(W, mom, pI);
-                    const LmResult rI = levenberg_marquardt<Sublinear>(W, pI, lm_trials, mom.swy2);
-                    init_exponential(W, mom, pII);
-                    const LmResult rII = levenberg_marquardt<Exponential>(W, pII, lm_trials, mom.swy2);
-                    sweeps[0] = rI.sweeps;
-                    sweeps[1] = rII.sweeps;
-                    if (rI.ok) S_out[0] = rI.S;
-                    if (rII.ok) S_out[1] = rII.S;
-                    const bool okI = rI.ok && finite_d(rI.S), okII = rII.ok && finite_d(rII.S);
-                    if (okI && (!okII || rI.S <= rII.S)) {   // a tie goes to family I
-                        family = 0;
+        const bool fits = status == SLAQ_JOB_FITTED && H >= min_fit_points;   // this lane's job gets curves fitted
+
+        if (__any_sync(kFull, fits)) {
+            const double inv_span = 1.0 / span;
+            Moments mom;
+            Family I, II;
+            first_guesses(S, H, k_all, inv_span, nz.ymin, nz.ymax, fits, mom, I.p, II.p);
+            SweepSums sums;
+            sweep(S, H, k_all, inv_span, I.p, fits, II.p, fits, sums);
+            I.ok = fits && sums.feasible && sums_finite_I(sums);
+            II.ok = fits && sums_finite_II(sums);
+            I.S = sums.sI; II.S = sums.sII;
+            I.lambda = II.lambda = kLambda0;
+            I.nu = II.nu = 2.0;
+            I.was_frozen = II.was_frozen = 0;
+            I.sweeps = II.sweeps = fits ? 1 : 0;
+            I.done = !I.ok; II.done = !II.ok;
+            I.has_trial = II.has_trial = false;
+            I.predicted = II.predicted = 0.0;
 #pragma unroll
-                        for (int a = 0; a < 4; ++a) p_out[a] = pI[a];
-                        fitted = true;
-                    } else if (okII) {
-                        family = 1;
-#pragma unroll
-                        for (int a = 0; a < 4; ++a) p_out[a] = pII[a];
-                        fitted = true;
-                    }
-                    n_sweep_points += (long long)H * (rI.sweeps + rII.sweeps);
+            for (int a = 0; a < 4; ++a) I.trial[a] = II.trial[a] = 0.0;
+            park_I(S, sums);
+            park_II(S, sums);
+            for (int t = 0; t < lm_trials; ++t) {
+                if (!__any_sync(kFull, !I.done || !II.done)) break;
+                {
+                    Sym4 A;
+                    double gr[4];
+                    normal_eq_I(S, mom.sw, A, gr);
+                    prepare_trial<4>(I, A, gr, !I.done, mom.swy2);
+                    normal_eq_II(S, mom.sw, A, gr);
+                    prepare_trial<3>(II, A, gr, !II.done, mom.swy2);
                 }
-                if (!fitted) {
-                    status = H >= min_fit_points ? SLAQ_JOB_FIT_FAILED : SLAQ_JOB_SHORT;
-                    const double y_new = win[H - 1];
-                    p_out[0] = nz.rho;
-                    p_out[1] = y_new > 0.0 ? y_new : CUDART_INF;
-                    p_out[2] = p_out[3] = CUDART_NAN;
+                if (!__any_sync(kFull, I.has_trial || II.has_trial)) continue;
+                sweep(S, H, k_all, inv_span, I.trial, I.has_trial, II.trial, II.has_trial, sums);
+                if (finish_trial(I, sums.feasible && sums_finite_I(sums), sums.sI)) park_I(S, sums);
+                if (finish_trial(II, sums_finite_II(sums), sums.sII)) park_II(S, sums);
+            }
+            if (fits) {
+                sweeps_out[0] = I.sweeps;
+                sweeps_out[1] = II.sweeps;
+                if (I.ok) S_out[0] = I.S;
+                if (II.ok) S_out[1] = II.S;
+                const bool okI = I.ok && finite_d(I.S), okII = II.ok && finite_d(II.S);
+                if (okI && (!okII || I.S <= II.S)) {   // a tie goes to family I
+                    family = 0;
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) p_out[a] = I.p[a];
+                } else if (okII) {
+                    family = 1;
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) p_out[a] = II.p[a];
                 }
             }
         }
-        if (status == SLAQ_JOB_FITTED) {
-            n_fit += 1;
-            n_sub += family == 0;
-            n_exp += family == 1;
-        } else if (status == SLAQ_JOB_SHORT || status == SLAQ_JOB_NEW || status == SLAQ_JOB_FIT_FAILED) {
-            n_fallback += 1;
+        if (status == SLAQ_JOB_NEW) {
+            p_out[0] = 1.0;   // one normalised unit per iteration
+            p_out[1] = 1.0;   // at most the whole normalised loss
+        } else if (status == SLAQ_JOB_FITTED && family < 0) {
+            status = H >= min_fit_points ? SLAQ_JOB_FIT_FAILED : SLAQ_JOB_SHORT;
+            const double y_new = S.y[lane - S.l];
+            p_out[0] = nz.rho;
+            p_out[1] = y_new > 0.0 ? y_new : CUDART_INF;
+            p_out[2] = p_out[3] = CUDART_NAN;
         }
-        if (lane == 0) {
+        if (S.l == 0 && H > 0) {
+            n_points += H;
+            n_sweep_points += (long long)H * (sweeps_out[0] + sweeps_out[1]);
+            if (status == SLAQ_JOB_FITTED) {
+                n_fit += 1;
+                n_sub += family == 0;
+                n_exp += family == 1;
+            } else if (status == SLAQ_JOB_SHORT || status == SLAQ_JOB_NEW || status == SLAQ_JOB_FIT_FAILED) {
+                n_fallback += 1;
+            }
             fit.status[j] = status;
             fit.family[j] = (int8_t)family;
 #pragma unroll
             for (int a = 0; a < 4; ++a) fit.params[4 * (size_t)j + a] = p_out[a];
             fit.residual[2 * (size_t)j] = S_out[0];
             fit.residual[2 * (size_t)j + 1] = S_out[1];
-            fit.sweeps[2 * (size_t)j] = sweeps[0];
-            fit.sweeps[2 * (size_t)j + 1] = sweeps[1];
-            fit.largest[j] = M;
+            fit.sweeps[2 * (size_t)j] = sweeps_out[0];
+            fit.sweeps[2 * (size_t)j + 1] = sweeps_out[1];
+            fit.largest[j] = nz.M;
             fit.span[j] = span;
         }
         __syncwarp();
     }
-    if (lane == 0) {
+    // per-warp totals of the statistics
+    for (int o = 16; o > 0; o >>= 1) {
+        n_points += __shfl_xor_sync(kFull, n_points, o);
+        n_sweep_points += __shfl_xor_sync(kFull, n_sweep_points, o);
+        n_fit += __shfl_xor_sync(kFull, n_fit, o);
+        n_sub += __shfl_xor_sync(kFull, n_sub, o);
+        n_exp += __shfl_xor_sync(kFull, n_exp, o);
+        n_fallback += __shfl_xor_sync(kFull, n_fallback, o);
+    }
+    if (lane == 0 && n_points > 0) {
         atomicAdd((unsigned long long*)&counters[0], (unsigned long long)n_points);
         atomicAdd((unsigned long long*)&counters[1], (unsigned long long)n_sweep_points);
         atomicAdd((unsigned long long*)&counters[2], (unsigned long long)n_fit);
@@ -553,7 +685,8 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
     }
 }
 
-// Normalisation only, written out for inspection: same staging and scaling code as the fit.
+// Normalisation only, written out for inspection: same staging and scaling code as the fit,
+// one warp per listed job.
 __global__ void __launch_bounds__(kMaxWarpsPerBlock * 32)
 normalise_export_kernel(JobArrays job, const int32_t* __restrict__ ids, const int64_t* __restrict__ offsets, int n,
                         const double* __restrict__ g_wtab, int max_hist, double* changes, double* levels,
@@ -561,74 +694,173 @@ normalise_export_kernel(JobArrays job, const int32_t* __restrict__ ids, const in
     extern __shared__ double smem[];
     double* wtab = smem;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    double* win = smem + max_hist + (size_t)warp * max_hist;
+    const int k_cap = (max_hist + 31) / 32;
+    Lanes S;
+    S.y = smem + max_hist + (size_t)warp * (k_cap + 1) * 32;
+    S.park = nullptr;
+    S.wtab = wtab;
+    S.lane = lane;
+    S.L = 32;
+    S.l = lane;
     for (int i = threadIdx.x; i < max_hist; i += blockDim.x) wtab[i] = g_wtab[i];
     __syncthreads();
     const int slot = blockIdx.x * (blockDim.x >> 5) + warp;
     if (slot >= n) return;
     const int j = ids[slot];
-    const int H = stage_window(job, j, max_hist, win, lane, err_word);
+    const int H = stage_window(job, j, max_hist, S, err_word);
+    __syncwarp();
     if (H <= 0) {
         if (lane == 0 && largest) largest[slot] = CUDART_NAN;
         return;
     }
     const int64_t base = offsets[slot];
-    const Normalised nz = normalise_window(win, H, job.m_seen[j], wtab, lane, changes ? changes + base : nullptr);
+    const int k_all = (H + 31) / 32;
+    const Normalised nz = normalise_window(S, H, k_all, job.m_seen[j], changes ? changes + base : nullptr);
     if (lane == 0 && largest) largest[slot] = nz.M;
-    if (nz.status != SLAQ_JOB_FITTED) {   // nothing was scaled: report NaN levels and changes
-        for (int i = lane; i < H; i += 32) {
-            if (levels) levels[base + i] = CUDART_NAN;
-            if (changes) changes[base + i] = CUDART_NAN;
+    for (int k = 0; k < k_all; ++k) {
+        const int m = lane + 32 * k;
+        if (m < H) {
+            if (nz.status != SLAQ_JOB_FITTED) {   // nothing was scaled: report NaN levels and changes
+                if (levels) levels[base + H - 1 - m] = CUDART_NAN;
+                if (changes) changes[base + H - 1 - m] = CUDART_NAN;
+            } else if (levels) {
+                levels[base + H - 1 - m] = S.y[k * 32 + lane];
+            }
         }
-        return;
     }
-    if (levels)
-        for (int i = lane; i < H; i += 32) levels[base + i] = win[i];
 }
 
-size_t fit_smem_bytes(int32_t max_hist, int warps) { return sizeof(double) * (size_t)max_hist * (warps + 1); }
+// ---- work list: job ids sorted by window length, longest first (counting sort) ----
 
-// Warps per block: as many as fit beside the weight table, each with a whole window.
-int warps_for(int32_t max_hist) {
-    int warps = kMaxWarpsPerBlock;
-    while (warps > 1 && fit_smem_bytes(max_hist, warps) > kSmemLimit) --warps;
-    return warps;
+__global__ void length_count_kernel(const int32_t* __restrict__ count, int max_jobs, int max_hist, int32_t* bucket) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= max_jobs) return;
+    int H = count[j];
+    H = H < 0 ? 0 : (H > max_hist ? max_hist : H);
+    atomicAdd(&bucket[H], 1);
+}
+
+// start[h] = number of jobs with a window longer than h (h = 0..max_hist); cursor = copy for the scatter.
+__global__ void __launch_bounds__(1024) length_scan_kernel(const int32_t* __restrict__ bucket, int max_hist,
+                                                           int32_t* start, int32_t* cursor) {
+    __shared__ int sh[1024];
+    const int t = threadIdx.x, n = max_hist + 1;
+    const int per = (n + 1023) / 1024;
+    // thread t owns lengths h = max_hist - (t * per + i): it walks from the longest down
+    int sum = 0;
+    for (int i = 0; i < per; ++i) {
+        const int h = max_hist - (t * per + i);
+        if (h >= 0) sum += bucket[h];
+    }
+    sh[t] = sum;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {
+        const int v = t >= o ? sh[t - o] : 0;
+        __syncthreads();
+        sh[t] += v;
+        __syncthreads();
+    }
+    int run = sh[t] - sum;   // jobs longer than this thread's first length
+    for (int i = 0; i < per; ++i) {
+        const int h = max_hist - (t * per + i);
+        if (h < 0) break;
+        start[h] = run;
+        cursor[h] = run;
+        run += bucket[h];
+    }
+}
+
+__global__ void length_scatter_kernel(const int32_t* __restrict__ count, int max_jobs, int max_hist, int32_t* cursor,
+                                      int32_t* order) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= max_jobs) return;
+    int H = count[j];
+    H = H < 0 ? 0 : (H > max_hist ? max_hist : H);
+    order[atomicAdd(&cursor[H], 1)] = j;
+}
+
+size_t fit_smem_bytes(const ClassRange& c, int warps) {
+    return sizeof(double) * ((size_t)c.h_hi + (size_t)warps * ((size_t)(c.k_cap + 1) * 32 + kParked * 32));
+}
+
+// Lanes per job for windows up to h_hi points: the smallest group whose warp slice stays
+// within `budget` bytes of shared memory.
+int lanes_for(int h_hi, size_t budget) {
+    for (int L = 1; L <= 32; L <<= 1) {
+        const size_t slice = sizeof(double) * ((size_t)((h_hi + L - 1) / L + 1) * 32 + kParked * 32);
+        if (slice <= budget) return L;
+    }
+    return 32;
 }
 
 }  // namespace
 
 int launch_fit(slaq_handle* h) {
-    const int warps = warps_for(h->max_hist);
-    const size_t smem = fit_smem_bytes(h->max_hist, warps);
-    cudaError_t e = cudaFuncSetAttribute(fit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaStream_t st = h->stream;
+    const int J = h->max_jobs, Hmax = h->max_hist;
+    int launches = 0;
+    // work list
+    {
+        const int threads = 256, blocks = (J + threads - 1) / threads;
+        length_count_kernel<<<blocks, threads, 0, st>>>(h->job.count, J, Hmax, h->scratch.bucket);
+        length_scan_kernel<<<1, 1024, 0, st>>>(h->scratch.bucket, Hmax, h->scratch.start, h->scratch.cursor);
+        length_scatter_kernel<<<blocks, threads, 0, st>>>(h->job.count, J, Hmax, h->scratch.cursor, h->scratch.order);
+        launches += 3;
+    }
+    cudaError_t e = cudaFuncSetAttribute(fit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
     if (e != cudaSuccess) {
         h->err = std::string("fit kernel shared memory: ") + cudaGetErrorString(e);
         return -1;
     }
-    int per_sm = 1;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fit_kernel, warps * 32, smem);
-    if (per_sm < 1) per_sm = 1;
-    const int n_work = h->max_jobs;
-    int blocks = h->sm_count * per_sm;
-    const int needed = (n_work + warps - 1) / warps;
-    if (blocks > needed) blocks = needed;
-    if (blocks < 1) blocks = 1;
-    fit_kernel<<<blocks, warps * 32, smem, h->stream>>>(
-        h->job, h->fit, h->wtab, nullptr, n_work, h->max_hist, h->lm_trials, h->min_fit_points,
-        h->scratch.ticket, h->scratch.counters, h->err_word);
+    // length classes, longest first: (max_hist/2, max_hist], (max_hist/4, max_hist/2], ... then (0, 64 or less]
+    int h_hi = Hmax, cls_index = 0;
+    while (h_hi > 0) {
+        int h_lo = h_hi > 64 ? (h_hi + 1) / 2 : 0;
+        if (cls_index == kMaxFitClasses - 1) h_lo = 0;
+        ClassRange c;
+        c.h_lo = h_lo;
+        c.h_hi = h_hi;
+        c.L = lanes_for(h_hi, h->fit_slice_bytes);
+        c.k_cap = (h_hi + c.L - 1) / c.L;
+        int warps = kMaxWarpsPerBlock;
+        while (warps > 1 && fit_smem_bytes(c, warps) > kSmemLimit) --warps;
+        const size_t smem = fit_smem_bytes(c, warps);
+        if (smem > kSmemLimit) {
+            h->err = "fit kernel: a window does not fit in shared memory";
+            return -1;
+        }
+        int per_sm = 1;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fit_kernel, warps * 32, smem);
+        if (per_sm < 1) per_sm = 1;
+        const int G = 32 / c.L;
+        int blocks = h->sm_count * per_sm;
+        const int needed = (J + warps * G - 1) / (warps * G);
+        if (blocks > needed) blocks = needed;
+        if (blocks < 1) blocks = 1;
+        fit_kernel<<<blocks, warps * 32, smem, st>>>(h->job, h->fit, h->wtab, h->scratch.order, h->scratch.start, c,
+                                                    h->lm_trials, h->min_fit_points,
+                                                    h->scratch.ticket + kFitQueueBase + cls_index, h->scratch.counters,
+                                                    h->err_word);
+        ++launches;
+        ++cls_index;
+        h_hi = h_lo;
+    }
     e = cudaGetLastError();
     if (e != cudaSuccess) {
         h->err = std::string("fit kernel launch: ") + cudaGetErrorString(e);
         return -1;
     }
-    return 1;
+    return launches;
 }
 
 int launch_normalise_export(slaq_handle* h, int32_t n, const int64_t* d_offsets, double* d_changes,
                             double* d_levels, double* d_largest) {
     if (n <= 0) return 0;
-    const int warps = warps_for(h->max_hist);
-    const size_t smem = fit_smem_bytes(h->max_hist, warps);
+    const int k_cap = (h->max_hist + 31) / 32;
+    int warps = kMaxWarpsPerBlock;
+    auto bytes = [&](int w) { return sizeof(double) * ((size_t)h->max_hist + (size_t)w * (k_cap + 1) * 32); };
+    while (warps > 1 && bytes(warps) > kSmemLimit) --warps;
+    const size_t smem = bytes(warps);
     cudaError_t e =
         cudaFuncSetAttribute(normalise_export_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) {

@@ -16,6 +16,9 @@ constexpr int kMaxCoresLimit = 1024;
 constexpr int kRadixBits = 11;
 constexpr int kRadixBins = 1 << kRadixBits;
 constexpr int kRadixPasses = 6;       // 11 + 11 + 11 + 11 + 11 + 9 bits, most significant first
+constexpr int kMaxFitClasses = 8;     // window-length classes of the fit (one launch each)
+constexpr int kFitQueueBase = 8;      // ticket[kFitQueueBase + c]: work queue head of class c
+constexpr int kTickets = 16;
 
 // Device-side state of one job, structure of arrays (index = job id).
 struct JobArrays {
@@ -52,15 +55,17 @@ struct SelectState {
 // Scratch of one epoch; [hist, hist + zero_bytes) is cleared at the start of every epoch.
 struct Scratch {
     unsigned long long* hist;        // [kRadixPasses][kRadixBins]
-    unsigned int* ticket;            // [8]: job queue head, then one block-completion counter per pass
+    unsigned int* ticket;            // [kTickets]: block-completion counter per radix pass, work queue per fit class
     SelectState* sel;
     long long* counters;             // [16] statistics accumulated by kernels
     size_t zero_bytes;
     int32_t* gt;                     // per job: candidate gains strictly above the threshold
     int32_t* eq;                     // per job: candidate gains equal to it
     long long* block_eq;             // per block of the count kernel: sum of eq
-    int32_t* order;                  // job ids, longest history first (fit kernel work list)
-    int32_t* bucket;                 // counting-sort buckets by history length
+    int32_t* bucket;                 // [max_hist + 1] jobs per window length (inside the cleared region)
+    int32_t* order;                  // job ids, longest window first (fit kernel work list)
+    int32_t* start;                  // [max_hist + 1] start[h] = jobs with a window longer than h
+    int32_t* cursor;                 // [max_hist + 1] scatter positions of the counting sort
 };
 
 struct Staging {
@@ -81,6 +86,7 @@ struct slaq_handle {
     int32_t max_cores = 64;
     double gamma = 0.9;
     int32_t lm_trials = 20, min_fit_points = 4;
+    size_t fit_slice_bytes = 16 * 1024;   // shared memory one warp of the fit kernel may use
     cudaStream_t stream = nullptr;
     bool owns_ws = false;
     void* ws = nullptr;
