@@ -8,14 +8,16 @@
 // (newest point x = 0, oldest x = -1); the family with the lower weighted residual wins.
 //
 // Work split.  Jobs are sorted by window length (counting sort, longest first) and cut into
-// length classes; one launch per class.  Inside a launch a group of L lanes (L = 1, 2, .. 32,
-// chosen per class so that a warp's windows fit its shared-memory slice) owns one job, so a
-// warp carries 32/L jobs.  A lane walks its job's points m = l, l + L, l + 2L, ... counted
+// length classes.  In class c a group of L lanes (L = 1, 2, .. 32, chosen so that a warp's
+// windows fit its shared-memory slice) owns one job, so a warp carries 32/L jobs.  One
+// persistent launch serves all classes from one work queue, longest windows first.  A lane walks its job's points m = l, l + L, l + 2L, ... counted
 // from the newest one; both families are evaluated in the same sweep over the window; the
 // partial sums of the normal equations are reduced over the L lanes with shuffles; every
 // lane of a group then runs the same small solve for its job.  All per-job control flow is
 // per lane, so the jobs of a warp may be in different phases of the solver.
 #include <math_constants.h>
+
+#include <algorithm>
 
 #include "slaq_internal.cuh"
 
@@ -24,7 +26,7 @@ namespace slaq {
 namespace {
 
 constexpr int kMaxWarpsPerBlock = 4;
-constexpr size_t kSmemLimit = 227 * 1024;   // shared memory one block may use on sm_100
+constexpr size_t kSmemLimit = 226 * 1024;   // shared memory one block may use on sm_100, less the static part
 constexpr unsigned kFull = 0xffffffffu;
 constexpr double kLambda0 = 1e-3, kLambdaMin = 1e-5, kLambdaMax = 1e12;
 constexpr int kParked = 20;                 // doubles per lane kept in shared memory between sweeps
@@ -531,30 +533,41 @@ __device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span,
     pII[3] = 0.0;
 }
 
-struct ClassRange {
-    int h_lo, h_hi;     // jobs with h_lo < H <= h_hi
-    int L, k_cap;       // lanes per job, sweeps a lane makes at most (ceil(h_hi / L))
+// Window-length classes, longest first: class c holds the jobs with h_lo[c] < H <= h_hi[c] and
+// gives each of them L[c] lanes.  All classes are served by one launch from one work queue
+// whose slots are numbered class by class, so the longest windows start first.
+struct FitClasses {
+    int n;
+    int h_lo[kMaxFitClasses], h_hi[kMaxFitClasses], L[kMaxFitClasses];
+    int rows;        // sweeps a lane makes at most, over all classes
+    int h_max;       // longest window
 };
 
 __global__ void __launch_bounds__(kMaxWarpsPerBlock * 32, 4)
 fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, const int32_t* __restrict__ order,
-           const int32_t* __restrict__ start, ClassRange cls, int lm_trials, int min_fit_points, unsigned int* queue,
+           const int32_t* __restrict__ start, FitClasses cls, int lm_trials, int min_fit_points, unsigned int* queue,
            long long* counters, int32_t* err_word) {
     extern __shared__ double smem[];
-    double* wtab = smem;                                   // [h_hi]
+    __shared__ int slot_base[kMaxFitClasses + 1];
+    double* wtab = smem;                                   // [h_max]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const size_t per_warp = (size_t)(cls.k_cap + 1) * 32 + kParked * 32;   // one spare row for neighbour reads
+    const size_t per_warp = (size_t)(cls.rows + 1) * 32 + kParked * 32;   // one spare row for neighbour reads
     Lanes S;
-    S.y = smem + cls.h_hi + warp * per_warp;
-    S.park = S.y + (size_t)(cls.k_cap + 1) * 32;
+    S.y = smem + cls.h_max + warp * per_warp;
+    S.park = S.y + (size_t)(cls.rows + 1) * 32;
     S.wtab = wtab;
     S.lane = lane;
-    S.L = cls.L;
-    S.l = lane & (cls.L - 1);
-    for (int i = threadIdx.x; i < cls.h_hi; i += blockDim.x) wtab[i] = g_wtab[i];
+    for (int i = threadIdx.x; i < cls.h_max; i += blockDim.x) wtab[i] = g_wtab[i];
+    if (threadIdx.x == 0) {   // queue slots of each class: one slot = one warp's worth of jobs
+        int run = 0;
+        for (int c = 0; c < cls.n; ++c) {
+            slot_base[c] = run;
+            const int jobs = start[cls.h_lo[c]] - start[cls.h_hi[c]], per_slot = 32 / cls.L[c];
+            run += (jobs + per_slot - 1) / per_slot;
+        }
+        for (int c = cls.n; c <= kMaxFitClasses; ++c) slot_base[c] = run;
+    }
     __syncthreads();
-    const int G = 32 / cls.L, g = lane / cls.L;
-    const int first = start[cls.h_hi], last = start[cls.h_lo];   // this class: order[first .. last)
 
     long long n_points = 0, n_sweep_points = 0;
     int n_fit = 0, n_sub = 0, n_exp = 0, n_fallback = 0;
@@ -562,13 +575,20 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         int slot = 0;
         if (lane == 0) slot = (int)atomicAdd(queue, 1u);
         slot = __shfl_sync(kFull, slot, 0);
-        const int base = first + slot * G;
-        if (base >= last) break;
+        if (slot >= slot_base[cls.n]) break;
+        int c = 0;
+        while (slot >= slot_base[c + 1]) ++c;
+        const int L = cls.L[c], h_hi = cls.h_hi[c];
+        S.L = L;
+        S.l = lane & (L - 1);
+        const int G = 32 / L, g = lane / L;
+        const int last = start[cls.h_lo[c]];
+        const int base = start[h_hi] + (slot - slot_base[c]) * G;
         const int idx = base + g;
         const int j = idx < last ? order[idx] : -1;
         __syncwarp();
-        const int H = stage_window(job, j, cls.h_hi, S, err_word);
-        const int k_all = warp_max_int((H + cls.L - 1) / cls.L);
+        const int H = stage_window(job, j, h_hi, S, err_word);
+        const int k_all = warp_max_int((H + L - 1) / L);
         __syncwarp();
         const double m_seen = j >= 0 ? job.m_seen[j] : -CUDART_INF;
         const Normalised nz = normalise_window(S, H, k_all, m_seen, nullptr);
@@ -779,8 +799,8 @@ __global__ void length_scatter_kernel(const int32_t* __restrict__ count, int max
     order[atomicAdd(&cursor[H], 1)] = j;
 }
 
-size_t fit_smem_bytes(const ClassRange& c, int warps) {
-    return sizeof(double) * ((size_t)c.h_hi + (size_t)warps * ((size_t)(c.k_cap + 1) * 32 + kParked * 32));
+size_t fit_smem_bytes(const FitClasses& c, int warps) {
+    return sizeof(double) * ((size_t)c.h_max + (size_t)warps * ((size_t)(c.rows + 1) * 32 + kParked * 32));
 }
 
 // Lanes per job for windows up to h_hi points: the smallest group whose warp slice stays
@@ -807,44 +827,46 @@ int launch_fit(slaq_handle* h) {
         length_scatter_kernel<<<blocks, threads, 0, st>>>(h->job.count, J, Hmax, h->scratch.cursor, h->scratch.order);
         launches += 3;
     }
-    cudaError_t e = cudaFuncSetAttribute(fit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+    // length classes, longest first: (max_hist/2, max_hist], (max_hist/4, max_hist/2], ... then (0, 64 or less]
+    FitClasses cls;
+    cls.n = 0;
+    cls.rows = 1;
+    cls.h_max = Hmax;
+    for (int h_hi = Hmax; h_hi > 0;) {
+        int h_lo = h_hi > 64 ? (h_hi + 1) / 2 : 0;
+        if (cls.n == kMaxFitClasses - 1) h_lo = 0;
+        const int L = lanes_for(h_hi, h->fit_slice_bytes);
+        cls.h_lo[cls.n] = h_lo;
+        cls.h_hi[cls.n] = h_hi;
+        cls.L[cls.n] = L;
+        cls.rows = std::max(cls.rows, (h_hi + L - 1) / L);
+        ++cls.n;
+        h_hi = h_lo;
+    }
+    for (int c = cls.n; c < kMaxFitClasses; ++c) cls.h_lo[c] = cls.h_hi[c] = 0, cls.L[c] = 32;
+    int warps = kMaxWarpsPerBlock;
+    while (warps > 1 && fit_smem_bytes(cls, warps) > kSmemLimit) --warps;
+    const size_t smem = fit_smem_bytes(cls, warps);
+    if (smem > kSmemLimit) {
+        h->err = "fit kernel: a window does not fit in shared memory";
+        return -1;
+    }
+    cudaError_t e = cudaFuncSetAttribute(fit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) {
         h->err = std::string("fit kernel shared memory: ") + cudaGetErrorString(e);
         return -1;
     }
-    // length classes, longest first: (max_hist/2, max_hist], (max_hist/4, max_hist/2], ... then (0, 64 or less]
-    int h_hi = Hmax, cls_index = 0;
-    while (h_hi > 0) {
-        int h_lo = h_hi > 64 ? (h_hi + 1) / 2 : 0;
-        if (cls_index == kMaxFitClasses - 1) h_lo = 0;
-        ClassRange c;
-        c.h_lo = h_lo;
-        c.h_hi = h_hi;
-        c.L = lanes_for(h_hi, h->fit_slice_bytes);
-        c.k_cap = (h_hi + c.L - 1) / c.L;
-        int warps = kMaxWarpsPerBlock;
-        while (warps > 1 && fit_smem_bytes(c, warps) > kSmemLimit) --warps;
-        const size_t smem = fit_smem_bytes(c, warps);
-        if (smem > kSmemLimit) {
-            h->err = "fit kernel: a window does not fit in shared memory";
-            return -1;
-        }
-        int per_sm = 1;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fit_kernel, warps * 32, smem);
-        if (per_sm < 1) per_sm = 1;
-        const int G = 32 / c.L;
-        int blocks = h->sm_count * per_sm;
-        const int needed = (J + warps * G - 1) / (warps * G);
-        if (blocks > needed) blocks = needed;
-        if (blocks < 1) blocks = 1;
-        fit_kernel<<<blocks, warps * 32, smem, st>>>(h->job, h->fit, h->wtab, h->scratch.order, h->scratch.start, c,
-                                                    h->lm_trials, h->min_fit_points,
-                                                    h->scratch.ticket + kFitQueueBase + cls_index, h->scratch.counters,
-                                                    h->err_word);
-        ++launches;
-        ++cls_index;
-        h_hi = h_lo;
-    }
+    int per_sm = 1;
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fit_kernel, warps * 32, smem);
+    if (per_sm < 1) per_sm = 1;
+    int blocks = h->sm_count * per_sm;
+    const int needed = (J + warps - 1) / warps;   // at least one job per slot
+    if (blocks > needed) blocks = needed;
+    if (blocks < 1) blocks = 1;
+    fit_kernel<<<blocks, warps * 32, smem, st>>>(h->job, h->fit, h->wtab, h->scratch.order, h->scratch.start, cls,
+                                                h->lm_trials, h->min_fit_points, h->scratch.ticket + kFitQueueBase,
+                                                h->scratch.counters, h->err_word);
+    ++launches;
     e = cudaGetLastError();
     if (e != cudaSuccess) {
         h->err = std::string("fit kernel launch: ") + cudaGetErrorString(e);
