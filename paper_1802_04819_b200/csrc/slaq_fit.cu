@@ -29,7 +29,7 @@ constexpr int kMaxWarpsPerBlock = 4;
 constexpr size_t kSmemLimit = 226 * 1024;   // shared memory one block may use on sm_100, less the static part
 constexpr unsigned kFull = 0xffffffffu;
 constexpr double kLambda0 = 1e-3, kLambdaMin = 1e-5, kLambdaMax = 1e12;
-constexpr int kParked = 20;                 // doubles per lane kept in shared memory between sweeps
+constexpr int kParked = 12;                 // doubles per lane kept in shared memory between sweeps
 
 __device__ __forceinline__ bool finite_d(double v) { return fabs(v) <= 1.7976931348623157e308; }
 
@@ -116,7 +116,8 @@ struct Normalised {
 // normalised change; then the window is scaled in place to levels y = l / M.  k_all: uniform
 // trip count of the warp.  changes_out (optional, global, indexed oldest first) receives the
 // normalised changes.
-__device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double m_seen, double* changes_out) {
+__device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double m_seen, int min_fit_points,
+                                       double* changes_out) {
     Normalised out;
     out.M = CUDART_NAN;
     out.rho = 0.0;
@@ -144,10 +145,12 @@ __device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double 
     }
     const bool usable = out.status == SLAQ_JOB_FITTED;
     const double M = out.M;
+    // the normalised changes feed only the linear extrapolation of short windows (and the export)
+    const bool want_changes = usable && (H < min_fit_points || changes_out != nullptr);
     double num = 0.0, den = 0.0;
     for (int k = 0; k < k_all; ++k) {
         const int m = S.l + S.L * k;
-        if (usable && m + 1 < H) {
+        if (want_changes && m + 1 < H) {
             const double change = __ddiv_rn(older_neighbour(S, k) - S.y[k * 32 + S.lane], M);
             const double w = S.wtab[m];
             num = fma(w, change, num);
@@ -176,6 +179,23 @@ __device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double 
     return out;
 }
 
+// Weighted mean normalised change per iteration from the scaled window (used when a window long
+// enough for a fit ends without one): sum w (y_{i-1} - y_i) / sum w.
+__device__ double mean_change_of_levels(const Lanes& S, int H, int k_all) {
+    double num = 0.0, den = 0.0;
+    for (int k = 0; k < k_all; ++k) {
+        const int m = S.l + S.L * k;
+        if (m + 1 < H) {
+            const double w = S.wtab[m];
+            num = fma(w, older_neighbour(S, k) - S.y[k * 32 + S.lane], num);
+            den += w;
+        }
+    }
+    num = group_sum(num, S.L);
+    den = group_sum(den, S.L);
+    return fmax(num / den, 0.0);
+}
+
 // ---- small dense algebra: every lane solves its own job's system ----
 
 struct Sym4 {   // symmetric 4x4, upper triangle
@@ -186,18 +206,18 @@ struct Sym4 {   // symmetric 4x4, upper triangle
 // B = L D L^T.  False if a pivot is not positive and finite or the solution is not finite.
 __device__ bool ldl_solve(const Sym4& B, const double (&r)[4], double (&x)[4]) {
     const double d0 = B.a00;
-    const double i0 = 1.0 / d0;
+    const double i0 = fast_rcp(d0);
     const double l10 = B.a01 * i0, l20 = B.a02 * i0, l30 = B.a03 * i0;
     const double d1 = fma(-l10, B.a01, B.a11);
-    const double i1 = 1.0 / d1;
+    const double i1 = fast_rcp(d1);
     const double t21 = fma(-l20, B.a01, B.a12), t31 = fma(-l30, B.a01, B.a13);
     const double l21 = t21 * i1, l31 = t31 * i1;
     const double d2 = fma(-l21, t21, fma(-l20, B.a02, B.a22));
-    const double i2 = 1.0 / d2;
+    const double i2 = fast_rcp(d2);
     const double t32 = fma(-l31, t21, fma(-l30, B.a02, B.a23));
     const double l32 = t32 * i2;
     const double d3 = fma(-l32, t32, fma(-l31, t31, fma(-l30, B.a03, B.a33)));
-    const double i3 = 1.0 / d3;
+    const double i3 = fast_rcp(d3);
     bool ok = d0 > 0.0 && d1 > 0.0 && d2 > 0.0 && d3 > 0.0 && finite_d(d0) && finite_d(d1) && finite_d(d2) &&
               finite_d(d3);
     const double z0 = r[0];
@@ -212,10 +232,10 @@ __device__ bool ldl_solve(const Sym4& B, const double (&r)[4], double (&x)[4]) {
     return ok;
 }
 
-// Solver state of one family for one job (held by every lane of the job's group).
+// Solver state of ONE family for one job.  The lanes of a group alternate: even lanes carry
+// family I, odd lanes family II, so one instruction stream advances both solvers at once.
 struct Family {
     double p[4];       // current parameters
-    double trial[4];   // trial point of the running sweep
     double S;          // weighted residual at p
     double lambda, nu;
     double predicted;  // reduction the quadratic model promises for the trial step
@@ -223,13 +243,14 @@ struct Family {
     int sweeps;
     bool ok;           // the starting point was usable
     bool done;         // no further trials
-    bool has_trial;    // the running sweep evaluates `trial`
+    bool has_trial;    // the running sweep evaluates the trial point
 };
 
-template <int P>
-__device__ __forceinline__ double lower_bound_of(int a) {
-    if (P == 4) return a == 3 ? -CUDART_INF : (a == 2 ? 1e-12 : 0.0);   // a >= 0, b >= 0, c >= 1e-12
-    return a == 1 ? 0.0 : -CUDART_INF;                                   // beta >= 0
+// Lower bounds.  Family I (fam 0): a >= 0, b >= 0, c >= 1e-12 keep the curve non-increasing ahead
+// of the newest point and its denominator positive there.  Family II (fam 1): beta >= 0.
+__device__ __forceinline__ double lower_bound_of(int fam, int a) {
+    if (fam == 0) return a == 3 ? -CUDART_INF : (a == 2 ? 1e-12 : 0.0);
+    return a == 1 ? 0.0 : -CUDART_INF;
 }
 
 // One Levenberg-Marquardt trial up to the point where the model must be evaluated: freeze
@@ -237,24 +258,29 @@ __device__ __forceinline__ double lower_bound_of(int a) {
 // outside (and keep them frozen from then on), solve (A + lambda diag A) step = g over the
 // rest, clip the trial point to the bounds, and record the reduction the quadratic model
 // promises.  `busy` = this lane has a trial to prepare; the re-solve loop runs while any
-// lane of the warp needs another round.
-template <int P>
-__device__ void prepare_trial(Family& F, const Sym4& A, const double (&g)[4], bool busy, double sum_wy2) {
+// lane of the warp needs another round.  Family II has three parameters: its fourth row is
+// a fixed identity row.
+__device__ void prepare_trial(Family& F, int fam, const Sym4& A, const double (&g)[4], bool busy, double sum_wy2,
+                              double (&trial)[4]) {
     F.has_trial = false;
     if (busy && F.S <= 1e-28 * sum_wy2) {   // residual is zero to rounding
         F.done = true;
         busy = false;
     }
-    unsigned frozen = 0;
+    const int P = fam == 0 ? 4 : 3;
+    double lo[4];
 #pragma unroll
-    for (int a = 0; a < P; ++a)
-        if (F.p[a] <= lower_bound_of<P>(a) && (g[a] < 0.0 || ((F.was_frozen >> a) & 1u))) frozen |= 1u << a;
+    for (int a = 0; a < 4; ++a) lo[a] = lower_bound_of(fam, a);
+    unsigned frozen = fam == 0 ? 0u : 8u;
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+        if (a < P && F.p[a] <= lo[a] && (g[a] < 0.0 || ((F.was_frozen >> a) & 1u))) frozen |= 1u << a;
     double step[4] = {0.0, 0.0, 0.0, 0.0};
     bool solved = false, again = busy;
-    for (int round = 0; round <= P; ++round) {
+    for (int round = 0; round <= 4; ++round) {
         if (!__any_sync(kFull, again)) break;
-        if (again) {
-            const bool f0 = frozen & 1u, f1 = frozen & 2u, f2 = frozen & 4u, f3 = P < 4 || (frozen & 8u);
+        if (again && round <= P) {
+            const bool f0 = frozen & 1u, f1 = frozen & 2u, f2 = frozen & 4u, f3 = frozen & 8u;
             Sym4 B;
             B.a00 = f0 ? 1.0 : fma(F.lambda, fmax(A.a00, 1e-300), A.a00);
             B.a11 = f1 ? 1.0 : fma(F.lambda, fmax(A.a11, 1e-300), A.a11);
@@ -271,11 +297,13 @@ __device__ void prepare_trial(Family& F, const Sym4& A, const double (&g)[4], bo
             unsigned grow = 0;
             if (solved) {
 #pragma unroll
-                for (int a = 0; a < P; ++a)
-                    if (!((frozen >> a) & 1u) && F.p[a] <= lower_bound_of<P>(a) && step[a] < 0.0) grow |= 1u << a;
+                for (int a = 0; a < 4; ++a)
+                    if (a < P && !((frozen >> a) & 1u) && F.p[a] <= lo[a] && step[a] < 0.0) grow |= 1u << a;
             }
             frozen |= grow;
             again = solved && grow != 0;
+        } else {
+            again = false;
         }
     }
     if (!busy) return;
@@ -285,11 +313,11 @@ __device__ void prepare_trial(Family& F, const Sym4& A, const double (&g)[4], bo
         F.nu *= 2.0;
         return;
     }
-    double d[4] = {0.0, 0.0, 0.0, 0.0};
+    double d[4];
 #pragma unroll
-    for (int a = 0; a < P; ++a) {
-        F.trial[a] = fmax(F.p[a] + step[a], lower_bound_of<P>(a));
-        d[a] = F.trial[a] - F.p[a];
+    for (int a = 0; a < 4; ++a) {
+        trial[a] = a < P ? fmax(F.p[a] + step[a], lo[a]) : 0.0;
+        d[a] = trial[a] - F.p[a];
     }
     const double dg = fma(d[0], g[0], fma(d[1], g[1], fma(d[2], g[2], d[3] * g[3])));
     const double Ad0 = fma(A.a00, d[0], fma(A.a01, d[1], fma(A.a02, d[2], A.a03 * d[3])));
@@ -304,13 +332,13 @@ __device__ void prepare_trial(Family& F, const Sym4& A, const double (&g)[4], bo
 
 // After the sweep at the trial point: accept it only if the residual strictly fell, and move
 // the damping by the gain ratio (Madsen, Nielsen, Tingleff 2004).  Returns whether accepted.
-__device__ __forceinline__ bool finish_trial(Family& F, bool ok_trial, double S_trial) {
+__device__ __forceinline__ bool finish_trial(Family& F, const double (&trial)[4], bool ok_trial, double S_trial) {
     if (!F.has_trial) return false;
     F.has_trial = false;
     if (ok_trial && S_trial < F.S) {
         const double S_before = F.S;
 #pragma unroll
-        for (int a = 0; a < 4; ++a) F.p[a] = F.trial[a];
+        for (int a = 0; a < 4; ++a) F.p[a] = trial[a];
         F.S = S_trial;
         const double rho = F.predicted > 0.0 ? (S_before - S_trial) / F.predicted : 0.0;
         const double c = 2.0 * rho - 1.0;
@@ -325,18 +353,22 @@ __device__ __forceinline__ bool finish_trial(Family& F, bool ok_trial, double S_
     return false;
 }
 
-// Sums of one sweep: family I needs the moments of w u^2 and w u (u = 1/q^2, J = (-u x^2, -u x, -u, 1)),
-// family II those of w e^2 and w e (J = (e, -x e, 1)).
+// What a lane keeps of one sweep: the sums of ITS family over the whole window.
+// Family I (u = 1/q^2, J = (-u x^2, -u x, -u, 1)): v[0..4] = sum w u^2 x^k, v[5..7] = sum w u x^k,
+// v[8..10] = sum w u r x^k, v[11] = sum w r, v[12] = S.
+// Family II (J = (e, -x e, 1)): v[0..2] = sum w e^2 x^k, v[3..4] = sum w e x^k, v[5..6] = sum w e r x^k,
+// v[7] = sum w r, v[8] = S.
 struct SweepSums {
-    double m0, m1, m2, m3, m4, n0, n1, n2, h0, h1, h2, gd, sI;   // family I
-    double e0, e1, e2, f0, f1, k0, k1, gc, sII;                  // family II
-    int feasible;                                                // family I: every denominator positive
+    double v[13];
+    bool usable;   // the model was defined at every point and all sums are finite
 };
 
-// One sweep over the window: both families at once, each at its own point (pI, pII).
-// doI / doII: per lane, whether that family is evaluated.
-__device__ __forceinline__ void sweep(const Lanes& S, int H, int k_all, double inv_span, const double (&pI)[4],
-                                      bool doI, const double (&pII)[4], bool doII, SweepSums& out) {
+// One sweep over the window: both families at once, each at its own point.  A lane adds up
+// both families over its points; the first reduction step hands each lane of a pair the other
+// lane's partial sums of its own family, the remaining steps run over lanes of the same parity.
+__device__ __forceinline__ void sweep(const Lanes& S, int fam, int H, int k_all, double inv_span,
+                                      const double (&pI)[4], bool doI, const double (&pII)[4], bool doII,
+                                      SweepSums& out) {
     double m0 = 0, m1 = 0, m2 = 0, m3 = 0, m4 = 0, n0 = 0, n1 = 0, n2 = 0, h0 = 0, h1 = 0, h2 = 0, gd = 0, sI = 0;
     double e0 = 0, e1 = 0, e2 = 0, f0 = 0, f1 = 0, k0 = 0, k1 = 0, gc = 0, sII = 0;
     int feasible = 1;
@@ -350,12 +382,12 @@ __device__ __forceinline__ void sweep(const Lanes& S, int H, int k_all, double i
     }
     double md = (double)S.l;
     const double dL = (double)S.L;
-    for (int k = 0; k < k_all; ++k, md += dL) {
-        const int m = S.l + S.L * k;
+    const double* yp = S.y + S.lane;
+    for (int k = 0, m = S.l; k < k_all; ++k, m += S.L, md += dL, yp += 32) {
         if (m < H) {
             const double x = -md * inv_span;
             const double w = S.wtab[m];
-            const double y = S.y[k * 32 + S.lane];
+            const double y = *yp;
             const double x2 = x * x;
             if (doI) {
                 const double q = fma(fma(pI[0], x, pI[1]), x, pI[2]);
@@ -395,57 +427,52 @@ __device__ __forceinline__ void sweep(const Lanes& S, int H, int k_all, double i
         }
         e *= ratio;
     }
-    for (int o = S.L >> 1; o > 0; o >>= 1) {
-        m0 += __shfl_xor_sync(kFull, m0, o); m1 += __shfl_xor_sync(kFull, m1, o);
-        m2 += __shfl_xor_sync(kFull, m2, o); m3 += __shfl_xor_sync(kFull, m3, o);
-        m4 += __shfl_xor_sync(kFull, m4, o); n0 += __shfl_xor_sync(kFull, n0, o);
-        n1 += __shfl_xor_sync(kFull, n1, o); n2 += __shfl_xor_sync(kFull, n2, o);
-        h0 += __shfl_xor_sync(kFull, h0, o); h1 += __shfl_xor_sync(kFull, h1, o);
-        h2 += __shfl_xor_sync(kFull, h2, o); gd += __shfl_xor_sync(kFull, gd, o);
-        sI += __shfl_xor_sync(kFull, sI, o);
-        e0 += __shfl_xor_sync(kFull, e0, o); e1 += __shfl_xor_sync(kFull, e1, o);
-        e2 += __shfl_xor_sync(kFull, e2, o); f0 += __shfl_xor_sync(kFull, f0, o);
-        f1 += __shfl_xor_sync(kFull, f1, o); k0 += __shfl_xor_sync(kFull, k0, o);
-        k1 += __shfl_xor_sync(kFull, k1, o); gc += __shfl_xor_sync(kFull, gc, o);
-        sII += __shfl_xor_sync(kFull, sII, o);
+    // pair step: an even lane hands over its family-II partials and receives family-I ones, an odd lane the reverse
+    const bool odd = fam != 0;
+    double v[13];
+#define SLAQ_PAIR(k, a, b) v[k] = (odd ? (b) : (a)) + __shfl_xor_sync(kFull, odd ? (a) : (b), 1)
+    SLAQ_PAIR(0, m0, e0); SLAQ_PAIR(1, m1, e1); SLAQ_PAIR(2, m2, e2); SLAQ_PAIR(3, m3, f0); SLAQ_PAIR(4, m4, f1);
+    SLAQ_PAIR(5, n0, k0); SLAQ_PAIR(6, n1, k1); SLAQ_PAIR(7, n2, gc); SLAQ_PAIR(8, h0, sII);
+#undef SLAQ_PAIR
+    v[9] = h1 + __shfl_xor_sync(kFull, h1, 1);    // family I only: odd lanes carry these along unused
+    v[10] = h2 + __shfl_xor_sync(kFull, h2, 1);
+    v[11] = gd + __shfl_xor_sync(kFull, gd, 1);
+    v[12] = sI + __shfl_xor_sync(kFull, sI, 1);
+    feasible &= __shfl_xor_sync(kFull, feasible, 1);
+    for (int o = 2; o < S.L; o <<= 1) {
+#pragma unroll
+        for (int k = 0; k < 13; ++k) v[k] += __shfl_xor_sync(kFull, v[k], o);
         feasible &= __shfl_xor_sync(kFull, feasible, o);
     }
-    out.m0 = m0; out.m1 = m1; out.m2 = m2; out.m3 = m3; out.m4 = m4; out.n0 = n0; out.n1 = n1; out.n2 = n2;
-    out.h0 = h0; out.h1 = h1; out.h2 = h2; out.gd = gd; out.sI = sI;
-    out.e0 = e0; out.e1 = e1; out.e2 = e2; out.f0 = f0; out.f1 = f1; out.k0 = k0; out.k1 = k1; out.gc = gc;
-    out.sII = sII;
-    out.feasible = feasible;
+    double chk = 0.0;
+#pragma unroll
+    for (int k = 0; k < 13; ++k) {
+        out.v[k] = v[k];
+        if (k < 9 || !odd) chk += v[k];
+    }
+    out.usable = finite_d(chk) && (odd || feasible);
 }
 
 // The sums of the last accepted point live in the lane's shared-memory column between sweeps.
-__device__ __forceinline__ void park_I(const Lanes& S, const SweepSums& s) {
+__device__ __forceinline__ void park(const Lanes& S, const SweepSums& s) {
     double* c = S.park + S.lane;
-    c[0 * 32] = s.m0; c[1 * 32] = s.m1; c[2 * 32] = s.m2; c[3 * 32] = s.m3; c[4 * 32] = s.m4;
-    c[5 * 32] = s.n0; c[6 * 32] = s.n1; c[7 * 32] = s.n2;
-    c[8 * 32] = s.h0; c[9 * 32] = s.h1; c[10 * 32] = s.h2; c[11 * 32] = s.gd;
+#pragma unroll
+    for (int k = 0; k < kParked; ++k) c[k * 32] = s.v[k];
 }
-__device__ __forceinline__ void park_II(const Lanes& S, const SweepSums& s) {
-    double* c = S.park + S.lane;
-    c[12 * 32] = s.e0; c[13 * 32] = s.e1; c[14 * 32] = s.e2; c[15 * 32] = s.f0; c[16 * 32] = s.f1;
-    c[17 * 32] = s.k0; c[18 * 32] = s.k1; c[19 * 32] = s.gc;
-}
-__device__ __forceinline__ void normal_eq_I(const Lanes& S, double sw, Sym4& A, double (&g)[4]) {
+
+// Normal equations A = sum w J J^T, g = sum w J r of the lane's family from the parked sums.
+__device__ __forceinline__ void normal_equations(const Lanes& S, int fam, double sw, Sym4& A, double (&g)[4]) {
     const double* c = S.park + S.lane;
-    A.a00 = c[4 * 32]; A.a01 = c[3 * 32]; A.a02 = c[2 * 32]; A.a11 = c[2 * 32]; A.a12 = c[1 * 32]; A.a22 = c[0 * 32];
-    A.a03 = -c[7 * 32]; A.a13 = -c[6 * 32]; A.a23 = -c[5 * 32]; A.a33 = sw;
-    g[0] = -c[10 * 32]; g[1] = -c[9 * 32]; g[2] = -c[8 * 32]; g[3] = c[11 * 32];
-}
-__device__ __forceinline__ void normal_eq_II(const Lanes& S, double sw, Sym4& A, double (&g)[4]) {
-    const double* c = S.park + S.lane;
-    A.a00 = c[12 * 32]; A.a01 = -c[13 * 32]; A.a11 = c[14 * 32]; A.a02 = c[15 * 32]; A.a12 = -c[16 * 32]; A.a22 = sw;
-    A.a03 = 0.0; A.a13 = 0.0; A.a23 = 0.0; A.a33 = 1.0;
-    g[0] = c[17 * 32]; g[1] = -c[18 * 32]; g[2] = c[19 * 32]; g[3] = 0.0;
-}
-__device__ __forceinline__ bool sums_finite_I(const SweepSums& s) {
-    return finite_d(s.m0 + s.m1 + s.m2 + s.m3 + s.m4 + s.n0 + s.n1 + s.n2 + s.h0 + s.h1 + s.h2 + s.gd + s.sI);
-}
-__device__ __forceinline__ bool sums_finite_II(const SweepSums& s) {
-    return finite_d(s.e0 + s.e1 + s.e2 + s.f0 + s.f1 + s.k0 + s.k1 + s.gc + s.sII);
+    if (fam == 0) {
+        A.a00 = c[4 * 32]; A.a01 = c[3 * 32]; A.a02 = c[2 * 32]; A.a11 = c[2 * 32]; A.a12 = c[1 * 32];
+        A.a22 = c[0 * 32];
+        A.a03 = -c[7 * 32]; A.a13 = -c[6 * 32]; A.a23 = -c[5 * 32]; A.a33 = sw;
+        g[0] = -c[10 * 32]; g[1] = -c[9 * 32]; g[2] = -c[8 * 32]; g[3] = c[11 * 32];
+    } else {
+        A.a00 = c[0 * 32]; A.a01 = -c[1 * 32]; A.a11 = c[2 * 32]; A.a02 = c[3 * 32]; A.a12 = -c[4 * 32]; A.a22 = sw;
+        A.a03 = 0.0; A.a13 = 0.0; A.a23 = 0.0; A.a33 = 1.0;
+        g[0] = c[5 * 32]; g[1] = -c[6 * 32]; g[2] = c[7 * 32]; g[3] = 0.0;
+    }
 }
 
 struct Moments {
@@ -543,7 +570,7 @@ struct FitClasses {
     int h_max;       // longest window
 };
 
-__global__ void __launch_bounds__(kMaxWarpsPerBlock * 32, 4)
+__global__ void __launch_bounds__(kMaxWarpsPerBlock * 32, 3)
 fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, const int32_t* __restrict__ order,
            const int32_t* __restrict__ start, FitClasses cls, int lm_trials, int min_fit_points, unsigned int* queue,
            long long* counters, int32_t* err_word) {
@@ -568,6 +595,8 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         for (int c = cls.n; c <= kMaxFitClasses; ++c) slot_base[c] = run;
     }
     __syncthreads();
+    const int fam = lane & 1;             // even lanes solve family I, odd lanes family II
+    const int even = lane & ~1, oddl = lane | 1;
 
     long long n_points = 0, n_sweep_points = 0;
     int n_fit = 0, n_sub = 0, n_exp = 0, n_fallback = 0;
@@ -591,7 +620,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         const int k_all = warp_max_int((H + L - 1) / L);
         __syncwarp();
         const double m_seen = j >= 0 ? job.m_seen[j] : -CUDART_INF;
-        const Normalised nz = normalise_window(S, H, k_all, m_seen, nullptr);
+        const Normalised nz = normalise_window(S, H, k_all, m_seen, min_fit_points, nullptr);
 
         int status = nz.status, family = -1;
         double p_out[4] = {CUDART_NAN, CUDART_NAN, CUDART_NAN, CUDART_NAN};
@@ -603,55 +632,74 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         if (__any_sync(kFull, fits)) {
             const double inv_span = 1.0 / span;
             Moments mom;
-            Family I, II;
-            first_guesses(S, H, k_all, inv_span, nz.ymin, nz.ymax, fits, mom, I.p, II.p);
+            Family F;
+            double pI[4], pII[4];      // the points the next sweep evaluates
+            first_guesses(S, H, k_all, inv_span, nz.ymin, nz.ymax, fits, mom, pI, pII);
             SweepSums sums;
-            sweep(S, H, k_all, inv_span, I.p, fits, II.p, fits, sums);
-            I.ok = fits && sums.feasible && sums_finite_I(sums);
-            II.ok = fits && sums_finite_II(sums);
-            I.S = sums.sI; II.S = sums.sII;
-            I.lambda = II.lambda = kLambda0;
-            I.nu = II.nu = 2.0;
-            I.was_frozen = II.was_frozen = 0;
-            I.sweeps = II.sweeps = fits ? 1 : 0;
-            I.done = !I.ok; II.done = !II.ok;
-            I.has_trial = II.has_trial = false;
-            I.predicted = II.predicted = 0.0;
+            sweep(S, fam, H, k_all, inv_span, pI, fits, pII, fits, sums);
 #pragma unroll
-            for (int a = 0; a < 4; ++a) I.trial[a] = II.trial[a] = 0.0;
-            park_I(S, sums);
-            park_II(S, sums);
+            for (int a = 0; a < 4; ++a) F.p[a] = fam ? pII[a] : pI[a];
+            F.ok = fits && sums.usable;
+            F.S = sums.v[fam ? 8 : 12];
+            F.lambda = kLambda0;
+            F.nu = 2.0;
+            F.was_frozen = 0;
+            F.sweeps = fits ? 1 : 0;
+            F.done = !F.ok;
+            F.has_trial = false;
+            F.predicted = 0.0;
+            park(S, sums);
             for (int t = 0; t < lm_trials; ++t) {
-                if (!__any_sync(kFull, !I.done || !II.done)) break;
+                if (!__any_sync(kFull, !F.done)) break;
+                double trial[4] = {0.0, 0.0, 0.0, 0.0};
                 {
                     Sym4 A;
                     double gr[4];
-                    normal_eq_I(S, mom.sw, A, gr);
-                    prepare_trial<4>(I, A, gr, !I.done, mom.swy2);
-                    normal_eq_II(S, mom.sw, A, gr);
-                    prepare_trial<3>(II, A, gr, !II.done, mom.swy2);
+                    normal_equations(S, fam, mom.sw, A, gr);
+                    prepare_trial(F, fam, A, gr, !F.done, mom.swy2, trial);
                 }
-                if (!__any_sync(kFull, I.has_trial || II.has_trial)) continue;
-                sweep(S, H, k_all, inv_span, I.trial, I.has_trial, II.trial, II.has_trial, sums);
-                if (finish_trial(I, sums.feasible && sums_finite_I(sums), sums.sI)) park_I(S, sums);
-                if (finish_trial(II, sums_finite_II(sums), sums.sII)) park_II(S, sums);
+                const unsigned trying = __ballot_sync(kFull, F.has_trial);
+                if (!trying) continue;
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {   // each lane of a pair fetches the other family's trial point
+                    pI[a] = __shfl_sync(kFull, trial[a], even);
+                    pII[a] = __shfl_sync(kFull, trial[a], oddl);
+                }
+                sweep(S, fam, H, k_all, inv_span, pI, (trying >> even) & 1u, pII, (trying >> oddl) & 1u, sums);
+                if (finish_trial(F, trial, sums.usable, sums.v[fam ? 8 : 12])) park(S, sums);
+            }
+            // both results of the job, in every lane
+            const double S_I = __shfl_sync(kFull, F.S, even), S_II = __shfl_sync(kFull, F.S, oddl);
+            const bool ok_I = __shfl_sync(kFull, (int)F.ok, even), ok_II = __shfl_sync(kFull, (int)F.ok, oddl);
+            sweeps_out[0] = __shfl_sync(kFull, F.sweeps, even);
+            sweeps_out[1] = __shfl_sync(kFull, F.sweeps, oddl);
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                pI[a] = __shfl_sync(kFull, F.p[a], even);
+                pII[a] = __shfl_sync(kFull, F.p[a], oddl);
             }
             if (fits) {
-                sweeps_out[0] = I.sweeps;
-                sweeps_out[1] = II.sweeps;
-                if (I.ok) S_out[0] = I.S;
-                if (II.ok) S_out[1] = II.S;
-                const bool okI = I.ok && finite_d(I.S), okII = II.ok && finite_d(II.S);
-                if (okI && (!okII || I.S <= II.S)) {   // a tie goes to family I
+                if (ok_I) S_out[0] = S_I;
+                if (ok_II) S_out[1] = S_II;
+                const bool okI = ok_I && finite_d(S_I), okII = ok_II && finite_d(S_II);
+                if (okI && (!okII || S_I <= S_II)) {   // a tie goes to family I
                     family = 0;
 #pragma unroll
-                    for (int a = 0; a < 4; ++a) p_out[a] = I.p[a];
+                    for (int a = 0; a < 4; ++a) p_out[a] = pI[a];
                 } else if (okII) {
                     family = 1;
 #pragma unroll
-                    for (int a = 0; a < 4; ++a) p_out[a] = II.p[a];
+                    for (int a = 0; a < 4; ++a) p_out[a] = pII[a];
                 }
+            } else {
+                sweeps_out[0] = sweeps_out[1] = 0;
             }
+        }
+        const bool fit_failed = fits && family < 0;
+        double rho = nz.rho;
+        if (__any_sync(kFull, fit_failed)) {   // rare: the whole warp walks its windows once more
+            const double from_levels = mean_change_of_levels(S, H, k_all);
+            if (fit_failed) rho = from_levels;
         }
         if (status == SLAQ_JOB_NEW) {
             p_out[0] = 1.0;   // one normalised unit per iteration
@@ -659,7 +707,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         } else if (status == SLAQ_JOB_FITTED && family < 0) {
             status = H >= min_fit_points ? SLAQ_JOB_FIT_FAILED : SLAQ_JOB_SHORT;
             const double y_new = S.y[lane - S.l];
-            p_out[0] = nz.rho;
+            p_out[0] = rho;
             p_out[1] = y_new > 0.0 ? y_new : CUDART_INF;
             p_out[2] = p_out[3] = CUDART_NAN;
         }
@@ -735,7 +783,7 @@ normalise_export_kernel(JobArrays job, const int32_t* __restrict__ ids, const in
     }
     const int64_t base = offsets[slot];
     const int k_all = (H + 31) / 32;
-    const Normalised nz = normalise_window(S, H, k_all, job.m_seen[j], changes ? changes + base : nullptr);
+    const Normalised nz = normalise_window(S, H, k_all, job.m_seen[j], 0, changes ? changes + base : nullptr);
     if (lane == 0 && largest) largest[slot] = nz.M;
     for (int k = 0; k < k_all; ++k) {
         const int m = lane + 32 * k;
@@ -806,7 +854,7 @@ size_t fit_smem_bytes(const FitClasses& c, int warps) {
 // Lanes per job for windows up to h_hi points: the smallest group whose warp slice stays
 // within `budget` bytes of shared memory.
 int lanes_for(int h_hi, size_t budget) {
-    for (int L = 1; L <= 32; L <<= 1) {
+    for (int L = 2; L <= 32; L <<= 1) {   // at least a pair: its lanes split the two families
         const size_t slice = sizeof(double) * ((size_t)((h_hi + L - 1) / L + 1) * 32 + kParked * 32);
         if (slice <= budget) return L;
     }
