@@ -97,10 +97,25 @@ __device__ int stage_window(const JobArrays& job, int j, int h_cap, const Lanes&
     }
     int newest = job.head[j] - 1;
     if (newest < 0) newest += cap;
-    for (int m = S.l, k = 0; m < H; m += S.L, ++k) {
+    // four loads in flight per lane; the values are read once, so they bypass the caches' keep lists
+    double* dst = S.y + S.lane;
+    int m = S.l;
+    for (; m + 3 * S.L < H; m += 4 * S.L, dst += 4 * 32) {
+        int p0 = newest - m, p1 = p0 - S.L, p2 = p1 - S.L, p3 = p2 - S.L;
+        p0 += p0 < 0 ? cap : 0;
+        p1 += p1 < 0 ? cap : 0;
+        p2 += p2 < 0 ? cap : 0;
+        p3 += p3 < 0 ? cap : 0;
+        const double v0 = __ldcs(row + p0), v1 = __ldcs(row + p1), v2 = __ldcs(row + p2), v3 = __ldcs(row + p3);
+        dst[0] = v0;
+        dst[32] = v1;
+        dst[64] = v2;
+        dst[96] = v3;
+    }
+    for (; m < H; m += S.L, dst += 32) {
         int pos = newest - m;
-        if (pos < 0) pos += cap;
-        S.y[k * 32 + S.lane] = row[pos];
+        pos += pos < 0 ? cap : 0;
+        *dst = __ldcs(row + pos);
     }
     return H;
 }
