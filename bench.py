@@ -35,8 +35,7 @@ FLOP_SWEEP_I, FLOP_SWEEP_II, FLOP_SETUP = 40.0, 25.0, 40.0
 FP64_LANES_PER_SM = 64          # fp64 FMA lanes per SM on B200
 
 
-def rank_info():
-    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+from paper_1802_04819_b200.partition import max_over_ranks, partition_seed_offset, rank_info, whole_job_rate  # noqa: E402
 
 
 class ClockSampler:
@@ -148,7 +147,7 @@ def run_gpu(args):
     import paper_1802_04819_b200 as slaq
     slaq.build()
 
-    wl = make_workload(CFG, n_jobs=args.jobs, seed_offset=rank)   # every rank: its own 100,000-job partition
+    wl = make_workload(CFG, n_jobs=args.jobs, seed_offset=partition_seed_offset(rank))   # each rank: its own partition
     J, cap = wl.n_jobs, wl.max_cores_per_job
     ids = np.arange(J, dtype=np.int32)
     stream = torch.cuda.current_stream()
@@ -217,10 +216,7 @@ def run_gpu(args):
     e2e_s = (time.perf_counter() - t0) / e2e_steps
     assert int(h_alloc.sum()) == wl.total_cores
 
-    times = torch.tensor([ms_step, e2e_s * 1e3], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_step, e2e_ms = float(times[0]), float(times[1])
+    ms_step, e2e_ms = max_over_ranks([ms_step, e2e_s * 1e3], device="cuda")
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
@@ -231,7 +227,7 @@ def run_gpu(args):
         achieved = fit_flops / (fit_ms_avg * 1e-3) / 1e12
         stage = np.mean(np.array(stage_ms), axis=0)
         line = {
-            "metric": METRIC, "value": world * J / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": whole_job_rate(J, world, ms_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": "config3_100k_jobs_400k_cores_cap64_hist3-1000_csr" if args.jobs is None
@@ -241,7 +237,7 @@ def run_gpu(args):
                        "l2": "inputs larger than L2 (401 MB of losses read per step)",
                        "parallelism": f"{world} independent cluster partition(s), one per GPU"},
             "clocks": clocks,
-            "e2e": {"value": world * J / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+            "e2e": {"value": whole_job_rate(J, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": int(J * (4 + 8 + 8)), "d2h_bytes_per_step": int(J * 4 + 4),
                     "steps": e2e_steps,
                     "what": "slaq_append_losses (host arrays, one new loss per job) + slaq_schedule (host out_alloc)"},
