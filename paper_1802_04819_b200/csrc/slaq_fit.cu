@@ -585,7 +585,7 @@ struct FitClasses {
     int h_max;       // longest window
 };
 
-__global__ void __launch_bounds__(kMaxWarpsPerBlock * 32, 3)
+__global__ void __launch_bounds__(kMaxWarpsPerBlock * 32, 4)
 fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, const int32_t* __restrict__ order,
            const int32_t* __restrict__ start, FitClasses cls, int lm_trials, int min_fit_points, unsigned int* queue,
            long long* counters, int32_t* err_word) {
@@ -919,6 +919,7 @@ int launch_fit(slaq_handle* h) {
         h->err = std::string("fit kernel shared memory: ") + cudaGetErrorString(e);
         return -1;
     }
+    cudaFuncSetAttribute(fit_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     int per_sm = 1;
     cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fit_kernel, warps * 32, smem);
     if (per_sm < 1) per_sm = 1;
