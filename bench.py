@@ -33,6 +33,9 @@ UNIT = "jobs/s"
 # algorithmic fp64 work of the fit, per stored point: one sweep of family I, one of family II, set-up
 FLOP_SWEEP_I, FLOP_SWEEP_II, FLOP_SETUP = 40.0, 25.0, 40.0
 FP64_LANES_PER_SM = 64          # fp64 FMA lanes per SM on B200
+# DRAM bytes per stored loss moved by the fit kernel (ncu: dram__bytes_read.sum + dram__bytes_write.sum =
+# 163.36 MB + 4.37 MB on a 20,068,408-loss cut of this workload; traffic grows with the stored losses)
+NCU_FIT_DRAM_BYTES_PER_LOSS = (163.36e6 + 4.37e6) / 20_068_408
 
 
 from paper_1802_04819_b200.partition import max_over_ranks, partition_seed_offset, rank_info, whole_job_rate  # noqa: E402
@@ -244,7 +247,9 @@ def run_gpu(args):
             "gpu_launches": launches,
             "stage_ms": {"fit": float(stage[0]), "gain": float(stage[1]), "alloc": float(stage[2])},
             "roofline": {"bound": "alu", "kernel": "fit_kernel", "achieved": achieved, "peak": peak_tflops,
-                         "unit": "TFLOP/s", "frac": achieved / peak_tflops, "traffic": None,
+                         "unit": "TFLOP/s", "frac": achieved / peak_tflops,
+                         "traffic": NCU_FIT_DRAM_BYTES_PER_LOSS * int(wl.offsets[-1]),
+                         "traffic_note": "bytes per launch, scaled by stored losses from the ncu capture of a 40,000-job cut",
                          "algorithmic_flops_per_launch": fit_flops, "ms_per_launch": fit_ms_avg,
                          "peak_is": f"{sm_count} SMs x {FP64_LANES_PER_SM} fp64 FMA lanes x 2 x {sm_max:.0f} MHz "
                                     f"(clock from MEASURED_PEAKS.json: {peak_kind})"},
