@@ -21,3 +21,50 @@ def test_config3_full_size_all_jobs(oracle_mod):
     info = compare_epoch(alloc, pred, ref, wl.total_cores, wl.max_cores_per_job)
     print("config 3 full size:", info, sched.get_stats().as_dict())
     assert alloc.sum() == wl.total_cores
+
+
+def test_config4_full_size_sampled(oracle_mod):
+    """1,000,000 jobs, ring of 64, 128 cores per job: predictions of a sample against the oracle one by one,
+    and the allocation through properties that hold at any size."""
+    import paper_1802_04819_b200 as slaq
+    slaq.build()
+    wl = make_workload(4)
+    sched = make_scheduler(wl)
+    alloc, rc = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    assert rc == 0
+    pred = sched.get_predictions()
+    cap = wl.max_cores_per_job
+    # sample: every 53rd job plus all clones and their sources
+    dst = np.nonzero(wl.clone_of >= 0)[0]
+    sample = np.unique(np.concatenate([np.arange(0, wl.n_jobs, 53), dst, wl.clone_of[dst]]))
+    H = wl.hist_len[sample]
+    off = np.zeros(sample.size + 1, np.int64)
+    np.cumsum(H, out=off[1:])
+    idx = np.concatenate([np.arange(wl.offsets[j], wl.offsets[j + 1]) for j in sample])
+    ref = oracle_mod.predict(off, wl.losses[idx], wl.m_seen[sample], wl.s[sample], wl.w[sample], wl.epoch_seconds, cap)
+    np.testing.assert_array_equal(pred["status"][sample], ref["status"])
+    np.testing.assert_array_equal(pred["M"][sample], ref["M"])
+    Rg, Rc = np.cumsum(pred["gain"][sample], axis=1), np.cumsum(ref["gain"], axis=1)
+    tied = pred["family"][sample] != ref["family"]
+    bad = (np.abs(Rg - Rc) > 1e-6 * np.abs(Rc) + 1e-9).any(axis=1) & ~tied
+    assert bad.sum() == 0, f"{bad.sum()} of {sample.size} sampled jobs exceed the tolerance"
+    for j in np.nonzero(tied)[0]:
+        S = ref["S"][j]
+        assert abs(S[0] - S[1]) <= 1e-9 * max(abs(S[0]), abs(S[1]))
+    # allocation: all cores handed out, floor and cap respected, and it is a top-C selection of the GPU's own gains:
+    # every gain taken beyond the floor is at least as large as every gain left
+    assert alloc.sum() == wl.total_cores and alloc.min() >= 1 and alloc.max() <= cap
+    g = pred["gain"]
+    cols = np.arange(cap)[None, :]
+    taken = (cols < alloc[:, None]) & (cols >= 1)
+    left = cols >= alloc[:, None]
+    tau = g[taken].min()
+    assert g[left].max() <= tau
+    # ties at the threshold go to the lowest job ids
+    at_tau_taken = np.nonzero(((g == tau) & taken).any(axis=1))[0]
+    at_tau_left = np.nonzero(((g == tau) & left).any(axis=1))[0]
+    if at_tau_taken.size and at_tau_left.size:
+        assert at_tau_taken.max() <= at_tau_left.min()
+    np.testing.assert_array_equal(g[dst], g[wl.clone_of[dst]])
+    R_direct = np.where(cols < alloc[:, None], g, 0.0).sum(axis=1)
+    np.testing.assert_allclose(pred["R"], R_direct, rtol=1e-12, atol=1e-15)

@@ -279,3 +279,58 @@ def test_parameters_change_the_fit(slaq, oracle_mod):
     ref = oracle_mod.schedule(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, wl.total_cores, 16,
                               gamma=0.8, lm_trials=7)
     compare_epoch(alloc, sched.get_predictions(), ref, wl.total_cores, 16)
+
+
+# ---------------------------------------------------------------- window lengths at every class edge
+def test_window_lengths_at_class_boundaries(slaq, oracle_mod):
+    lengths = [4, 5, 7, 8, 9, 15, 16, 17, 31, 32, 33, 62, 63, 64, 65, 66, 124, 125, 126, 127, 128, 129, 249, 250, 251,
+               252, 255, 256, 257, 499, 500, 501, 502, 511, 512, 513, 998, 999, 1000] * 3
+    wl = make_workload(3, hist_lengths=lengths)
+    for packed in (False, True):
+        sched = make_scheduler(wl, packed=packed)
+        alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+        compare_epoch(alloc, sched.get_predictions(), oracle_epoch(oracle_mod, wl), wl.total_cores,
+                      wl.max_cores_per_job)
+
+
+def test_longest_supported_windows(slaq, oracle_mod):
+    lengths = [6000, 5999, 4097, 3001, 3000, 1501, 1500, 751, 750, 400, 100, 20, 4, 3]
+    wl = make_workload(3, hist_lengths=lengths)
+    assert wl.max_hist == 6000
+    sched = make_scheduler(wl, packed=True)
+    alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    compare_epoch(alloc, sched.get_predictions(), oracle_epoch(oracle_mod, wl), wl.total_cores, wl.max_cores_per_job)
+    ids = np.arange(wl.n_jobs)
+    offsets, changes, levels, largest = sched.get_normalised(ids, capacity=int(wl.offsets[-1]))
+    M, dn, y = oracle_mod.normalise(wl.offsets, wl.losses, wl.m_seen)
+    np.testing.assert_array_equal(levels, y)
+    np.testing.assert_array_equal(changes, dn)
+
+
+@pytest.mark.parametrize("slice_bytes", [8192, 12288, 32768, 65536, 200 * 1024])
+def test_lanes_per_job_do_not_change_results_beyond_rounding(slaq, oracle_mod, slice_bytes):
+    wl = make_workload(3, n_jobs=1500)
+    sched = make_scheduler(wl, packed=True)
+    sched.set_param(5, slice_bytes)          # shared memory per warp: decides how many lanes share a job
+    alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    compare_epoch(alloc, sched.get_predictions(), oracle_epoch(oracle_mod, wl), wl.total_cores, wl.max_cores_per_job)
+
+
+@pytest.mark.parametrize("gamma", [1.0, 0.5, 0.99])
+def test_other_weight_bases(slaq, oracle_mod, gamma):
+    wl = make_workload(2, n_jobs=1200)
+    sched = make_scheduler(wl)
+    sched.set_param(1, gamma)
+    alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    ref = oracle_mod.schedule(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, wl.total_cores,
+                              wl.max_cores_per_job, gamma=gamma)
+    compare_epoch(alloc, sched.get_predictions(), ref, wl.total_cores, wl.max_cores_per_job)
+
+
+def test_other_seeds(slaq, oracle_mod):
+    for seed in (1, 2, 3):
+        wl = make_workload(2, seed_offset=seed)
+        sched = make_scheduler(wl, packed=True)
+        alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+        compare_epoch(alloc, sched.get_predictions(), oracle_epoch(oracle_mod, wl), wl.total_cores,
+                      wl.max_cores_per_job)

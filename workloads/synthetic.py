@@ -106,9 +106,12 @@ def _past_max_reduction(family, params, k0):
     return out
 
 
-def make_workload(cfg: int, n_jobs: int | None = None, seed_offset: int = 0) -> Workload:
-    """Draw workload `cfg` (0..4).  `n_jobs` overrides J (cores scale with it)."""
+def make_workload(cfg: int, n_jobs: int | None = None, seed_offset: int = 0, hist_lengths=None) -> Workload:
+    """Draw workload `cfg` (0..4).  `n_jobs` overrides J (cores scale with it); `hist_lengths`
+    (one entry per job) replaces the drawn history lengths, for tests that need exact lengths."""
     spec = CONFIGS[cfg]
+    if hist_lengths is not None:
+        n_jobs = len(hist_lengths)
     J = int(spec["J"] if n_jobs is None else n_jobs)
     rng = np.random.default_rng(SEED_BASE + cfg + 1000 * seed_offset)
     cap = spec["cap"]
@@ -134,6 +137,8 @@ def make_workload(cfg: int, n_jobs: int | None = None, seed_offset: int = 0) -> 
         w = rng.uniform(1.0, 100.0, J)
 
     H = rng.integers(spec["hmin"], spec["hmax"] + 1, J).astype(np.int64)
+    if hist_lengths is not None:
+        H = np.asarray(hist_lengths, dtype=np.int64).copy()
     k0 = np.zeros(J, dtype=np.int64)
     sigma = np.full(J, spec["sigma"])
     converged = np.zeros(J, dtype=bool)
@@ -207,7 +212,7 @@ def make_workload(cfg: int, n_jobs: int | None = None, seed_offset: int = 0) -> 
     m_seen = np.maximum(past, win)
 
     return Workload(
-        cfg=cfg, n_jobs=J, total_cores=C, max_cores_per_job=cap, max_hist=int(spec["hmax"]),
+        cfg=cfg, n_jobs=J, total_cores=C, max_cores_per_job=cap, max_hist=int(max(spec["hmax"], H.max())),
         epoch_seconds=float(spec["T"]), offsets=offsets, losses=losses,
         k_last=k0 + H - 1, m_seen=m_seen, s=s, w=w, family=family, params=params,
         sigma=sigma, clone_of=clone_of,
