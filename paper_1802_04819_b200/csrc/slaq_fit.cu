@@ -516,7 +516,7 @@ __device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span,
             swx3 = fma(wx2, x, swx3);
             swx4 = fma(wx2 * x, x, swx4);
             swy2 = fma(w * y, y, swy2);
-            const double wz = w / (y - d0);
+            const double wz = w * fast_rcp(y - d0);
             r2 += wz;
             r1 = fma(wz, x, r1);
             r0 = fma(wz * x, x, r0);

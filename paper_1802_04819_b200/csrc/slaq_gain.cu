@@ -5,8 +5,8 @@
 // An iteration on n cores takes t(n) = s + w/n seconds, so an epoch of T seconds runs
 // m(n) = T n / (s n + w) iterations; in window coordinates that is X_n = m(n) / span ahead
 // of the newest point, and R(n) = f(0) - f(X_n).  g(n) = R(n) - R(n-1) is evaluated without
-// cancellation, clamped to +0 where it is not a positive finite number, and made
-// non-increasing in n by a running minimum.  One warp per job; the row is written once,
+// cancellation (divisions by Newton reciprocals: a gain is good to a few ulp), clamped to +0
+// where it is not a positive finite number, and made non-increasing in n by a running minimum.  One warp per job; the row is written once,
 // coalesced, and its keys feed the first histogram of the threshold selection.
 #include <math_constants.h>
 
@@ -54,39 +54,44 @@ __device__ bool time_law(const JobArrays& job, int j, int max_jobs, double& s, d
     return finite_d(s) && finite_d(w) && w > 0.0 && s >= 0.0;
 }
 
+// Reciprocal to about one ulp: hardware seed and two Newton steps.
+__device__ __forceinline__ double fast_rcp(double q) {
+    double x;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(x) : "d"(q));
+    double e = fma(-q, x, 1.0);
+    x = fma(x, e, x);
+    e = fma(-q, x, 1.0);
+    return fma(x, e, x);
+}
+
 struct Curve {
     int kind;        // 0 family I, 1 family II, 2 linear extrapolation, 3 no gain
     double p0, p1, p2;
-    double span, s, w, T;
+    double inv_span, s, w, T;
+    double step_scale;   // T w / span: X_n - X_{n-1} = step_scale / ((s n + w)(s (n-1) + w))
 };
 
-// after an epoch on n cores: s n + w, iterations completed, and the same in window coordinates
-__device__ __forceinline__ void ahead(const Curve& c, int n, double& X, double& den, double& m) {
-    den = __dadd_rn(__dmul_rn(c.s, (double)n), c.w);
-    m = __ddiv_rn(__dmul_rn(c.T, (double)n), den);
-    X = __ddiv_rn(m, c.span);
-}
-
+// Gain of the n-th core.  After an epoch on n cores the job has run m(n) = T n / (s n + w) iterations,
+// X_n = m(n) / span in window coordinates.
 __device__ double raw_gain(const Curve& c, int n) {
-    double X, den, m, Xp = 0.0, denp = c.w, mp = 0.0;
-    ahead(c, n, X, den, m);
-    if (n > 1) ahead(c, n - 1, Xp, denp, mp);
+    const double den = fma(c.s, (double)n, c.w), denp = fma(c.s, (double)(n - 1), c.w);
+    const double inv_den = fast_rcp(den), inv_denp = fast_rcp(denp);
+    const double m = c.T * (double)n * inv_den, mp = c.T * (double)(n - 1) * inv_denp;
+    const double X = m * c.inv_span, Xp = mp * c.inv_span;
     double gain;
     if (c.kind == 0) {
         // 1/q(Xp) - 1/q(X) = (q(X) - q(Xp)) / (q(X) q(Xp)), q(X) - q(Xp) = (X - Xp)(a (X + Xp) + b)
-        const double dX = __ddiv_rn(__dmul_rn(c.T, c.w), __dmul_rn(__dmul_rn(c.span, den), denp));
-        const double q_now = __dadd_rn(__dadd_rn(__dmul_rn(__dmul_rn(c.p0, X), X), __dmul_rn(c.p1, X)), c.p2);
-        const double q_prev = __dadd_rn(__dadd_rn(__dmul_rn(__dmul_rn(c.p0, Xp), Xp), __dmul_rn(c.p1, Xp)), c.p2);
-        const double dq = __dmul_rn(dX, __dadd_rn(__dmul_rn(c.p0, __dadd_rn(X, Xp)), c.p1));
-        gain = __ddiv_rn(dq, __dmul_rn(q_now, q_prev));
+        const double dX = c.step_scale * inv_den * inv_denp;
+        const double q_now = fma(fma(c.p0, X, c.p1), X, c.p2);
+        const double q_prev = fma(fma(c.p0, Xp, c.p1), Xp, c.p2);
+        const double dq = dX * fma(c.p0, X + Xp, c.p1);
+        gain = dq * fast_rcp(q_now * q_prev);
     } else if (c.kind == 1) {
         // e^(alpha - beta Xp) - e^(alpha - beta X) = e^(alpha - beta Xp) (1 - e^(-beta (X - Xp)))
-        const double dX = __ddiv_rn(__dmul_rn(c.T, c.w), __dmul_rn(__dmul_rn(c.span, den), denp));
-        gain = exp(__dsub_rn(c.p0, __dmul_rn(c.p1, Xp))) * (-expm1(-__dmul_rn(c.p1, dX)));
+        const double dX = c.step_scale * inv_den * inv_denp;
+        gain = exp(fma(-c.p1, Xp, c.p0)) * (-expm1(-c.p1 * dX));
     } else {
-        const double R = fmin(__dmul_rn(c.p0, m), c.p1);
-        const double Rp = n > 1 ? fmin(__dmul_rn(c.p0, mp), c.p1) : 0.0;
-        gain = __dsub_rn(R, Rp);
+        gain = fmin(c.p0 * m, c.p1) - fmin(c.p0 * mp, c.p1);
     }
     return (finite_d(gain) && gain > 0.0) ? gain : 0.0;
 }
@@ -105,8 +110,8 @@ gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int f
         Curve c;
         c.kind = 3;
         c.T = T;
-        c.span = fit.span[j];
-        c.s = c.w = c.p0 = c.p1 = c.p2 = 0.0;
+        c.inv_span = 1.0 / fit.span[j];
+        c.s = c.w = c.p0 = c.p1 = c.p2 = c.step_scale = 0.0;
         const bool predicts = status == SLAQ_JOB_FITTED || status == SLAQ_JOB_SHORT || status == SLAQ_JOB_NEW ||
                               status == SLAQ_JOB_FIT_FAILED;
         if (active && status != SLAQ_JOB_NONFINITE && status != SLAQ_JOB_FLAT) {
@@ -118,6 +123,7 @@ gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int f
                 c.p1 = fit.params[4 * (size_t)j + 1];
                 c.p2 = fit.params[4 * (size_t)j + 2];
                 c.kind = status == SLAQ_JOB_FITTED ? (int)fit.family[j] : 2;
+                c.step_scale = T * c.w * c.inv_span;
             }
         }
         double carry = CUDART_INF;   // running minimum of the gains before this chunk

@@ -334,3 +334,38 @@ def test_other_seeds(slaq, oracle_mod):
         alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
         compare_epoch(alloc, sched.get_predictions(), oracle_epoch(oracle_mod, wl), wl.total_cores,
                       wl.max_cores_per_job)
+
+
+# ---------------------------------------------------------------- streaming: append -> schedule with the allocation fed back
+def test_streaming_epochs_with_allocation_feedback(slaq, oracle_mod):
+    """Several epochs in a row: each job runs as many iterations as its allocation allows in the epoch, reports
+    their losses and times (booked at the allocation), and is scheduled again.  Both sides carry their own state."""
+    from workloads import true_curve
+    wl = make_workload(1)
+    J, cap, max_hist = wl.n_jobs, wl.max_cores_per_job, 24          # short ring: it wraps within the run
+    sched = slaq.Scheduler(J, max_hist, cap)
+    ref = oracle_mod.OracleScheduler(J, max_hist, cap)
+    rng = np.random.default_rng(77)
+    k_next = np.zeros(J, dtype=np.int64)
+    alloc = np.ones(J, dtype=np.int32)
+    T = wl.epoch_seconds
+    for epoch in range(7):
+        # iterations each job completes this epoch on its current cores (at least one, so every job reports)
+        iters = np.maximum(1, np.floor(T * alloc / (wl.s * alloc + wl.w)).astype(np.int64))
+        iters = np.minimum(iters, 6)
+        for step in range(int(iters.max())):
+            live = np.nonzero(step < iters)[0]
+            k = k_next[live].astype(np.float64)
+            losses = true_curve(wl.family[live], wl.params[live], k) * np.exp(0.01 * rng.standard_normal(live.size))
+            times = wl.s[live] + wl.w[live] / alloc[live]
+            sched.append_losses(live, losses, times)             # booked at the last allocation on both sides
+            ref.append_losses(live, losses, times)
+            k_next[live] += 1
+        got, rc = sched.schedule(T, wl.total_cores)
+        out = ref.schedule(T, wl.total_cores)
+        compare_epoch(got, sched.get_predictions(), out, wl.total_cores, cap)
+        s, w = sched.get_time_model()
+        np.testing.assert_array_equal(s, out["s"])
+        np.testing.assert_array_equal(w, out["w"])
+        alloc = got.copy()
+    assert (k_next >= 7).all()
