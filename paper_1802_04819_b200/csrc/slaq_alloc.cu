@@ -7,7 +7,8 @@
 // gains it serves (job id ascending, n ascending).  Here: a most-significant-digit-first
 // radix select over the 64-bit patterns of the gains (all >= +0, so the IEEE pattern
 // orders like the value) finds the threshold tau and how many gains equal to tau are
-// still wanted; then per job  a_j = floor + #{g > tau} + clamp(wanted - P_j, 0, #{g = tau})
+// still wanted - after the first two passes it reads only the short segment of each row
+// that still agrees with the threshold's leading digits; then per job  a_j = floor + #{g > tau} + clamp(wanted - P_j, 0, #{g = tau})
 // with P_j the number of gains equal to tau in jobs with a lower id.
 #include <math_constants.h>
 
@@ -70,12 +71,15 @@ __device__ void pick_bin(const unsigned long long* hist, int pass, SelectState* 
     }
 }
 
-// Histogram of one digit over the candidates that match the prefix found so far; the
-// last block to finish picks the bin.
+// Rows are non-increasing, so the candidates of a row whose leading digits equal the threshold
+// prefix found so far form one contiguous segment [seg_lo, seg_hi) of the row.  Pass p narrows every
+// segment by the bin chosen for digit p - 1 (elements with a larger digit lie before it, with a smaller
+// one behind it) and histograms digit p over what is left; from the second pass on only the
+// segments are read.  The last block to finish picks the bin of digit p.
 __global__ void __launch_bounds__(kSelectThreads)
 select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap,
                    int first_unit, int pass, unsigned long long* __restrict__ hist_all, SelectState* sel,
-                   unsigned int* ticket) {
+                   unsigned int* ticket, int32_t* __restrict__ seg_lo, int32_t* __restrict__ seg_hi) {
     __shared__ unsigned int sh_hist[kRadixBins];
     __shared__ unsigned long long sh_scan[kSelectThreads + 1];
     __shared__ bool is_last;
@@ -85,16 +89,33 @@ select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ 
     __syncthreads();
     const unsigned long long prefix = sel->prefix;
     const int shift = pass_shift(pass), bits = pass_bits(pass);
-    const int hi_shift = shift + bits;                     // bits from here up are already fixed
+    const int prev_shift = pass_shift(pass - 1), prev_bits = pass_bits(pass - 1);
+    const unsigned prev_bin = (unsigned)(prefix >> prev_shift) & ((1u << prev_bits) - 1u);
     const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(gain);
     const int lane = threadIdx.x & 31;
     const int warps_total = gridDim.x * (kSelectThreads / 32);
     for (int j = blockIdx.x * (kSelectThreads / 32) + (threadIdx.x >> 5); j < max_jobs; j += warps_total) {
         if (count[j] <= 0) continue;
-        for (int n = first_unit + lane; n <= cap; n += 32) {
-            const unsigned long long key = keys[(size_t)j * cap + (n - 1)];
-            if ((key >> hi_shift) == (prefix >> hi_shift))
-                atomicAdd(&sh_hist[(unsigned)(key >> shift) & ((1u << bits) - 1u)], 1u);
+        int lo = first_unit - 1, hi = cap;      // 0-based positions n - 1
+        if (pass > 1) {
+            lo = seg_lo[j];
+            hi = seg_hi[j];
+        }
+        int above = 0, same = 0;
+        for (int base = lo; base < hi; base += 32) {
+            const int i = base + lane;
+            const bool in = i < hi;
+            unsigned long long key = 0;
+            if (in) key = keys[(size_t)j * cap + i];
+            const unsigned d_prev = (unsigned)(key >> prev_shift) & ((1u << prev_bits) - 1u);
+            const bool match = in && d_prev == prev_bin;
+            above += __popc(__ballot_sync(kFull, in && d_prev > prev_bin));
+            same += __popc(__ballot_sync(kFull, match));
+            if (match) atomicAdd(&sh_hist[(unsigned)(key >> shift) & ((1u << bits) - 1u)], 1u);
+        }
+        if (lane == 0) {
+            seg_lo[j] = lo + above;
+            seg_hi[j] = lo + above + same;
         }
     }
     __syncthreads();
@@ -146,30 +167,42 @@ first_hist_kernel(const double* __restrict__ gain, const int32_t* __restrict__ c
     }
 }
 
-// Per job: how many candidate gains lie above the threshold and how many equal it.
+// Per job: how many candidate gains lie above the threshold and how many equal it.  The segments
+// left by the last pass hold the candidates that agree with the threshold in all but the last digit;
+// one more narrowing by that digit's bin gives the gains equal to the threshold, and everything in
+// front of them is larger.  gt / eq overwrite seg_lo / seg_hi in place.
 __global__ void __launch_bounds__(256)
 count_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap, int first_unit,
              const SelectState* __restrict__ sel, int32_t* __restrict__ gt, int32_t* __restrict__ eq,
              long long* __restrict__ block_eq) {
     __shared__ int sh_eq[8];
+    const bool none_wanted = sel->done != 0;
     const unsigned long long tau = sel->prefix;
+    constexpr int last = kRadixPasses - 1;
+    const unsigned last_bin = (unsigned)(tau >> pass_shift(last)) & ((1u << pass_bits(last)) - 1u);
     const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(gain);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int eq_sum = 0;
-    for (int i = 0; i < 32; ++i) {
-        const int j = blockIdx.x * kJobsPerBlock + warp * 32 + i;
+    for (int r = 0; r < 32; ++r) {
+        const int j = blockIdx.x * kJobsPerBlock + warp * 32 + r;
         if (j >= max_jobs) break;
         int n_gt = 0, n_eq = 0;
-        if (count[j] > 0) {
-            for (int base = first_unit; base <= cap; base += 32) {
-                const int n = base + lane;
+        if (count[j] > 0 && !none_wanted) {
+            const int lo = gt[j], hi = eq[j];   // segment [lo, hi) written by the last pass
+            int above = 0, same = 0;
+            for (int base = lo; base < hi; base += 32) {
+                const int i = base + lane;
+                const bool in = i < hi;
                 unsigned long long key = 0;
-                const bool in = n <= cap;
-                if (in) key = keys[(size_t)j * cap + (n - 1)];
-                n_gt += __popc(__ballot_sync(kFull, in && key > tau));
-                n_eq += __popc(__ballot_sync(kFull, in && key == tau));
+                if (in) key = keys[(size_t)j * cap + i];
+                const unsigned d = (unsigned)(key >> pass_shift(last)) & ((1u << pass_bits(last)) - 1u);
+                above += __popc(__ballot_sync(kFull, in && d > last_bin));
+                same += __popc(__ballot_sync(kFull, in && d == last_bin));
             }
+            n_gt = lo + above - (first_unit - 1);
+            n_eq = same;
         }
+        __syncwarp();
         if (lane == 0) {
             gt[j] = n_gt;
             eq[j] = n_eq;
@@ -293,7 +326,8 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
     ++launches;
     for (int pass = 1; pass < kRadixPasses; ++pass) {
         select_pass_kernel<<<grid, kSelectThreads, 0, st>>>(h->gain, h->job.count, J, cap, first_unit, pass,
-                                                           h->scratch.hist, h->scratch.sel, h->scratch.ticket);
+                                                           h->scratch.hist, h->scratch.sel, h->scratch.ticket,
+                                                           h->scratch.gt, h->scratch.eq);
         ++launches;
     }
     const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
@@ -396,7 +430,7 @@ extern "C" int slaq_allocate_static(const double* d_gain, int32_t n_jobs, int32_
     pick_first_kernel<<<1, kSelectThreads, 0, st>>>(sc->hist, &sc->sel);
     for (int pass = 1; pass < kRadixPasses; ++pass)
         select_pass_kernel<<<grid, kSelectThreads, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, pass,
-                                                           sc->hist, &sc->sel, sc->ticket);
+                                                           sc->hist, &sc->sel, sc->ticket, sc->gt, sc->eq);
     const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
     count_kernel<<<blocks, 256, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, &sc->sel, sc->gt, sc->eq,
                                          sc->block_eq);

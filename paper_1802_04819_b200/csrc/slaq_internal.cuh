@@ -59,8 +59,8 @@ struct Scratch {
     SelectState* sel;
     long long* counters;             // [16] statistics accumulated by kernels
     size_t zero_bytes;
-    int32_t* gt;                     // per job: candidate gains strictly above the threshold
-    int32_t* eq;                     // per job: candidate gains equal to it
+    int32_t* gt;                     // per job: during the passes the start of its candidate segment, then gains above the threshold
+    int32_t* eq;                     // per job: during the passes the end of its segment, then gains equal to the threshold
     long long* block_eq;             // per block of the count kernel: sum of eq
     int32_t* bucket;                 // [max_hist + 1] jobs per window length (inside the cleared region)
     int32_t* order;                  // job ids, longest window first (fit kernel work list)
