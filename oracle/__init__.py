@@ -36,12 +36,8 @@ def build(force: bool = False) -> Path:
 _lib = None
 
 
-def _load():
-    global _lib
-    if _lib is not None:
-        return _lib
-    build()
-    lib = ctypes.CDLL(str(_LIB))
+def _bind(lib):
+    """Declare the argument types of every entry point of an oracle library."""
     c_i64, c_i32, c_f64, vp = ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_void_p
     lib.oracle_max_threads.restype = ctypes.c_int
     lib.oracle_normalise.argtypes = [c_i64, vp, vp, vp, vp, vp, vp]
@@ -56,8 +52,16 @@ def _load():
     lib.oracle_family_eval.argtypes = [c_i32, vp, c_f64, vp, vp]
     lib.oracle_lm_line.argtypes = [c_i64, vp, vp, vp, c_i32, c_f64, vp, vp]
     lib.oracle_fit_family.argtypes = [c_i32, c_i64, vp, c_f64, c_f64, c_i32, vp, vp, vp, vp]
-    _lib = lib
     return lib
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    build()
+    _lib = _bind(ctypes.CDLL(str(_LIB)))
+    return _lib
 
 
 def _p(a):
