@@ -104,29 +104,47 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
 
 
+def host_threads() -> int:
+    """Host cores this process may use (launchers often set OMP_NUM_THREADS=1: the oracle is told explicitly)."""
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
 def run_reference(args):
-    """The CPU oracle, as it stands, on a bounded sample of the same workload."""
+    """The CPU oracle, as it stands, on a bounded sample of the same workload.
+
+    The sample (the first jobs of the config-3 generator) is sized from one calibration step so that the
+    whole --steps/--warmup run stays within about two minutes."""
     rank, _, world = rank_info()
     if rank != 0:
         return
     import oracle
     oracle.build()
-    sample_jobs = 20_000
-    wl = make_workload(CFG, n_jobs=sample_jobs)
-    cores = oracle.max_threads()
+    cores = host_threads()
 
-    def step():
+    def step(wl):
         return oracle.schedule(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, wl.total_cores,
                                wl.max_cores_per_job, threads=cores)
 
+    probe = make_workload(CFG, n_jobs=1000)
+    step(probe)
+    t0 = time.perf_counter()
+    step(probe)
+    per_job = (time.perf_counter() - t0) / probe.n_jobs
+    budget = 120.0 / (args.steps + args.warmup)
+    sample_jobs = int(min(20_000, max(500, budget / per_job)))
+    wl = make_workload(CFG, n_jobs=sample_jobs)
     for _ in range(args.warmup):
-        step()
+        step(wl)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        step()
+        step(wl)
     dt = (time.perf_counter() - t0) / args.steps
     value = sample_jobs / dt
-    sample = f"first {sample_jobs} jobs of the config-3 generator ({int(wl.offsets[-1])} stored losses), one epoch per step"
+    sample = (f"first {sample_jobs} jobs of the config-3 generator ({int(wl.offsets[-1])} stored losses), "
+              f"one epoch per step")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -257,7 +275,7 @@ def run_gpu(args):
         if args.cpu_baseline:
             import oracle
             oracle.build()
-            cores = oracle.max_threads()
+            cores = host_threads()
             t0 = time.perf_counter()
             oracle.schedule(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, wl.total_cores, cap,
                             threads=cores)
