@@ -168,12 +168,12 @@ def run_gpu(args):
     import paper_1802_04819_b200 as slaq
     slaq.build()
 
-    wl = make_workload(CFG, n_jobs=args.jobs, seed_offset=partition_seed_offset(rank))   # each rank: its own partition
+    wl = make_workload(args.cfg, n_jobs=args.jobs, seed_offset=partition_seed_offset(rank))   # each rank: its own partition
     J, cap = wl.n_jobs, wl.max_cores_per_job
     ids = np.arange(J, dtype=np.int32)
     stream = torch.cuda.current_stream()
     sched = slaq.Scheduler(J, wl.max_hist, cap, stream=stream)
-    sched.load_histories(ids, wl.offsets, wl.losses, wl.k_last, wl.m_seen, packed=True)
+    sched.load_histories(ids, wl.offsets, wl.losses, wl.k_last, wl.m_seen, packed=args.cfg == CFG)   # config 4: rings
     sched.set_time_model(ids, wl.s, wl.w)
     d_alloc = torch.zeros(J, dtype=torch.int32, device="cuda")
 
@@ -251,11 +251,13 @@ def run_gpu(args):
             "metric": METRIC, "value": whole_job_rate(J, world, ms_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "config3_100k_jobs_400k_cores_cap64_hist3-1000_csr" if args.jobs is None
-                       else f"config3 generator cut to {J} jobs (profiling run, not the benchmark)", "jobs_per_gpu": J,
+            "config": {"workload": "config3_100k_jobs_400k_cores_cap64_hist3-1000_csr"
+                       if args.jobs is None and args.cfg == CFG
+                       else f"config {args.cfg} generator at {J} jobs (profiling run, not the benchmark)",
+                       "jobs_per_gpu": J,
                        "stored_losses_per_gpu": int(wl.offsets[-1]), "total_cores_per_gpu": wl.total_cores,
                        "max_cores_per_job": cap, "epoch_seconds": wl.epoch_seconds,
-                       "l2": "inputs larger than L2 (401 MB of losses read per step)",
+                       "l2": f"inputs larger than L2 ({int(wl.offsets[-1]) * 8 / 1e6:.0f} MB of losses read per step)",
                        "parallelism": f"{world} independent cluster partition(s), one per GPU"},
             "clocks": clocks,
             "e2e": {"value": whole_job_rate(J, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
@@ -295,6 +297,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--cfg", type=int, default=CFG, choices=[2, 3, 4],
+                    help="profiling aid: another workload generator (the reported line is then not the benchmark)")
     ap.add_argument("--jobs", type=int, default=None,
                     help="profiling aid: a smaller cut of the same generator (the reported line is then not the benchmark)")
     args = ap.parse_args()

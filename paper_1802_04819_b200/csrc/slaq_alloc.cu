@@ -94,28 +94,42 @@ select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ 
     const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(gain);
     const int lane = threadIdx.x & 31;
     const int warps_total = gridDim.x * (kSelectThreads / 32);
-    for (int j = blockIdx.x * (kSelectThreads / 32) + (threadIdx.x >> 5); j < max_jobs; j += warps_total) {
-        if (count[j] <= 0) continue;
-        int lo = first_unit - 1, hi = cap;      // 0-based positions n - 1
-        if (pass > 1) {
-            lo = seg_lo[j];
-            hi = seg_hi[j];
+    // a warp takes 32 rows at a time: each lane looks up one row's segment, then the warp walks the
+    // rows whose segment is not empty (after the second pass most are)
+    for (int j0 = (blockIdx.x * (kSelectThreads / 32) + (threadIdx.x >> 5)) * 32; j0 < max_jobs; j0 += warps_total * 32) {
+        const int mine = j0 + lane;
+        int my_lo = first_unit - 1, my_hi = cap;      // 0-based positions n - 1
+        bool live = mine < max_jobs && count[mine] > 0;
+        if (live && pass > 1) {
+            my_lo = seg_lo[mine];
+            my_hi = seg_hi[mine];
         }
-        int above = 0, same = 0;
-        for (int base = lo; base < hi; base += 32) {
-            const int i = base + lane;
-            const bool in = i < hi;
-            unsigned long long key = 0;
-            if (in) key = keys[(size_t)j * cap + i];
-            const unsigned d_prev = (unsigned)(key >> prev_shift) & ((1u << prev_bits) - 1u);
-            const bool match = in && d_prev == prev_bin;
-            above += __popc(__ballot_sync(kFull, in && d_prev > prev_bin));
-            same += __popc(__ballot_sync(kFull, match));
-            if (match) atomicAdd(&sh_hist[(unsigned)(key >> shift) & ((1u << bits) - 1u)], 1u);
+        unsigned todo = __ballot_sync(kFull, live && my_lo < my_hi);
+        while (todo) {
+            const int r = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const int j = j0 + r;
+            const int lo = __shfl_sync(kFull, my_lo, r), hi = __shfl_sync(kFull, my_hi, r);
+            int above = 0, same = 0;
+            for (int base = lo; base < hi; base += 32) {
+                const int i = base + lane;
+                const bool in = i < hi;
+                unsigned long long key = 0;
+                if (in) key = keys[(size_t)j * cap + i];
+                const unsigned d_prev = (unsigned)(key >> prev_shift) & ((1u << prev_bits) - 1u);
+                const bool match = in && d_prev == prev_bin;
+                above += __popc(__ballot_sync(kFull, in && d_prev > prev_bin));
+                same += __popc(__ballot_sync(kFull, match));
+                if (match) atomicAdd(&sh_hist[(unsigned)(key >> shift) & ((1u << bits) - 1u)], 1u);
+            }
+            if (lane == r) {
+                my_lo = lo + above;
+                my_hi = lo + above + same;
+            }
         }
-        if (lane == 0) {
-            seg_lo[j] = lo + above;
-            seg_hi[j] = lo + above + same;
+        if (live) {
+            seg_lo[mine] = my_lo;
+            seg_hi[mine] = my_hi;
         }
     }
     __syncthreads();
@@ -182,33 +196,43 @@ count_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count,
     const unsigned last_bin = (unsigned)(tau >> pass_shift(last)) & ((1u << pass_bits(last)) - 1u);
     const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(gain);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int eq_sum = 0;
-    for (int r = 0; r < 32; ++r) {
-        const int j = blockIdx.x * kJobsPerBlock + warp * 32 + r;
-        if (j >= max_jobs) break;
-        int n_gt = 0, n_eq = 0;
-        if (count[j] > 0 && !none_wanted) {
-            const int lo = gt[j], hi = eq[j];   // segment [lo, hi) written by the last pass
-            int above = 0, same = 0;
-            for (int base = lo; base < hi; base += 32) {
-                const int i = base + lane;
-                const bool in = i < hi;
-                unsigned long long key = 0;
-                if (in) key = keys[(size_t)j * cap + i];
-                const unsigned d = (unsigned)(key >> pass_shift(last)) & ((1u << pass_bits(last)) - 1u);
-                above += __popc(__ballot_sync(kFull, in && d > last_bin));
-                same += __popc(__ballot_sync(kFull, in && d == last_bin));
-            }
-            n_gt = lo + above - (first_unit - 1);
-            n_eq = same;
-        }
-        __syncwarp();
-        if (lane == 0) {
-            gt[j] = n_gt;
-            eq[j] = n_eq;
-        }
-        eq_sum += n_eq;
+    // each lane owns one of the warp's 32 rows; the warp walks the rows whose segment is not empty
+    const int mine = blockIdx.x * kJobsPerBlock + warp * 32 + lane;
+    const bool live = mine < max_jobs && count[mine] > 0 && !none_wanted;
+    int my_lo = 0, my_hi = 0;
+    if (live) {
+        my_lo = gt[mine];    // segment [lo, hi) written by the last pass
+        my_hi = eq[mine];
     }
+    int my_gt = live ? my_lo - (first_unit - 1) : 0, my_eq = 0;
+    unsigned todo = __ballot_sync(kFull, live && my_lo < my_hi);
+    while (todo) {
+        const int r = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int j = blockIdx.x * kJobsPerBlock + warp * 32 + r;
+        const int lo = __shfl_sync(kFull, my_lo, r), hi = __shfl_sync(kFull, my_hi, r);
+        int above = 0, same = 0;
+        for (int base = lo; base < hi; base += 32) {
+            const int i = base + lane;
+            const bool in = i < hi;
+            unsigned long long key = 0;
+            if (in) key = keys[(size_t)j * cap + i];
+            const unsigned d = (unsigned)(key >> pass_shift(last)) & ((1u << pass_bits(last)) - 1u);
+            above += __popc(__ballot_sync(kFull, in && d > last_bin));
+            same += __popc(__ballot_sync(kFull, in && d == last_bin));
+        }
+        if (lane == r) {
+            my_gt += above;
+            my_eq = same;
+        }
+    }
+    if (mine < max_jobs) {
+        gt[mine] = my_gt;
+        eq[mine] = my_eq;
+    }
+    int eq_sum = my_eq;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) eq_sum += __shfl_xor_sync(kFull, eq_sum, o);
     if (lane == 0) sh_eq[warp] = eq_sum;
     __syncthreads();
     if (threadIdx.x == 0) {

@@ -815,12 +815,38 @@ normalise_export_kernel(JobArrays job, const int32_t* __restrict__ ids, const in
 
 // ---- work list: job ids sorted by window length, longest first (counting sort) ----
 
-__global__ void length_count_kernel(const int32_t* __restrict__ count, int max_jobs, int max_hist, int32_t* bucket) {
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= max_jobs) return;
-    int H = count[j];
-    H = H < 0 ? 0 : (H > max_hist ? max_hist : H);
-    atomicAdd(&bucket[H], 1);
+// Jobs per window length.  Many jobs share a length (a full ring), so lengths are first counted
+// in shared memory, lanes with equal lengths adding once, and each block then adds its non-zero
+// bins to the global table.
+constexpr int kSortThreads = 256;
+constexpr int kSortJobsPerBlock = 8192;
+
+__device__ __forceinline__ int clamped_length(const int32_t* __restrict__ count, int j, int max_hist) {
+    const int H = count[j];
+    return H < 0 ? 0 : (H > max_hist ? max_hist : H);
+}
+
+__global__ void __launch_bounds__(kSortThreads)
+length_count_kernel(const int32_t* __restrict__ count, int max_jobs, int max_hist, int32_t* bucket) {
+    extern __shared__ int sh_count[];   // [max_hist + 1]
+    for (int i = threadIdx.x; i <= max_hist; i += blockDim.x) sh_count[i] = 0;
+    __syncthreads();
+    const int lo = blockIdx.x * kSortJobsPerBlock, hi = min(lo + kSortJobsPerBlock, max_jobs);
+    for (int base = lo; base < hi; base += blockDim.x) {
+        const int j = base + threadIdx.x;
+        const bool in = j < hi;
+        const int H = in ? clamped_length(count, j, max_hist) : 0;
+        const unsigned live = __ballot_sync(kFull, in);
+        if (in) {
+            const unsigned peers = __match_any_sync(live, H);
+            if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&sh_count[H], __popc(peers));
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i <= max_hist; i += blockDim.x) {
+        const int v = sh_count[i];
+        if (v) atomicAdd(&bucket[i], v);
+    }
 }
 
 // start[h] = number of jobs with a window longer than h (h = 0..max_hist); cursor = copy for the scatter.
@@ -853,13 +879,48 @@ __global__ void __launch_bounds__(1024) length_scan_kernel(const int32_t* __rest
     }
 }
 
-__global__ void length_scatter_kernel(const int32_t* __restrict__ count, int max_jobs, int max_hist, int32_t* cursor,
-                                      int32_t* order) {
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= max_jobs) return;
-    int H = count[j];
-    H = H < 0 ? 0 : (H > max_hist ? max_hist : H);
-    order[atomicAdd(&cursor[H], 1)] = j;
+// Scatter: a block counts its jobs per length again, reserves one contiguous range per non-zero
+// length with a single global atomic, and places its jobs inside those ranges.
+__global__ void __launch_bounds__(kSortThreads)
+length_scatter_kernel(const int32_t* __restrict__ count, int max_jobs, int max_hist, int32_t* cursor,
+                      int32_t* order) {
+    extern __shared__ int sh_sort[];    // [max_hist + 1] counts, then [max_hist + 1] next free position
+    int* sh_count = sh_sort;
+    int* sh_next = sh_sort + (max_hist + 1);
+    for (int i = threadIdx.x; i <= max_hist; i += blockDim.x) sh_count[i] = 0;
+    __syncthreads();
+    const int lo = blockIdx.x * kSortJobsPerBlock, hi = min(lo + kSortJobsPerBlock, max_jobs);
+    const int lane = threadIdx.x & 31;
+    for (int base = lo; base < hi; base += blockDim.x) {
+        const int j = base + threadIdx.x;
+        const bool in = j < hi;
+        const int H = in ? clamped_length(count, j, max_hist) : 0;
+        const unsigned live = __ballot_sync(kFull, in);
+        if (in) {
+            const unsigned peers = __match_any_sync(live, H);
+            if ((int)(__ffs(peers) - 1) == lane) atomicAdd(&sh_count[H], __popc(peers));
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i <= max_hist; i += blockDim.x) {
+        const int v = sh_count[i];
+        sh_next[i] = v ? atomicAdd(&cursor[i], v) : 0;
+    }
+    __syncthreads();
+    for (int base = lo; base < hi; base += blockDim.x) {
+        const int j = base + threadIdx.x;
+        const bool in = j < hi;
+        const int H = in ? clamped_length(count, j, max_hist) : 0;
+        const unsigned live = __ballot_sync(kFull, in);
+        if (in) {
+            const unsigned peers = __match_any_sync(live, H);
+            const int leader = __ffs(peers) - 1;
+            int first = 0;
+            if (lane == leader) first = atomicAdd(&sh_next[H], __popc(peers));
+            first = __shfl_sync(peers, first, leader);
+            order[first + __popc(peers & ((1u << lane) - 1u))] = j;
+        }
+    }
 }
 
 size_t fit_smem_bytes(const FitClasses& c, int warps) {
@@ -884,10 +945,13 @@ int launch_fit(slaq_handle* h) {
     int launches = 0;
     // work list
     {
-        const int threads = 256, blocks = (J + threads - 1) / threads;
-        length_count_kernel<<<blocks, threads, 0, st>>>(h->job.count, J, Hmax, h->scratch.bucket);
+        const int blocks = (J + kSortJobsPerBlock - 1) / kSortJobsPerBlock;
+        const size_t one = sizeof(int) * ((size_t)Hmax + 1);
+        cudaFuncSetAttribute(length_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * one));
+        length_count_kernel<<<blocks, kSortThreads, one, st>>>(h->job.count, J, Hmax, h->scratch.bucket);
         length_scan_kernel<<<1, 1024, 0, st>>>(h->scratch.bucket, Hmax, h->scratch.start, h->scratch.cursor);
-        length_scatter_kernel<<<blocks, threads, 0, st>>>(h->job.count, J, Hmax, h->scratch.cursor, h->scratch.order);
+        length_scatter_kernel<<<blocks, kSortThreads, 2 * one, st>>>(h->job.count, J, Hmax, h->scratch.cursor,
+                                                                     h->scratch.order);
         launches += 3;
     }
     // length classes, longest first: (max_hist/2, max_hist], (max_hist/4, max_hist/2], ... then (0, 64 or less]
