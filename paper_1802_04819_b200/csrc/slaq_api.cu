@@ -324,10 +324,12 @@ int do_append(slaq_handle* h, int32_t n, const int32_t* ids, const double* losse
                                                                   (times && cores) ? h->stage.cores : nullptr);
     CK(cudaGetLastError(), "append kernel");
     CK(cudaStreamSynchronize(st), "append");   // the caller may reuse its buffers
-    for (int32_t i = 0; i < n; ++i) {
-        if (!h->active[ids[i]]) {
-            h->active[ids[i]] = 1;
-            h->n_active += 1;
+    if (h->n_active < h->max_jobs) {   // nothing to do once every id is active
+        for (int32_t i = 0; i < n; ++i) {
+            if (!h->active[ids[i]]) {
+                h->active[ids[i]] = 1;
+                h->n_active += 1;
+            }
         }
     }
     return SLAQ_OK;
@@ -633,7 +635,7 @@ int slaq_schedule(slaq_t* h, double epoch_seconds, int64_t total_cores, int32_t*
     if (rc < 0) return rc;
     CK(cudaMemcpyAsync(out_alloc, h->alloc, sizeof(int32_t) * (size_t)h->max_jobs, cudaMemcpyDeviceToHost, h->stream),
        "copy allocation");
-    const int ec = check_device_errors(h);
+    const int ec = check_device_errors(h);   // its synchronisation also completes the copy above
     return ec ? ec : rc;
 }
 
