@@ -231,6 +231,38 @@ int slaq_allocate_only(slaq_t* h, int64_t total_cores, int32_t* out_alloc);
 int slaq_get_stats(slaq_t* h, slaq_stats* out);
 
 /*
+ * One cluster sharded over several GPUs.  The jobs of ONE cluster are split into contiguous
+ * blocks of job ids, block r on GPU r (shard r: its own handle, local ids 0..max_jobs-1 in global
+ * order), and all shards share the cluster's cores.  Normalise, fit and gains need no exchange.  The
+ * greedy loop of "Scheduling Based on Quality Improvements" picks the globally largest gain at every
+ * step, so the threshold search needs the SUM over shards of each digit histogram (2048 x uint64 per
+ * pass, six passes) and the tie rule (lowest job id first) needs the number of threshold-equal gains in
+ * lower shards.  These calls are the steps between which the caller performs that exchange with its
+ * collective library (an all-reduce per pass, one all-gather of one integer per shard); every shard
+ * must make the same calls in the same order:
+ *   slaq_get_active_count                      -> sum over shards = J; floor iff C >= J;
+ *                                                 want = min(C, J x max_cores_per_job) - (floor ? J : 0)
+ *   slaq_shard_predict(T, floor)               normalise + fit + gains + local histogram of digit 0
+ *   for pass = 0..5:
+ *       if pass > 0: slaq_shard_pass(pass)     narrow by the bin of digit pass-1, local histogram of digit pass
+ *       slaq_shard_histogram(pass, buf, 0)     export; all-reduce(sum) buf over shards;
+ *       slaq_shard_histogram(pass, buf, 1)     import the summed histogram
+ *       slaq_shard_pick(pass, want)            same bin on every shard
+ *   slaq_shard_count(&ties)                    all-gather ties; ties_before = sum over lower shards
+ *   slaq_shard_finalise(ties_before, out_alloc)
+ * d_hist is device memory of 2048 uint64 owned by the caller; out_alloc is a host array of max_jobs
+ * entries.  The result equals slaq_schedule on one handle holding all jobs.  All calls are ordered on
+ * the handle's stream; slaq_shard_count and slaq_shard_finalise return after the stream has finished.
+ */
+int slaq_get_active_count(slaq_t* h, int32_t* out_active);
+int slaq_shard_predict(slaq_t* h, double epoch_seconds, int32_t with_floor);
+int slaq_shard_histogram(slaq_t* h, int32_t pass, uint64_t* d_hist, int32_t import_it);
+int slaq_shard_pick(slaq_t* h, int32_t pass, int64_t want);
+int slaq_shard_pass(slaq_t* h, int32_t pass);
+int slaq_shard_count(slaq_t* h, int64_t* out_local_ties);
+int slaq_shard_finalise(slaq_t* h, int64_t ties_before, int32_t* out_alloc);
+
+/*
  * The allocation step for callers that must not allocate device memory.  (The paper has
  * no counterpart: it is the selection of slaq_allocate_only, packaged so that it touches
  * the allocator nowhere.)

@@ -10,3 +10,4 @@ from .binding import (  # noqa: F401
     EXPORTED_SYMBOLS, STATIC_MAX_JOBS, Scheduler, SlaqError, Stats, allocate_static, load_library, workspace_bytes,
 )
 from .build import build  # noqa: F401
+from .sharded import LocalExchange, ProcessGroupExchange, schedule_sharded  # noqa: F401

@@ -18,7 +18,8 @@ EXPORTED_SYMBOLS = [
     "slaq_set_param", "slaq_get_param", "slaq_append_losses", "slaq_append_losses_ex", "slaq_load_histories",
     "slaq_load_histories_packed", "slaq_set_time_model", "slaq_remove_jobs", "slaq_schedule", "slaq_schedule_device",
     "slaq_get_predictions", "slaq_get_normalised", "slaq_get_time_model", "slaq_set_gains", "slaq_allocate_only",
-    "slaq_get_stats", "slaq_allocate_static",
+    "slaq_get_stats", "slaq_allocate_static", "slaq_get_active_count", "slaq_shard_predict", "slaq_shard_histogram",
+    "slaq_shard_pick", "slaq_shard_pass", "slaq_shard_count", "slaq_shard_finalise",
 ]
 
 
@@ -76,6 +77,13 @@ def load_library():
         "slaq_allocate_only": (c_int, [vp, c_int64, vp]),
         "slaq_get_stats": (c_int, [vp, POINTER(Stats)]),
         "slaq_allocate_static": (c_int, [vp, c_int32, c_int32, c_int64, vp, vp, vp]),
+        "slaq_get_active_count": (c_int, [vp, POINTER(c_int32)]),
+        "slaq_shard_predict": (c_int, [vp, c_double, c_int32]),
+        "slaq_shard_histogram": (c_int, [vp, c_int32, vp, c_int32]),
+        "slaq_shard_pick": (c_int, [vp, c_int32, c_int64]),
+        "slaq_shard_pass": (c_int, [vp, c_int32]),
+        "slaq_shard_count": (c_int, [vp, POINTER(c_int64)]),
+        "slaq_shard_finalise": (c_int, [vp, c_int64, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -246,6 +254,36 @@ class Scheduler:
         out = np.empty(self.max_jobs, np.int32)
         rc = self._check(self._lib.slaq_allocate_only(self._h, int(total_cores), _ptr(out)))
         return out, rc
+
+    # -- one cluster sharded over several GPUs: the steps between which histograms are summed --
+    def get_active_count(self) -> int:
+        out = c_int32()
+        self._check(self._lib.slaq_get_active_count(self._h, ctypes.byref(out)))
+        return out.value
+
+    def shard_predict(self, epoch_seconds: float, with_floor: bool):
+        return self._check(self._lib.slaq_shard_predict(self._h, float(epoch_seconds), int(bool(with_floor))))
+
+    def shard_histogram(self, pass_index: int, d_hist, import_it: bool):
+        """``d_hist``: torch int64 CUDA tensor of 2048 entries (the counts stay far below 2^63)."""
+        return self._check(self._lib.slaq_shard_histogram(self._h, pass_index, c_void_p(d_hist.data_ptr()),
+                                                          int(bool(import_it))))
+
+    def shard_pick(self, pass_index: int, want: int):
+        return self._check(self._lib.slaq_shard_pick(self._h, pass_index, int(want)))
+
+    def shard_pass(self, pass_index: int):
+        return self._check(self._lib.slaq_shard_pass(self._h, pass_index))
+
+    def shard_count(self) -> int:
+        out = c_int64()
+        self._check(self._lib.slaq_shard_count(self._h, ctypes.byref(out)))
+        return out.value
+
+    def shard_finalise(self, ties_before: int):
+        out = np.empty(self.max_jobs, np.int32)
+        self._check(self._lib.slaq_shard_finalise(self._h, int(ties_before), _ptr(out)))
+        return out
 
     def get_stats(self) -> Stats:
         st = Stats()

@@ -79,7 +79,7 @@ __device__ void pick_bin(const unsigned long long* hist, int pass, SelectState* 
 __global__ void __launch_bounds__(kSelectThreads)
 select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap,
                    int first_unit, int pass, unsigned long long* __restrict__ hist_all, SelectState* sel,
-                   unsigned int* ticket, int32_t* __restrict__ seg_lo, int32_t* __restrict__ seg_hi) {
+                   unsigned int* ticket, int32_t* __restrict__ seg_lo, int32_t* __restrict__ seg_hi, int do_pick) {
     __shared__ unsigned int sh_hist[kRadixBins];
     __shared__ unsigned long long sh_scan[kSelectThreads + 1];
     __shared__ bool is_last;
@@ -137,6 +137,7 @@ select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ 
         const unsigned v = sh_hist[i];
         if (v) atomicAdd(&hist[i], (unsigned long long)v);
     }
+    if (!do_pick) return;   // the histogram is completed elsewhere (summed over GPUs) before the bin is picked
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) is_last = atomicAdd(&ticket[1 + pass], 1u) == gridDim.x - 1;
@@ -151,6 +152,14 @@ select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ 
 __global__ void __launch_bounds__(kSelectThreads) pick_first_kernel(unsigned long long* hist_all, SelectState* sel) {
     __shared__ unsigned long long sh_scan[kSelectThreads + 1];
     pick_bin(hist_all, 0, sel, sh_scan);
+}
+
+// Pick the bin of any pass from a histogram that is complete when the kernel starts.
+__global__ void __launch_bounds__(kSelectThreads)
+pick_pass_kernel(unsigned long long* hist_all, int pass, SelectState* sel) {
+    __shared__ unsigned long long sh_scan[kSelectThreads + 1];
+    if (sel->done) return;
+    pick_bin(hist_all + (size_t)pass * kRadixBins, pass, sel, sh_scan);
 }
 
 __global__ void init_select_kernel(SelectState* sel, long long want) {
@@ -242,7 +251,7 @@ count_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count,
     }
 }
 
-// Exclusive prefix sum of block_eq[0..n), one block of 1024 threads.
+// Exclusive prefix sum of block_eq[0..n), one block of 1024 threads; block_eq[n] receives the total.
 __global__ void __launch_bounds__(1024) scan_blocks_kernel(long long* block_eq, int n) {
     __shared__ long long sh[1024];
     const int t = threadIdx.x;
@@ -264,6 +273,8 @@ __global__ void __launch_bounds__(1024) scan_blocks_kernel(long long* block_eq, 
         block_eq[i] = run;
         run += v;
     }
+    __syncthreads();
+    if (t == 1023) block_eq[n] = sh[1023];
 }
 
 // a_j from the counts, the predicted reduction at a_j, and the allocation becomes the job's core count.
@@ -271,7 +282,8 @@ __global__ void __launch_bounds__(256)
 finalise_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap, int floor_units,
                 const SelectState* __restrict__ sel, const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
                 const long long* __restrict__ block_prefix, int32_t* __restrict__ alloc, double* __restrict__ reduction,
-                int32_t* __restrict__ last_alloc, int32_t* __restrict__ out_alloc, long long* counters) {
+                int32_t* __restrict__ last_alloc, int32_t* __restrict__ out_alloc, long long* counters,
+                long long ties_before) {
     __shared__ long long sh_pre[kJobsPerBlock];
     __shared__ int sh_alloc[kJobsPerBlock];
     const int t = threadIdx.x;
@@ -286,7 +298,8 @@ finalise_kernel(const double* __restrict__ gain, const int32_t* __restrict__ cou
         sh_pre[t] += v;
         __syncthreads();
     }
-    const long long before = block_prefix[blockIdx.x] + sh_pre[t] - my_eq;   // ties in jobs with a lower id
+    // ties in jobs with a lower id (ties_before: those held by lower-numbered shards of the same cluster)
+    const long long before = ties_before + block_prefix[blockIdx.x] + sh_pre[t] - my_eq;
     int a = 0;
     long long ties_taken = 0;
     if (jt < max_jobs && count[jt] > 0) {
@@ -351,7 +364,7 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
     for (int pass = 1; pass < kRadixPasses; ++pass) {
         select_pass_kernel<<<grid, kSelectThreads, 0, st>>>(h->gain, h->job.count, J, cap, first_unit, pass,
                                                            h->scratch.hist, h->scratch.sel, h->scratch.ticket,
-                                                           h->scratch.gt, h->scratch.eq);
+                                                           h->scratch.gt, h->scratch.eq, 1);
         ++launches;
     }
     const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
@@ -360,7 +373,7 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
     scan_blocks_kernel<<<1, 1024, 0, st>>>(h->scratch.block_eq, blocks);
     finalise_kernel<<<blocks, 256, 0, st>>>(h->gain, h->job.count, J, cap, first_unit - 1, h->scratch.sel, h->scratch.gt,
                                             h->scratch.eq, h->scratch.block_eq, h->alloc, h->reduction,
-                                            h->job.last_alloc, d_out_alloc, h->scratch.counters);
+                                            h->job.last_alloc, d_out_alloc, h->scratch.counters, 0);
     launches += 3;
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
@@ -368,6 +381,61 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
         return -1;
     }
     return launches;
+}
+
+// ---- one cluster sharded over several GPUs: the same kernels, driven step by step so that the
+// histograms can be summed over the shards between the steps ----
+
+static int check_launch(slaq_handle* h, const char* what) {
+    const cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) return 0;
+    h->err = std::string(what) + ": " + cudaGetErrorString(e);
+    return -1;
+}
+
+// Pick the bin of `pass` from its (summed) histogram; pass 0 first sets what is wanted over all shards.
+int launch_shard_pick(slaq_handle* h, int pass, long long want) {
+    int launches = 0;
+    if (pass == 0) {
+        init_select_kernel<<<1, 1, 0, h->stream>>>(h->scratch.sel, want);
+        ++launches;
+    }
+    pick_pass_kernel<<<1, kSelectThreads, 0, h->stream>>>(h->scratch.hist, pass, h->scratch.sel);
+    ++launches;
+    return check_launch(h, "shard pick") ? -1 : launches;
+}
+
+// Narrow this shard's segments by the bin of digit pass - 1 and histogram digit `pass` locally.
+int launch_shard_pass(slaq_handle* h, int pass, int first_unit) {
+    const int J = h->max_jobs;
+    int grid = h->sm_count * 8;
+    const int needed = (J + (kSelectThreads / 32) - 1) / (kSelectThreads / 32);
+    if (grid > needed) grid = needed;
+    select_pass_kernel<<<grid, kSelectThreads, 0, h->stream>>>(h->gain, h->job.count, J, h->max_cores, first_unit, pass,
+                                                              h->scratch.hist, h->scratch.sel, h->scratch.ticket,
+                                                              h->scratch.gt, h->scratch.eq, 0);
+    return check_launch(h, "shard pass") ? -1 : 1;
+}
+
+// Per-job counts of this shard; *d_total points at the shard's number of gains equal to the threshold.
+int launch_shard_count(slaq_handle* h, int first_unit, const long long** d_total) {
+    const int J = h->max_jobs;
+    const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
+    count_kernel<<<blocks, 256, 0, h->stream>>>(h->gain, h->job.count, J, h->max_cores, first_unit, h->scratch.sel,
+                                                h->scratch.gt, h->scratch.eq, h->scratch.block_eq);
+    scan_blocks_kernel<<<1, 1024, 0, h->stream>>>(h->scratch.block_eq, blocks);
+    *d_total = h->scratch.block_eq + blocks;
+    return check_launch(h, "shard count") ? -1 : 2;
+}
+
+int launch_shard_finalise(slaq_handle* h, int first_unit, long long ties_before, int32_t* d_out_alloc) {
+    const int J = h->max_jobs;
+    const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
+    finalise_kernel<<<blocks, 256, 0, h->stream>>>(h->gain, h->job.count, J, h->max_cores, first_unit - 1, h->scratch.sel,
+                                                   h->scratch.gt, h->scratch.eq, h->scratch.block_eq, h->alloc,
+                                                   h->reduction, h->job.last_alloc, d_out_alloc, h->scratch.counters,
+                                                   ties_before);
+    return check_launch(h, "shard finalise") ? -1 : 1;
 }
 
 // ---------------------------------------------------------------------------------
@@ -454,14 +522,14 @@ extern "C" int slaq_allocate_static(const double* d_gain, int32_t n_jobs, int32_
     pick_first_kernel<<<1, kSelectThreads, 0, st>>>(sc->hist, &sc->sel);
     for (int pass = 1; pass < kRadixPasses; ++pass)
         select_pass_kernel<<<grid, kSelectThreads, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, pass,
-                                                           sc->hist, &sc->sel, sc->ticket, sc->gt, sc->eq);
+                                                           sc->hist, &sc->sel, sc->ticket, sc->gt, sc->eq, 1);
     const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
     count_kernel<<<blocks, 256, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, &sc->sel, sc->gt, sc->eq,
                                          sc->block_eq);
     scan_blocks_kernel<<<1, 1024, 0, st>>>(sc->block_eq, blocks);
     finalise_kernel<<<blocks, 256, 0, st>>>(d_gain, sc->every_row_active, J, cap, floor_units, &sc->sel, sc->gt, sc->eq,
                                             sc->block_eq, d_out_alloc, d_out_reduction, sc->cores_now, nullptr,
-                                            sc->counters);
+                                            sc->counters, 0);
     if (cudaGetLastError() != cudaSuccess) return SLAQ_E_CUDA;
     if (total_cores < J) return SLAQ_W_OVERSUBSCRIBED;
     if (total_cores > (long long)J * cap) return SLAQ_W_UNDERFILLED;

@@ -659,6 +659,92 @@ int slaq_allocate_only(slaq_t* h, int64_t total_cores, int32_t* out_alloc) {
     return rc;
 }
 
+// ---- one cluster sharded over several GPUs ----
+
+int slaq_get_active_count(slaq_t* h, int32_t* out_active) {
+    if (!h || !out_active) return SLAQ_E_ARG;
+    *out_active = h->n_active;
+    return SLAQ_OK;
+}
+
+int slaq_shard_predict(slaq_t* h, double epoch_seconds, int32_t with_floor) {
+    if (!h) return SLAQ_E_ARG;
+    if (!(epoch_seconds > 0.0 && std::isfinite(epoch_seconds))) return fail(h, SLAQ_E_ARG, "epoch_seconds must be positive");
+    const int rc = ensure_weights(h);
+    if (rc) return rc;
+    cudaStream_t st = h->stream;
+    int launches = 0, k;
+    h->shard_first_unit = with_floor ? 2 : 1;
+    CK(cudaMemsetAsync(h->scratch.hist, 0, h->scratch.zero_bytes, st), "clear scratch");
+    CK(cudaEventRecord(h->ev[0], st), "event");
+    if ((k = launch_fit(h)) < 0) return SLAQ_E_CUDA;
+    launches += k;
+    CK(cudaEventRecord(h->ev[1], st), "event");
+    if ((k = launch_gain(h, epoch_seconds, h->shard_first_unit)) < 0) return SLAQ_E_CUDA;
+    launches += k;
+    CK(cudaEventRecord(h->ev[2], st), "event");
+    CK(cudaEventRecord(h->ev[3], st), "event");
+    h->have_epoch = true;
+    h->last_launches = launches;
+    return SLAQ_OK;
+}
+
+int slaq_shard_histogram(slaq_t* h, int32_t pass, uint64_t* d_hist, int32_t import_it) {
+    if (!h || !d_hist) return SLAQ_E_ARG;
+    if (pass < 0 || pass >= kRadixPasses) return fail(h, SLAQ_E_ARG, "pass outside 0..5");
+    unsigned long long* mine = h->scratch.hist + (size_t)pass * kRadixBins;
+    const size_t bytes = sizeof(unsigned long long) * kRadixBins;
+    if (import_it)
+        CK(cudaMemcpyAsync(mine, d_hist, bytes, cudaMemcpyDeviceToDevice, h->stream), "import histogram");
+    else
+        CK(cudaMemcpyAsync(d_hist, mine, bytes, cudaMemcpyDeviceToDevice, h->stream), "export histogram");
+    return SLAQ_OK;
+}
+
+int slaq_shard_pick(slaq_t* h, int32_t pass, int64_t want) {
+    if (!h) return SLAQ_E_ARG;
+    if (pass < 0 || pass >= kRadixPasses) return fail(h, SLAQ_E_ARG, "pass outside 0..5");
+    const int k = launch_shard_pick(h, pass, want);
+    if (k < 0) return SLAQ_E_CUDA;
+    h->last_launches += k;
+    return SLAQ_OK;
+}
+
+int slaq_shard_pass(slaq_t* h, int32_t pass) {
+    if (!h) return SLAQ_E_ARG;
+    if (pass < 1 || pass >= kRadixPasses) return fail(h, SLAQ_E_ARG, "pass outside 1..5");
+    const int k = launch_shard_pass(h, pass, h->shard_first_unit);
+    if (k < 0) return SLAQ_E_CUDA;
+    h->last_launches += k;
+    return SLAQ_OK;
+}
+
+int slaq_shard_count(slaq_t* h, int64_t* out_local_ties) {
+    if (!h || !out_local_ties) return SLAQ_E_ARG;
+    const long long* d_total = nullptr;
+    const int k = launch_shard_count(h, h->shard_first_unit, &d_total);
+    if (k < 0) return SLAQ_E_CUDA;
+    h->last_launches += k;
+    long long total = 0;
+    CK(cudaMemcpyAsync(&total, d_total, sizeof total, cudaMemcpyDeviceToHost, h->stream), "read tie count");
+    CK(cudaStreamSynchronize(h->stream), "read tie count");
+    *out_local_ties = total;
+    return SLAQ_OK;
+}
+
+int slaq_shard_finalise(slaq_t* h, int64_t ties_before, int32_t* out_alloc) {
+    if (!h) return SLAQ_E_ARG;
+    if (!out_alloc) return fail(h, SLAQ_E_ARG, "out_alloc is null");
+    if (ties_before < 0) return fail(h, SLAQ_E_ARG, "ties_before must not be negative");
+    const int k = launch_shard_finalise(h, h->shard_first_unit, ties_before, nullptr);
+    if (k < 0) return SLAQ_E_CUDA;
+    h->last_launches += k;
+    CK(cudaEventRecord(h->ev[3], h->stream), "event");
+    CK(cudaMemcpyAsync(out_alloc, h->alloc, sizeof(int32_t) * (size_t)h->max_jobs, cudaMemcpyDeviceToHost, h->stream),
+       "copy allocation");
+    return check_device_errors(h);
+}
+
 int slaq_get_predictions(slaq_t* h, double* out_reduction, double* out_gain, int8_t* out_family, double* out_params,
                          double* out_residual, int32_t* out_status, int32_t* out_sweeps, double* out_largest) {
     if (!h) return SLAQ_E_ARG;

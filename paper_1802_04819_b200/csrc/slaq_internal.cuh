@@ -114,6 +114,7 @@ struct slaq_handle {
     std::vector<uint8_t> in_packed;   // host: job's row lives in the packed pool
     uint32_t stamp_epoch = 0;
     int32_t n_active = 0;
+    int shard_first_unit = 2;         // set by slaq_shard_predict for the steps that follow
     std::string err;
 };
 
@@ -126,5 +127,9 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
 int launch_normalise_export(slaq_handle* h, int32_t n, const int64_t* d_offsets, double* d_changes,
                             double* d_levels, double* d_largest);
 int launch_time_model(slaq_handle* h, double* d_s, double* d_w);
+int launch_shard_pick(slaq_handle* h, int pass, long long want);
+int launch_shard_pass(slaq_handle* h, int pass, int first_unit);
+int launch_shard_count(slaq_handle* h, int first_unit, const long long** d_total);
+int launch_shard_finalise(slaq_handle* h, int first_unit, long long ties_before, int32_t* d_out_alloc);
 
 }  // namespace slaq

@@ -1,0 +1,100 @@
+"""One cluster sharded over several GPUs: the driver of the step-by-step calls.
+
+Shard r holds a contiguous block of the cluster's job ids (block r, in global order) in its
+own ``Scheduler``.  The driver below runs the protocol of ``include/slaq.h`` ("One cluster
+sharded over several GPUs"): per radix pass one sum of a 2048-entry histogram over the shards,
+at the end one gather of each shard's number of threshold-equal gains.  Two ways to exchange:
+
+* ``ProcessGroupExchange``: one shard per process, ``torch.distributed`` (NCCL) does the sums;
+* ``LocalExchange``: several shards in one process on one GPU, summed directly - the same
+  steps in the same order, used to check the protocol where only one GPU is available.
+"""
+
+from __future__ import annotations
+
+N_PASSES = 6
+N_BINS = 2048
+
+
+class LocalExchange:
+    """All shards live in this process."""
+
+    def sum_ints(self, values):
+        total = sum(int(v) for v in values)
+        return [total] * len(values)
+
+    def sum_histograms(self, buffers):
+        total = buffers[0].clone()
+        for b in buffers[1:]:
+            total += b
+        for b in buffers:
+            b.copy_(total)
+
+    def gather_ints(self, values):
+        allv = [int(v) for v in values]
+        return [allv] * len(values)
+
+    def ranks(self, n_local):
+        return list(range(n_local))
+
+
+class ProcessGroupExchange:
+    """One shard per process; ``torch.distributed`` must be initialised (NCCL for GPU tensors)."""
+
+    def __init__(self, group=None, device="cuda"):
+        import torch.distributed as dist
+        self.dist, self.group, self.device = dist, group, device
+
+    def sum_ints(self, values):
+        import torch
+        assert len(values) == 1
+        t = torch.tensor([int(values[0])], dtype=torch.int64, device=self.device)
+        self.dist.all_reduce(t, group=self.group)
+        return [int(t.item())]
+
+    def sum_histograms(self, buffers):
+        assert len(buffers) == 1
+        self.dist.all_reduce(buffers[0], group=self.group)
+
+    def gather_ints(self, values):
+        import torch
+        world = self.dist.get_world_size(self.group)
+        t = torch.tensor([int(values[0])], dtype=torch.int64, device=self.device)
+        out = [torch.zeros_like(t) for _ in range(world)]
+        self.dist.all_gather(out, t, group=self.group)
+        return [[int(o.item()) for o in out]]
+
+    def ranks(self, n_local):
+        return [self.dist.get_rank(self.group)]
+
+
+def schedule_sharded(shards, exchange, epoch_seconds: float, total_cores: int):
+    """One epoch of one cluster whose jobs are split over ``shards`` (list of ``Scheduler``; one entry
+    per process with ``ProcessGroupExchange``).  Returns the list of per-shard allocations."""
+    import torch
+    cap = shards[0].max_cores_per_job
+    assert all(s.max_cores_per_job == cap for s in shards)
+    n_jobs = exchange.sum_ints([s.get_active_count() for s in shards])[0]
+    with_floor = total_cores >= n_jobs
+    want = min(total_cores, n_jobs * cap) - (n_jobs if with_floor else 0)
+    for s in shards:
+        s.shard_predict(epoch_seconds, with_floor)
+    buffers = [torch.zeros(N_BINS, dtype=torch.int64, device="cuda") for _ in shards]
+    for p in range(N_PASSES):
+        if p > 0:
+            for s in shards:
+                s.shard_pass(p)
+        for s, b in zip(shards, buffers):
+            s.shard_histogram(p, b, import_it=False)
+        torch.cuda.synchronize()          # the library's stream and the collective's stream meet here
+        exchange.sum_histograms(buffers)
+        torch.cuda.synchronize()
+        for s, b in zip(shards, buffers):
+            s.shard_histogram(p, b, import_it=True)
+            s.shard_pick(p, want)
+    ties = [s.shard_count() for s in shards]
+    gathered = exchange.gather_ints(ties)
+    out = []
+    for s, all_ties, rank in zip(shards, gathered, exchange.ranks(len(shards))):
+        out.append(s.shard_finalise(sum(all_ties[:rank])))
+    return out

@@ -42,6 +42,41 @@ def test_two_ranks_partition_and_timing():
     assert a["checksums"][0] != a["checksums"][1]             # the two partitions hold different jobs
 
 
+def _exchange_worker(rank, world, port, out):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    from paper_1802_04819_b200.sharded import N_BINS, ProcessGroupExchange
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        ex = ProcessGroupExchange(device="cpu")
+        hist = torch.arange(N_BINS, dtype=torch.int64) * (rank + 1)
+        ex.sum_histograms([hist])
+        out[rank] = dict(total=ex.sum_ints([10 + rank]), ties=ex.gather_ints([7 * (rank + 1)]), ranks=ex.ranks(1),
+                         hist_ok=bool((hist == torch.arange(N_BINS) * 3).all()))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_shard_exchange_over_a_process_group():
+    """What the shards of one cluster exchange per epoch (sums of histograms and counts, gathered tie counts),
+    over gloo on CPU; on GPUs the same calls run over NCCL."""
+    world, port = 2, 29931 + os.getpid() % 400
+    out = mp.Manager().dict()
+    mp.spawn(_exchange_worker, args=(world, port, out), nprocs=world, join=True)
+    for rank in range(world):
+        assert out[rank]["total"] == [21]
+        assert out[rank]["ties"] == [[7, 14]]
+        assert out[rank]["ranks"] == [rank]
+        assert out[rank]["hist_ok"]
+    # the local exchange used on one GPU gives every shard the same answers
+    from paper_1802_04819_b200.sharded import LocalExchange
+    ex = LocalExchange()
+    assert ex.sum_ints([10, 11]) == [21, 21] and ex.gather_ints([7, 14]) == [[7, 14], [7, 14]] and ex.ranks(2) == [0, 1]
+    a, b = torch.arange(4), torch.arange(4) * 2
+    ex.sum_histograms([a, b])
+    assert (a == torch.arange(4) * 3).all() and (b == a).all()
+
+
 def test_single_process_is_identity():
     from paper_1802_04819_b200.partition import max_over_ranks, whole_job_rate
     assert max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
