@@ -398,6 +398,7 @@ __device__ __forceinline__ void sweep(const Lanes& S, int fam, int H, int k_all,
     double md = (double)S.l;
     const double dL = (double)S.L;
     const double* yp = S.y + S.lane;
+#pragma unroll 1   // unrolling only adds register pressure here: the body already holds 22 independent sums
     for (int k = 0, m = S.l; k < k_all; ++k, m += S.L, md += dL, yp += 32) {
         if (m < H) {
             const double x = -md * inv_span;
