@@ -8,13 +8,14 @@
 // (newest point x = 0, oldest x = -1); the family with the lower weighted residual wins.
 //
 // Work split.  Jobs are sorted by window length (counting sort, longest first) and cut into
-// length classes.  In class c a group of L lanes (L = 1, 2, .. 32, chosen so that a warp's
+// length classes.  In class c a group of L lanes (L = 2, 4, .. 32, chosen so that a warp's
 // windows fit its shared-memory slice) owns one job, so a warp carries 32/L jobs.  One
-// persistent launch serves all classes from one work queue, longest windows first.  A lane walks its job's points m = l, l + L, l + 2L, ... counted
-// from the newest one; both families are evaluated in the same sweep over the window; the
-// partial sums of the normal equations are reduced over the L lanes with shuffles; every
-// lane of a group then runs the same small solve for its job.  All per-job control flow is
-// per lane, so the jobs of a warp may be in different phases of the solver.
+// persistent launch serves all classes from one work queue, longest windows first.  A lane
+// walks its job's points m = l, l + L, l + 2L, ... counted from the newest one; both families
+// are evaluated in the same sweep over the window; the partial sums of the normal equations
+// are reduced over the L lanes with shuffles; the even lanes of a group then run family I's
+// solver step for the job and the odd lanes family II's.  All per-job control flow is per
+// lane, so the jobs of a warp may be in different phases of the solver.
 #include <math_constants.h>
 
 #include <algorithm>
