@@ -821,7 +821,7 @@ normalise_export_kernel(JobArrays job, const int32_t* __restrict__ ids, const in
 // in shared memory, lanes with equal lengths adding once, and each block then adds its non-zero
 // bins to the global table.
 constexpr int kSortThreads = 256;
-constexpr int kSortJobsPerBlock = 8192;
+constexpr int kSortJobsPerBlock = 2048;
 
 __device__ __forceinline__ int clamped_length(const int32_t* __restrict__ count, int j, int max_hist) {
     const int H = count[j];
