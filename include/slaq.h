@@ -28,6 +28,7 @@
  *   - The handle owns all scheduler state on the device.  Calls on one handle must not
  *     overlap; work is ordered on the handle's stream (slaq_set_stream).  Functions
  *     that take or fill host buffers return after the stream has finished that work.
+ *   - Calls on a handle must be made with the handle's device current (SLAQ_E_ARG otherwise).
  *   - Job ids are 0 .. max_jobs-1.  A job is active from its first loss until removed.
  *   - The library needs a CUDA device: there is no CPU path.
  */

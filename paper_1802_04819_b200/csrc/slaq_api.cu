@@ -219,7 +219,16 @@ __global__ void set_time_kernel(JobArrays job, int max_jobs, int n, const int32_
     job.w_set[j] = w[i];
 }
 
+// Kernels and copies go to the current device: it must be the one the handle lives on.
+int check_device(slaq_handle* h) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return fail(h, SLAQ_E_CUDA, "cudaGetDevice failed");
+    if (dev != h->device) return fail(h, SLAQ_E_ARG, "the handle was created on another device than the current one");
+    return SLAQ_OK;
+}
+
 int check_ids(slaq_handle* h, int32_t n, const int32_t* ids, bool forbid_dups) {
+    if (const int rc = check_device(h)) return rc;
     if (n < 0) return fail(h, SLAQ_E_ARG, "negative count");
     if (n > 0 && !ids) return fail(h, SLAQ_E_ARG, "job_ids is null");
     if (n > h->max_jobs) return fail(h, SLAQ_E_ARG, "more entries than job ids");
@@ -432,6 +441,7 @@ int do_load(slaq_handle* h, int32_t n, const int32_t* ids, const int64_t* offset
 int run_epoch(slaq_handle* h, double T, int64_t C, int32_t* d_out, bool only_allocate) {
     if (!only_allocate && !(T > 0.0 && std::isfinite(T))) return fail(h, SLAQ_E_ARG, "epoch_seconds must be positive");
     if (C < 0) return fail(h, SLAQ_E_ARG, "total_cores must not be negative");
+    if (const int dc = check_device(h)) return dc;
     const int rc = ensure_weights(h);
     if (rc) return rc;
     const int64_t active = h->n_active, cap = h->max_cores;
@@ -670,6 +680,7 @@ int slaq_get_active_count(slaq_t* h, int32_t* out_active) {
 int slaq_shard_predict(slaq_t* h, double epoch_seconds, int32_t with_floor) {
     if (!h) return SLAQ_E_ARG;
     if (!(epoch_seconds > 0.0 && std::isfinite(epoch_seconds))) return fail(h, SLAQ_E_ARG, "epoch_seconds must be positive");
+    if (const int dc = check_device(h)) return dc;
     const int rc = ensure_weights(h);
     if (rc) return rc;
     cudaStream_t st = h->stream;
