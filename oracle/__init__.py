@@ -43,6 +43,10 @@ def _bind(lib):
     lib.oracle_normalise.argtypes = [c_i64, vp, vp, vp, vp, vp, vp]
     lib.oracle_predict.argtypes = [c_i64, vp, vp, vp, vp, vp, c_f64, c_i32, c_f64, c_i32, c_i32,
                                    vp, vp, vp, vp, vp, vp, vp]
+    lib.oracle_predict_warm.argtypes = [c_i64, vp, vp, vp, vp, vp, c_f64, c_i32, c_f64, c_i32, c_i32,
+                                        vp, vp, vp, vp, vp, vp, vp] + [vp] * 8
+    lib.oracle_carry.argtypes = [c_i32, vp, c_f64, c_f64, c_f64, vp]
+    lib.oracle_carry.restype = None
     lib.oracle_allocate.argtypes = [c_i64, c_i32, vp, vp, c_i64, vp]
     lib.oracle_allocate.restype = c_i64
     lib.oracle_reduction_at.argtypes = [c_i64, c_i32, vp, vp, vp]
@@ -94,8 +98,13 @@ def normalise(offsets, losses, m_seen=None):
 
 
 def predict(offsets, losses, m_seen, s, w, epoch_seconds, cap, gamma=0.9, lm_trials=20, threads=0,
-            want_gain=True):
-    """Steps 1-3.  Returns a dict with family, params, S, status, evals, M and gain [J, cap]."""
+            want_gain=True, k_last=None, warm=None):
+    """Steps 1-3.  Returns a dict with family, params, S, status, evals, M, gain [J, cap], and both
+    families' final parameters (`both` [J, 8], `mask`).
+
+    warm: dict(valid uint8 [J], p [J, 8], K int64 [J], span [J], M [J]) from an earlier epoch; the
+    families it covers start from those parameters carried into this epoch's coordinates
+    (k_last = index of each job's newest iteration now)."""
     lib = _load()
     offsets, losses = _i64(offsets), _f64(losses)
     J = offsets.size - 1
@@ -105,10 +114,27 @@ def predict(offsets, losses, m_seen, s, w, epoch_seconds, cap, gamma=0.9, lm_tri
         family=np.empty(J, np.int8), params=np.empty((J, 4)), S=np.empty((J, 2)),
         status=np.empty(J, np.int32), evals=np.empty((J, 2), np.int32), M=np.empty(J),
         gain=np.empty((J, cap)) if want_gain else None,
+        both=np.empty((J, 8)), mask=np.empty(J, np.uint8),
     )
-    lib.oracle_predict(J, _p(offsets), _p(losses), _p(m_seen), _p(s), _p(w), float(epoch_seconds), int(cap),
-                       float(gamma), int(lm_trials), int(threads), _p(out["family"]), _p(out["params"]),
-                       _p(out["S"]), _p(out["status"]), _p(out["evals"]), _p(out["M"]), _p(out["gain"]))
+    wv = wp = wK = wS = wM = None
+    if warm is not None:
+        wv = np.ascontiguousarray(warm["valid"], dtype=np.uint8)
+        wp, wK, wS, wM = _f64(warm["p"]), _i64(warm["K"]), _f64(warm["span"]), _f64(warm["M"])
+        k_last = _i64(k_last)
+    lib.oracle_predict_warm(J, _p(offsets), _p(losses), _p(m_seen), _p(s), _p(w), float(epoch_seconds), int(cap),
+                            float(gamma), int(lm_trials), int(threads), _p(out["family"]), _p(out["params"]),
+                            _p(out["S"]), _p(out["status"]), _p(out["evals"]), _p(out["M"]), _p(out["gain"]),
+                            _p(k_last) if warm is not None else None, _p(wv), _p(wp), _p(wK), _p(wS), _p(wM),
+                            _p(out["both"]), _p(out["mask"]))
+    return out
+
+
+def carry(family, p, t, r, sigma):
+    """A family's parameters in window coordinates shifted by t, stretched by r, levels scaled by sigma."""
+    lib = _load()
+    p = _f64(p)
+    out = np.empty(4)
+    lib.oracle_carry(int(family), _p(p), float(t), float(r), float(sigma), _p(out))
     return out
 
 
@@ -144,9 +170,11 @@ def time_model(cnt, su, suu, st, sut, stn, umin, umax):
     return s, w
 
 
-def schedule(offsets, losses, m_seen, s, w, epoch_seconds, total_cores, cap, gamma=0.9, lm_trials=20, threads=0):
+def schedule(offsets, losses, m_seen, s, w, epoch_seconds, total_cores, cap, gamma=0.9, lm_trials=20, threads=0,
+             k_last=None, warm=None):
     """One whole epoch on CSR histories.  Returns dict(alloc, R, gain, ...fit record)."""
-    out = predict(offsets, losses, m_seen, s, w, epoch_seconds, cap, gamma, lm_trials, threads)
+    out = predict(offsets, losses, m_seen, s, w, epoch_seconds, cap, gamma, lm_trials, threads,
+                  k_last=k_last, warm=warm)
     active = (np.diff(_i64(offsets)) > 0)
     out["alloc"] = allocate(out["gain"], active, total_cores)
     out["R"] = reduction_at(out["gain"], out["alloc"])
@@ -200,6 +228,30 @@ class OracleScheduler:
         self.s_set = np.full(max_jobs, np.nan)
         self.w_set = np.full(max_jobs, np.nan)
         self.last_alloc = np.ones(max_jobs, np.int32)
+        # warm start: `fitted` is what the last epoch found, `warm` what the next fit starts from.
+        # A job's `warm` is refreshed from `fitted` when its history changes, so an epoch repeated
+        # without new losses starts from the same point and gives the same result.
+        self.warm_start = False
+        self.fitted = self._no_fit(max_jobs)
+        self.warm = self._no_fit(max_jobs)
+
+    @staticmethod
+    def _no_fit(n):
+        return dict(valid=np.zeros(n, np.uint8), p=np.full((n, 8), np.nan), K=np.zeros(n, np.int64),
+                    span=np.ones(n), M=np.full(n, np.nan))
+
+    def _carry_over(self, j):
+        for key in self.warm:
+            self.warm[key][j] = self.fitted[key][j]
+
+    def _forget_fit(self, j):
+        self.fitted["valid"][j] = 0
+        self.warm["valid"][j] = 0
+
+    def set_fit_state(self, state):
+        """Make `state` (dict valid, p, K, span, M) the starting point of every job's next fit."""
+        self.fitted = {k: np.array(state[k]) for k in ("valid", "p", "K", "span", "M")}
+        self.warm = {k: np.array(state[k]) for k in ("valid", "p", "K", "span", "M")}
 
     def append_losses(self, job_ids, losses, iter_times=None, cores_used=None):
         for i, j in enumerate(job_ids):
@@ -209,6 +261,7 @@ class OracleScheduler:
                 self.m_seen[j] = max(self.m_seen[j], win[-1] - loss)
             win.append(loss)
             self.k_last[j] += 1
+            self._carry_over(j)
             if iter_times is not None:
                 n = int(cores_used[i]) if cores_used is not None else max(int(self.last_alloc[j]), 1)
                 t = float(iter_times[i])
@@ -223,6 +276,7 @@ class OracleScheduler:
             self.window[j] = deque((float(v) for v in rows[-self.max_hist:]), maxlen=self.max_hist)
             self.k_last[j] = int(k_last[i])
             self.m_seen[j] = -np.inf if m_seen is None else float(m_seen[i])
+            self._forget_fit(j)
 
     def set_time_model(self, job_ids, s, w):
         for i, j in enumerate(job_ids):
@@ -237,6 +291,7 @@ class OracleScheduler:
             self.umin[j], self.umax[j] = np.inf, -np.inf
             self.s_set[j] = self.w_set[j] = np.nan
             self.last_alloc[j] = 1
+            self._forget_fit(j)
 
     def time_model(self):
         s, w = time_model(*(self.tm[:, i] for i in range(6)), self.umin, self.umax)
@@ -254,8 +309,12 @@ class OracleScheduler:
         offsets, losses = self.csr()
         s, w = self.time_model()
         out = schedule(offsets, losses, self.m_seen, s, w, epoch_seconds, total_cores, self.cap,
-                       self.gamma, self.lm_trials, threads)
-        active = np.diff(offsets) > 0
+                       self.gamma, self.lm_trials, threads, k_last=self.k_last,
+                       warm=self.warm if self.warm_start else None)
+        H = np.diff(offsets)
+        self.fitted = dict(valid=out["mask"].copy(), p=out["both"].copy(), K=self.k_last.copy(),
+                           span=np.maximum(H - 1, 1).astype(np.float64), M=out["M"].copy())
+        active = H > 0
         self.last_alloc = np.where(active, out["alloc"], self.last_alloc).astype(np.int32)
         out["s"], out["w"] = s, w
         return out

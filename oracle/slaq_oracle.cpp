@@ -431,7 +431,47 @@ FitData make_fit_data(const double* loss, int64_t H, double M, double gamma) {
     return D;
 }
 
+// ---------------------------------------------------------------------------------
+// Warm start ("short time intervals ... continued rebalancing", Evaluation,
+// "Scalability and efficiency"): a scheduler that refits every few seconds may start
+// each family from the parameters it found last epoch instead of from the linearised
+// first guess.  The paper does not say how its fits are started; this is this
+// implementation's rule.  The fitted curve is a function of the iteration index k and
+// the raw loss, but its parameters are kept in window coordinates, and those move from
+// epoch to epoch: with x0 = (k - K0)/span0 and y0 = l/M0 last epoch, x = (k - K)/span and
+// y = l/M now,
+//     x0 = t + r x,  t = (K - K0)/span0,  r = span/span0,      y = sigma y0,  sigma = M0/M.
+// Substituting into either family gives the same curve in the new coordinates.
+// ---------------------------------------------------------------------------------
+struct WarmStart {
+    uint8_t valid = 0;   // bit 0: family I parameters present, bit 1: family II
+    double pI[4] = {kNaN, kNaN, kNaN, kNaN};
+    double pII[4] = {kNaN, kNaN, kNaN, kNaN};
+    int64_t K = 0;       // index of the newest iteration when the parameters were fitted
+    double span = 1.0;   // their window span
+    double M = kNaN;     // their scale
+};
+
+// 1/(a x0^2 + b x0 + c) + d with x0 = t + r x, times sigma.
+void carry_sublinear(const double* p, double t, double r, double sigma, double* out) {
+    const double a = p[0], b = p[1], c = p[2], d = p[3];
+    out[0] = a * r * r / sigma;
+    out[1] = (2.0 * a * t + b) * r / sigma;
+    out[2] = ((a * t + b) * t + c) / sigma;
+    out[3] = sigma * d;
+}
+
+// (exp(alpha - beta x0) + c) sigma with x0 = t + r x.
+void carry_exponential(const double* p, double t, double r, double sigma, double* out) {
+    out[0] = p[0] - p[1] * t + std::log(sigma);
+    out[1] = p[1] * r;
+    out[2] = sigma * p[2];
+    out[3] = 0.0;
+}
+
 struct JobFit {
+    uint8_t fitted_mask = 0;       // bit 0 / 1: family I / II ended with a finite residual
+    double both[8] = {kNaN, kNaN, kNaN, kNaN, kNaN, kNaN, kNaN, kNaN};   // final parameters of I then II
     int32_t status = ST_INACTIVE;
     int8_t family = -1;            // 0 = sublinear, 1 = exponential, -1 = none
     double params[4] = {kNaN, kNaN, kNaN, kNaN};
@@ -443,8 +483,11 @@ struct JobFit {
     double span = 1.0;
 };
 
-// Steps 1 and 2 for one job.
-JobFit fit_job(const double* loss, int64_t H, double m_seen, const Settings& cfg) {
+// Steps 1 and 2 for one job.  With `warm` (and K, the index of the newest iteration), a
+// family whose carried-over parameters give a finite residual starts from them; otherwise,
+// and always without `warm`, it starts from its first guess.
+JobFit fit_job(const double* loss, int64_t H, double m_seen, const Settings& cfg, const WarmStart* warm = nullptr,
+               int64_t K = 0) {
     JobFit out;
     if (H <= 0) return out;
     if (!all_finite(loss, H) || std::isnan(m_seen) || m_seen == kInf) {
@@ -471,12 +514,44 @@ JobFit fit_job(const double* loss, int64_t H, double m_seen, const Settings& cfg
     bool fitted = false;
     if (H >= cfg.min_fit_points) {
         double pI[4], pII[4];
-        init_sublinear(D, pI);
-        const LmOutcome rI = levenberg_marquardt<Sublinear>(pI, D, cfg.lm_trials, 1e-3);
-        init_exponential(D, pII);
-        const LmOutcome rII = levenberg_marquardt<Exponential>(pII, D, cfg.lm_trials, 1e-3);
-        out.evals[0] = rI.evals;
-        out.evals[1] = rII.evals;
+        LmOutcome rI, rII;
+        int spentI = 0, spentII = 0;   // the sweep of a carried-over start that was not usable
+        bool startedI = false, startedII = false;
+        if (warm && warm->valid && warm->span > 0.0 && warm->M > 0.0 && std::isfinite(warm->M)) {
+            const double t = (double)(K - warm->K) / warm->span;
+            const double r = D.span / warm->span;
+            const double sigma = warm->M / M;
+            if (warm->valid & 1) {
+                carry_sublinear(warm->pI, t, r, sigma, pI);
+                rI = levenberg_marquardt<Sublinear>(pI, D, cfg.lm_trials, 1e-3);
+                startedI = rI.ok;
+                spentI = startedI ? 0 : 1;
+            }
+            if (warm->valid & 2) {
+                carry_exponential(warm->pII, t, r, sigma, pII);
+                rII = levenberg_marquardt<Exponential>(pII, D, cfg.lm_trials, 1e-3);
+                startedII = rII.ok;
+                spentII = startedII ? 0 : 1;
+            }
+        }
+        if (!startedI) {
+            init_sublinear(D, pI);
+            rI = levenberg_marquardt<Sublinear>(pI, D, cfg.lm_trials, 1e-3);
+        }
+        if (!startedII) {
+            init_exponential(D, pII);
+            rII = levenberg_marquardt<Exponential>(pII, D, cfg.lm_trials, 1e-3);
+        }
+        out.evals[0] = rI.evals + spentI;
+        out.evals[1] = rII.evals + spentII;
+        if (rI.ok && std::isfinite(rI.S)) {
+            out.fitted_mask |= 1;
+            std::memcpy(out.both, pI, sizeof pI);
+        }
+        if (rII.ok && std::isfinite(rII.S)) {
+            out.fitted_mask |= 2;
+            std::memcpy(out.both + 4, pII, sizeof pII);
+        }
         if (rI.ok) out.S[0] = rI.S;
         if (rII.ok) out.S[1] = rII.S;
         const bool okI = rI.ok && std::isfinite(rI.S);
@@ -664,10 +739,17 @@ int oracle_normalise(int64_t n_jobs, const int64_t* offsets, const double* losse
 }
 
 // Steps 1-3 over CSR histories: fit record and gain rows gain[j*cap + (n-1)], n = 1..cap.
-int oracle_predict(int64_t n_jobs, const int64_t* offsets, const double* losses, const double* m_seen,
-                   const double* s, const double* w, double epoch_seconds, int32_t cap, double gamma,
-                   int32_t lm_trials, int32_t threads, int8_t* out_family, double* out_params,
-                   double* out_S, int32_t* out_status, int32_t* out_evals, double* out_M, double* out_gain) {
+// With warm_valid: the warm-started variant; warm_p holds [n_jobs][8] (family I then II),
+// warm_K / warm_span / warm_M the coordinates those parameters refer to, k_last the index of
+// each job's newest iteration now.  out_both [n_jobs][8] and out_mask receive both families'
+// final parameters and which of them ended with a finite residual.
+int oracle_predict_warm(int64_t n_jobs, const int64_t* offsets, const double* losses, const double* m_seen,
+                        const double* s, const double* w, double epoch_seconds, int32_t cap, double gamma,
+                        int32_t lm_trials, int32_t threads, int8_t* out_family, double* out_params,
+                        double* out_S, int32_t* out_status, int32_t* out_evals, double* out_M, double* out_gain,
+                        const int64_t* k_last, const uint8_t* warm_valid, const double* warm_p,
+                        const int64_t* warm_K, const double* warm_span, const double* warm_M, double* out_both,
+                        uint8_t* out_mask) {
     Settings cfg;
     cfg.gamma = gamma;
     cfg.lm_trials = lm_trials;
@@ -675,7 +757,19 @@ int oracle_predict(int64_t n_jobs, const int64_t* offsets, const double* losses,
 #pragma omp parallel for schedule(dynamic, 16)
     for (int64_t j = 0; j < n_jobs; ++j) {
         const int64_t lo = offsets[j], H = offsets[j + 1] - lo;
-        JobFit fit = fit_job(losses + lo, H, m_seen ? m_seen[j] : -kInf, cfg);
+        WarmStart warm;
+        if (warm_valid && warm_valid[j]) {
+            warm.valid = warm_valid[j];
+            std::memcpy(warm.pI, warm_p + 8 * j, sizeof warm.pI);
+            std::memcpy(warm.pII, warm_p + 8 * j + 4, sizeof warm.pII);
+            warm.K = warm_K[j];
+            warm.span = warm_span[j];
+            warm.M = warm_M[j];
+        }
+        JobFit fit = fit_job(losses + lo, H, m_seen ? m_seen[j] : -kInf, cfg, warm.valid ? &warm : nullptr,
+                             k_last ? k_last[j] : 0);
+        if (out_both) std::memcpy(out_both + 8 * j, fit.both, sizeof fit.both);
+        if (out_mask) out_mask[j] = fit.fitted_mask;
         const bool has_time = std::isfinite(s[j]) && std::isfinite(w[j]) && w[j] > 0.0 && s[j] >= 0.0;
         if (fit.status != ST_INACTIVE && fit.status != ST_NONFINITE && fit.status != ST_FLAT && !has_time)
             fit.status = ST_NO_TIME;
@@ -694,6 +788,15 @@ int oracle_predict(int64_t n_jobs, const int64_t* offsets, const double* losses,
         if (out_gain) job_gains(fit, s[j], w[j], epoch_seconds, cap, out_gain + (int64_t)j * cap);
     }
     return 0;
+}
+
+int oracle_predict(int64_t n_jobs, const int64_t* offsets, const double* losses, const double* m_seen,
+                   const double* s, const double* w, double epoch_seconds, int32_t cap, double gamma,
+                   int32_t lm_trials, int32_t threads, int8_t* out_family, double* out_params,
+                   double* out_S, int32_t* out_status, int32_t* out_evals, double* out_M, double* out_gain) {
+    return oracle_predict_warm(n_jobs, offsets, losses, m_seen, s, w, epoch_seconds, cap, gamma, lm_trials, threads,
+                               out_family, out_params, out_S, out_status, out_evals, out_M, out_gain, nullptr,
+                               nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
 }
 
 // Step 4 alone on given gain rows.  Returns cores handed out.
@@ -737,6 +840,12 @@ int oracle_lm_line(int64_t H, const double* x, const double* y, const double* w,
     const LmOutcome r = levenberg_marquardt<Line>(p, D, trials, lambda0);
     *out_S = r.S;
     return r.ok ? r.evals : -1;
+}
+
+// A family's parameters carried into new window coordinates (x_old = t + r x_new, y_new = sigma y_old).
+void oracle_carry(int32_t family, const double* p, double t, double r, double sigma, double* out) {
+    if (family == 0) carry_sublinear(p, t, r, sigma, out);
+    else carry_exponential(p, t, r, sigma, out);
 }
 
 // Fit one family only, from its own initial guess, on one history; returns sweeps used or -1.

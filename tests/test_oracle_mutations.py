@@ -12,6 +12,7 @@ import test_oracle_allocate as t_alloc
 import test_oracle_fit as t_fit
 import test_oracle_gains as t_gains
 import test_oracle_normalise as t_norm
+import test_oracle_warm_start as t_warm
 
 SRC = Path(__file__).resolve().parent.parent / "oracle" / "slaq_oracle.cpp"
 
@@ -43,6 +44,13 @@ MUTATIONS = [
     ("no one-core floor", "alloc[j] = 1;\n                ++handed;", "alloc[j] = 0;"),
     ("time law: slope and intercept mixed up", "const double ss = (st - ww * su) / cnt;",
      "const double ss = (st + ww * su) / cnt;"),
+    ("warm start: family I carried without the shift of the origin", "out[1] = (2.0 * a * t + b) * r / sigma;",
+     "out[1] = b * r / sigma;"),
+    ("warm start: family II carried without the change of scale", "out[0] = p[0] - p[1] * t + std::log(sigma);",
+     "out[0] = p[0] - p[1] * t;"),
+    ("warm start: stretch of the window inverted", "const double r = D.span / warm->span;",
+     "const double r = warm->span / D.span;"),
+    ("warm start: an unusable carried point is kept", "startedI = rI.ok;", "startedI = true;"),
 ]
 
 PINS = [
@@ -58,6 +66,9 @@ PINS = [
     lambda m: t_alloc.test_greedy_equals_brute_force_on_tiny_clusters(m),
     lambda m: t_alloc.test_capacity_and_floor(m),
     lambda m: t_alloc.test_ties_go_to_the_lowest_job_id(m),
+    lambda m: [t_warm.test_carried_parameters_describe_the_same_curve(m, f) for f in (0, 1)],
+    lambda m: t_warm.test_the_solver_never_ends_above_its_carried_starting_point(m),
+    lambda m: t_warm.test_an_unusable_carried_point_falls_back_to_the_first_guess(m),
 ]
 
 
