@@ -62,8 +62,17 @@ enum {
     SLAQ_P_LM_TRIALS = 2,         /* Levenberg-Marquardt trials per family; default 20; 0 .. 1000 */
     SLAQ_P_MAX_CORES_PER_JOB = 3, /* cap on a_j; default 64; 1 .. what the handle was created for */
     SLAQ_P_MIN_FIT_POINTS = 4,    /* fewer stored points than this use linear extrapolation; default 4; >= 4 */
-    SLAQ_P_FIT_SLICE_BYTES = 5    /* tuning: shared memory one warp of the fit kernel may use (8 KB..200 KB);
+    SLAQ_P_FIT_SLICE_BYTES = 5,   /* tuning: shared memory one warp of the fit kernel may use (8 KB..200 KB);
                                      decides how many lanes share a job; results stay within rounding */
+    SLAQ_P_WARM_START = 6         /* 0 (default) or 1.  The scheduler refits every job at short intervals
+                                     (Evaluation, "Scalability and efficiency"); with 1, a family starts from the
+                                     parameters the job's last epoch ended with, carried into this epoch's window
+                                     coordinates, instead of from its linearised first guess (which it still uses
+                                     where there is no earlier fit or the carried point has no finite residual).
+                                     The starting point of a job changes only when its history changes, so
+                                     slaq_schedule stays repeatable.  Together with a smaller SLAQ_P_LM_TRIALS
+                                     this spreads a fit's iterations over the epochs.  The paper does not say how
+                                     its fits are started. */
 };
 
 /* per-job status written by slaq_schedule (slaq_get_predictions, out_status) */
@@ -220,6 +229,26 @@ int slaq_get_normalised(slaq_t* h, int32_t n, const int32_t* job_ids, int64_t ca
 
 /* Iteration-time law in use for every job (NaN where none yet).  Host pointers [max_jobs]. */
 int slaq_get_time_model(slaq_t* h, double* out_s, double* out_w);
+
+/*
+ * The fitted curves as scheduler state (for SLAQ_P_WARM_START: to carry them over a restart,
+ * or to inspect them).  Per job: both families' parameters in window coordinates
+ * (out_params [max_jobs][8]: family I a, b, c, d, then family II alpha, beta, c, and one unused
+ * slot), which of them ended with a finite residual (out_mask [max_jobs], bit 0 family I,
+ * bit 1 family II, 0 = no fit), and what the coordinates refer to: the index of the newest
+ * iteration at that fit (out_k [max_jobs]), the window span max(H-1, 1) (out_span) and the
+ * largest reduction the window was scaled by (out_scale).  slaq_get_fit_state reports the last
+ * epoch's end points.  slaq_set_fit_state makes the given entries both the last epoch's record
+ * and the starting points of each job's next fit; entries with mask 0 clear a job's.  It
+ * returns SLAQ_E_ARG for a mask above 3, a masked entry of a job without losses, or a masked
+ * entry whose span or scale is not positive and finite; parameters are not checked (a family
+ * whose carried-over point has no finite residual starts from its first guess).  Host pointers.
+ * The paper has no counterpart.
+ */
+int slaq_get_fit_state(slaq_t* h, double* out_params, uint8_t* out_mask, int64_t* out_k, double* out_span,
+                       double* out_scale);
+int slaq_set_fit_state(slaq_t* h, const double* params, const uint8_t* mask, const int64_t* k, const double* span,
+                       const double* scale);
 
 /*
  * Test hook for the allocation step alone: overwrite the gain rows (host,

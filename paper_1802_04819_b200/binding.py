@@ -10,14 +10,15 @@ import numpy as np
 from .build import LIB
 
 JOB_INACTIVE, JOB_FITTED, JOB_SHORT, JOB_NEW, JOB_FIT_FAILED, JOB_FLAT, JOB_NONFINITE, JOB_NO_TIME = -1, 0, 1, 2, 3, 4, 5, 6
-P_GAMMA, P_LM_TRIALS, P_MAX_CORES_PER_JOB, P_MIN_FIT_POINTS, P_FIT_SLICE_BYTES = 1, 2, 3, 4, 5
+P_GAMMA, P_LM_TRIALS, P_MAX_CORES_PER_JOB, P_MIN_FIT_POINTS, P_FIT_SLICE_BYTES, P_WARM_START = 1, 2, 3, 4, 5, 6
 W_OVERSUBSCRIBED, W_UNDERFILLED = 1, 2
 
 EXPORTED_SYMBOLS = [
     "slaq_create", "slaq_create_in", "slaq_workspace_bytes", "slaq_destroy", "slaq_last_error", "slaq_set_stream",
     "slaq_set_param", "slaq_get_param", "slaq_append_losses", "slaq_append_losses_ex", "slaq_load_histories",
     "slaq_load_histories_packed", "slaq_set_time_model", "slaq_remove_jobs", "slaq_schedule", "slaq_schedule_device",
-    "slaq_get_predictions", "slaq_get_normalised", "slaq_get_time_model", "slaq_set_gains", "slaq_allocate_only",
+    "slaq_get_predictions", "slaq_get_normalised", "slaq_get_time_model", "slaq_get_fit_state",
+    "slaq_set_fit_state", "slaq_set_gains", "slaq_allocate_only",
     "slaq_get_stats", "slaq_allocate_static", "slaq_get_active_count", "slaq_shard_predict", "slaq_shard_histogram",
     "slaq_shard_pick", "slaq_shard_pass", "slaq_shard_count", "slaq_shard_finalise",
 ]
@@ -73,6 +74,8 @@ def load_library():
         "slaq_get_predictions": (c_int, [vp] * 9),
         "slaq_get_normalised": (c_int, [vp, c_int32, vp, c_int64, vp, vp, vp, vp]),
         "slaq_get_time_model": (c_int, [vp, vp, vp]),
+        "slaq_get_fit_state": (c_int, [vp, vp, vp, vp, vp, vp]),
+        "slaq_set_fit_state": (c_int, [vp, vp, vp, vp, vp, vp]),
         "slaq_set_gains": (c_int, [vp, vp]),
         "slaq_allocate_only": (c_int, [vp, c_int64, vp]),
         "slaq_get_stats": (c_int, [vp, POINTER(Stats)]),
@@ -244,6 +247,23 @@ class Scheduler:
         s, w = np.empty(self.max_jobs), np.empty(self.max_jobs)
         self._check(self._lib.slaq_get_time_model(self._h, _ptr(s), _ptr(w)))
         return s, w
+
+    def get_fit_state(self):
+        """Both families' end points of the last epoch: dict(p [J, 8], valid uint8 [J], K int64 [J], span, M)."""
+        J = self.max_jobs
+        st = dict(p=np.empty((J, 8)), valid=np.empty(J, np.uint8), K=np.empty(J, np.int64), span=np.empty(J),
+                  M=np.empty(J))
+        self._check(self._lib.slaq_get_fit_state(self._h, _ptr(st["p"]), _ptr(st["valid"]), _ptr(st["K"]),
+                                                 _ptr(st["span"]), _ptr(st["M"])))
+        return st
+
+    def set_fit_state(self, state):
+        """Make `state` (as returned by get_fit_state) the starting point of every job's next fit."""
+        J = self.max_jobs
+        p, valid = _arr(state["p"], np.float64), _arr(state["valid"], np.uint8)
+        K, span, M = _arr(state["K"], np.int64), _arr(state["span"], np.float64), _arr(state["M"], np.float64)
+        assert p.shape == (J, 8) and valid.shape == (J,) and K.shape == (J,) and span.shape == (J,) and M.shape == (J,)
+        return self._check(self._lib.slaq_set_fit_state(self._h, _ptr(p), _ptr(valid), _ptr(K), _ptr(span), _ptr(M)))
 
     def set_gains(self, gain):
         g = _arr(gain, np.float64)

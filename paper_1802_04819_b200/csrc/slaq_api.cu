@@ -52,6 +52,14 @@ size_t layout(slaq_handle* h, char* base, int32_t J, int32_t Hmax, int32_t cap) 
     fit.sweeps = b.take<int32_t>(2 * Js);
     fit.largest = b.take<double>(Js);
     fit.span = b.take<double>(Js);
+    fit.both = b.take<double>(8 * Js);
+    fit.mask = b.take<uint8_t>(Js);
+    fit.k_fit = b.take<int64_t>(Js);
+    fit.warm_p = b.take<double>(8 * Js);
+    fit.warm_mask = b.take<uint8_t>(Js);
+    fit.warm_k = b.take<int64_t>(Js);
+    fit.warm_span = b.take<double>(Js);
+    fit.warm_scale = b.take<double>(Js);
     Scratch sc;
     sc.hist = b.take<unsigned long long>((size_t)kRadixPasses * kRadixBins);
     const size_t zero_from = b.off - sizeof(unsigned long long) * (size_t)kRadixPasses * kRadixBins;
@@ -135,14 +143,16 @@ __global__ void init_jobs_kernel(JobArrays job, FitArrays fit, double* ring, int
     fit.sweeps[2 * (size_t)j] = fit.sweeps[2 * (size_t)j + 1] = 0;
     fit.largest[j] = CUDART_NAN;
     fit.span[j] = 1.0;
+    fit.mask[j] = 0;
+    fit.warm_mask[j] = 0;
     alloc[j] = 0;
     reduction[j] = 0.0;
 }
 
 // One new iteration per listed job: ring write, iteration index, largest reduction seen,
 // and the sums of the iteration-time law (booked at the given or the current core count).
-__global__ void append_kernel(JobArrays job, int max_jobs, int n, const int32_t* ids, const double* losses,
-                              const double* times, const int32_t* cores) {
+__global__ void append_kernel(JobArrays job, FitArrays fit, int max_jobs, int n, const int32_t* ids,
+                              const double* losses, const double* times, const int32_t* cores) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const int j = ids[i];
@@ -162,6 +172,15 @@ __global__ void append_kernel(JobArrays job, int max_jobs, int n, const int32_t*
     job.head[j] = head;
     job.count[j] = count < cap ? count + 1 : cap;
     job.k_last[j] += 1;
+    // the history changes: what the last epoch fitted becomes the next fit's starting point
+    const uint8_t fitted = fit.mask[j];
+    fit.warm_mask[j] = fitted;
+    if (fitted) {
+        for (int k = 0; k < 8; ++k) fit.warm_p[8 * (size_t)j + k] = fit.both[8 * (size_t)j + k];
+        fit.warm_k[j] = fit.k_fit[j];
+        fit.warm_span[j] = fit.span[j];
+        fit.warm_scale[j] = fit.largest[j];
+    }
     if (times) {
         int nc = cores ? cores[i] : job.last_alloc[j];
         if (nc < 1) nc = 1;
@@ -180,7 +199,8 @@ __global__ void append_kernel(JobArrays job, int max_jobs, int n, const int32_t*
 }
 
 // Bulk load: one warp per listed job copies (ring mode) or adopts (packed mode) its row.
-__global__ void load_kernel(JobArrays job, double* ring, int max_jobs, int max_hist, int n, const int32_t* ids,
+__global__ void load_kernel(JobArrays job, FitArrays fit, double* ring, int max_jobs, int max_hist, int n,
+                            const int32_t* ids,
                             const int64_t* offsets, const double* src, const int64_t* k_last, const double* m_seen,
                             int packed) {
     const int slot = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
@@ -206,6 +226,8 @@ __global__ void load_kernel(JobArrays job, double* ring, int max_jobs, int max_h
         job.count[j] = (int)H;
         job.k_last[j] = H > 0 ? k_last[slot] : -1;
         job.m_seen[j] = m_seen ? m_seen[slot] : -CUDART_INF;
+        fit.mask[j] = 0;        // a replaced history has no earlier fit to start from
+        fit.warm_mask[j] = 0;
     }
 }
 
@@ -328,9 +350,9 @@ int do_append(slaq_handle* h, int32_t n, const int32_t* ids, const double* losse
     if (times && cores)
         CK(cudaMemcpyAsync(h->stage.cores, cores, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy cores");
     const int threads = 256;
-    append_kernel<<<(n + threads - 1) / threads, threads, 0, st>>>(h->job, h->max_jobs, n, h->stage.ids, h->stage.losses,
-                                                                  times ? h->stage.times : nullptr,
-                                                                  (times && cores) ? h->stage.cores : nullptr);
+    append_kernel<<<(n + threads - 1) / threads, threads, 0, st>>>(
+        h->job, h->fit, h->max_jobs, n, h->stage.ids, h->stage.losses, times ? h->stage.times : nullptr,
+        (times && cores) ? h->stage.cores : nullptr);
     CK(cudaGetLastError(), "append kernel");
     CK(cudaStreamSynchronize(st), "append");   // the caller may reuse its buffers
     if (h->n_active < h->max_jobs) {   // nothing to do once every id is active
@@ -417,9 +439,9 @@ int do_load(slaq_handle* h, int32_t n, const int32_t* ids, const int64_t* offset
             e = cudaMemcpyAsync(h->stage.m_seen, m_seen, sizeof(double) * n, cudaMemcpyHostToDevice, st);
         if (e == cudaSuccess) {
             const int threads = 256, warps = threads / 32;
-            load_kernel<<<(n + warps - 1) / warps, threads, 0, st>>>(h->job, h->ring_pool, h->max_jobs, h->max_hist, n,
-                                                                    h->stage.ids, h->stage.offsets, d_src, h->stage.k_last,
-                                                                    m_seen ? h->stage.m_seen : nullptr, packed ? 1 : 0);
+            load_kernel<<<(n + warps - 1) / warps, threads, 0, st>>>(
+                h->job, h->fit, h->ring_pool, h->max_jobs, h->max_hist, n, h->stage.ids, h->stage.offsets, d_src,
+                h->stage.k_last, m_seen ? h->stage.m_seen : nullptr, packed ? 1 : 0);
             e = cudaGetLastError();
         }
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // `rel` and the caller's buffers are free again
@@ -554,6 +576,10 @@ int slaq_set_param(slaq_t* h, int key, double value) {
             if (!(value >= 8192 && value <= 200 * 1024)) return fail(h, SLAQ_E_ARG, "fit slice must lie in 8 KB..200 KB");
             h->fit_slice_bytes = (size_t)value;
             return SLAQ_OK;
+        case SLAQ_P_WARM_START:
+            if (!(value == 0.0 || value == 1.0)) return fail(h, SLAQ_E_ARG, "warm start must be 0 or 1");
+            h->warm_start = value != 0.0;
+            return SLAQ_OK;
         default:
             return fail(h, SLAQ_E_ARG, "unknown parameter key");
     }
@@ -567,6 +593,7 @@ int slaq_get_param(const slaq_t* h, int key, double* out_value) {
         case SLAQ_P_MAX_CORES_PER_JOB: *out_value = h->max_cores; return SLAQ_OK;
         case SLAQ_P_MIN_FIT_POINTS: *out_value = h->min_fit_points; return SLAQ_OK;
         case SLAQ_P_FIT_SLICE_BYTES: *out_value = (double)h->fit_slice_bytes; return SLAQ_OK;
+        case SLAQ_P_WARM_START: *out_value = h->warm_start ? 1.0 : 0.0; return SLAQ_OK;
         default: return SLAQ_E_ARG;
     }
 }
@@ -833,6 +860,49 @@ int slaq_get_time_model(slaq_t* h, double* out_s, double* out_w) {
     CK(cudaMemcpyAsync(out_s, h->stage.losses, sizeof(double) * J, cudaMemcpyDeviceToHost, h->stream), "copy s");
     CK(cudaMemcpyAsync(out_w, h->stage.times, sizeof(double) * J, cudaMemcpyDeviceToHost, h->stream), "copy w");
     CK(cudaStreamSynchronize(h->stream), "copy time law");
+    return SLAQ_OK;
+}
+
+int slaq_get_fit_state(slaq_t* h, double* out_params, uint8_t* out_mask, int64_t* out_k, double* out_span,
+                       double* out_scale) {
+    if (!h || !out_params || !out_mask || !out_k || !out_span || !out_scale) return SLAQ_E_ARG;
+    if (const int rc = check_device(h)) return rc;
+    const size_t J = (size_t)h->max_jobs;
+    int rc;
+    if ((rc = fetch(h, out_params, h->fit.both, 8 * J, "copy fitted parameters"))) return rc;
+    if ((rc = fetch(h, out_mask, h->fit.mask, J, "copy fit masks"))) return rc;
+    if ((rc = fetch(h, out_k, h->fit.k_fit, J, "copy fit iteration indices"))) return rc;
+    if ((rc = fetch(h, out_span, h->fit.span, J, "copy fit spans"))) return rc;
+    if ((rc = fetch(h, out_scale, h->fit.largest, J, "copy fit scales"))) return rc;
+    CK(cudaStreamSynchronize(h->stream), "copy fit state");
+    return SLAQ_OK;
+}
+
+int slaq_set_fit_state(slaq_t* h, const double* params, const uint8_t* mask, const int64_t* k, const double* span,
+                       const double* scale) {
+    if (!h || !params || !mask || !k || !span || !scale) return SLAQ_E_ARG;
+    if (const int rc = check_device(h)) return rc;
+    const size_t J = (size_t)h->max_jobs;
+    for (size_t j = 0; j < J; ++j) {
+        if (!mask[j]) continue;
+        if (mask[j] > 3) return fail(h, SLAQ_E_ARG, "fit mask above 3");
+        if (!h->active[j]) return fail(h, SLAQ_E_ARG, "fit state for a job without losses");
+        if (!(span[j] > 0.0 && std::isfinite(span[j]) && scale[j] > 0.0 && std::isfinite(scale[j])))
+            return fail(h, SLAQ_E_ARG, "fit state needs a positive finite span and scale");
+    }
+    cudaStream_t st = h->stream;
+    const cudaMemcpyKind up = cudaMemcpyHostToDevice;
+    CK(cudaMemcpyAsync(h->fit.both, params, sizeof(double) * 8 * J, up, st), "copy fitted parameters");
+    CK(cudaMemcpyAsync(h->fit.warm_p, params, sizeof(double) * 8 * J, up, st), "copy fitted parameters");
+    CK(cudaMemcpyAsync(h->fit.mask, mask, sizeof(uint8_t) * J, up, st), "copy fit masks");
+    CK(cudaMemcpyAsync(h->fit.warm_mask, mask, sizeof(uint8_t) * J, up, st), "copy fit masks");
+    CK(cudaMemcpyAsync(h->fit.k_fit, k, sizeof(int64_t) * J, up, st), "copy fit iteration indices");
+    CK(cudaMemcpyAsync(h->fit.warm_k, k, sizeof(int64_t) * J, up, st), "copy fit iteration indices");
+    CK(cudaMemcpyAsync(h->fit.span, span, sizeof(double) * J, up, st), "copy fit spans");
+    CK(cudaMemcpyAsync(h->fit.warm_span, span, sizeof(double) * J, up, st), "copy fit spans");
+    CK(cudaMemcpyAsync(h->fit.largest, scale, sizeof(double) * J, up, st), "copy fit scales");
+    CK(cudaMemcpyAsync(h->fit.warm_scale, scale, sizeof(double) * J, up, st), "copy fit scales");
+    CK(cudaStreamSynchronize(st), "copy fit state");
     return SLAQ_OK;
 }
 

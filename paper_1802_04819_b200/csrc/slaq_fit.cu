@@ -499,32 +499,41 @@ struct Moments {
 // First guesses.  d0 lies below every level; with the offset fixed at d0, 1/(y - d0) is a
 // quadratic in x (family I: weighted linear least squares, or the line through the oldest and
 // newest transformed points if that fit is not a decreasing curve with a positive denominator)
-// and log(y - d0) is a line in x (family II: weighted linear regression).
+// and log(y - d0) is a line in x (family II: weighted linear regression).  needI / needII: the
+// job wants that family's guess (a family that starts from last epoch's parameters does not);
+// the weight sums in `mom` are always produced.
 __device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span, double ymin, double ymax, bool busy,
-                              Moments& mom, double (&pI)[4], double (&pII)[4]) {
+                              bool needI, bool needII, Moments& mom, double (&pI)[4], double (&pII)[4]) {
     const double d0 = ymax > ymin ? ymin - 0.1 * (ymax - ymin) : ymin - 1e-3 * fmax(fabs(ymin), 1.0);
     double sw = 0, swx = 0, swx2 = 0, swx3 = 0, swx4 = 0, swy2 = 0, r0 = 0, r1 = 0, r2 = 0, su = 0, sxu = 0;
     double md = (double)S.l;
+    const bool any_guess = needI || needII;
     for (int k = 0; k < k_all; ++k, md += (double)S.L) {
         const int m = S.l + S.L * k;
         if (busy && m < H) {
             const double x = -md * inv_span;
             const double w = S.wtab[m];
             const double y = S.y[k * 32 + S.lane];
-            const double wx = w * x, wx2 = wx * x;
             sw += w;
-            swx += wx;
-            swx2 += wx2;
-            swx3 = fma(wx2, x, swx3);
-            swx4 = fma(wx2 * x, x, swx4);
             swy2 = fma(w * y, y, swy2);
-            const double wz = w * fast_rcp(y - d0);
-            r2 += wz;
-            r1 = fma(wz, x, r1);
-            r0 = fma(wz * x, x, r0);
-            const double wu = w * log(y - d0);
-            su += wu;
-            sxu = fma(wu, x, sxu);
+            if (any_guess) {
+                const double wx = w * x, wx2 = wx * x;
+                swx += wx;
+                swx2 += wx2;
+                swx3 = fma(wx2, x, swx3);
+                swx4 = fma(wx2 * x, x, swx4);
+            }
+            if (needI) {
+                const double wz = w * fast_rcp(y - d0);
+                r2 += wz;
+                r1 = fma(wz, x, r1);
+                r0 = fma(wz * x, x, r0);
+            }
+            if (needII) {
+                const double wu = w * log(y - d0);
+                su += wu;
+                sxu = fma(wu, x, sxu);
+            }
         }
     }
     for (int o = S.L >> 1; o > 0; o >>= 1) {
@@ -538,36 +547,38 @@ __device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span,
     mom.sw = sw;
     mom.swy2 = swy2;
     // family I
-    Sym4 B;
-    B.a00 = swx4; B.a01 = swx3; B.a02 = swx2; B.a11 = swx2; B.a12 = swx; B.a22 = sw;
-    B.a03 = B.a13 = B.a23 = 0.0; B.a33 = 1.0;
-    const double rhs[4] = {r0, r1, r2, 0.0};
-    double sol[4] = {0.0, 0.0, 0.0, 0.0};
-    bool good = busy && ldl_solve(B, rhs, sol) && sol[0] >= 0.0 && sol[1] >= 0.0;
-    int pos = 1;
-    md = (double)S.l;
-    for (int k = 0; k < k_all; ++k, md += (double)S.L) {
-        const int m = S.l + S.L * k;
-        if (busy && m < H) {
-            const double x = -md * inv_span;
-            pos &= fma(fma(sol[0], x, sol[1]), x, sol[2]) > 0.0 ? 1 : 0;
+    if (__any_sync(kFull, needI)) {
+        Sym4 B;
+        B.a00 = swx4; B.a01 = swx3; B.a02 = swx2; B.a11 = swx2; B.a12 = swx; B.a22 = sw;
+        B.a03 = B.a13 = B.a23 = 0.0; B.a33 = 1.0;
+        const double rhs[4] = {r0, r1, r2, 0.0};
+        double sol[4] = {0.0, 0.0, 0.0, 0.0};
+        bool good = needI && ldl_solve(B, rhs, sol) && sol[0] >= 0.0 && sol[1] >= 0.0;
+        int pos = 1;
+        md = (double)S.l;
+        for (int k = 0; k < k_all; ++k, md += (double)S.L) {
+            const int m = S.l + S.L * k;
+            if (needI && m < H) {
+                const double x = -md * inv_span;
+                pos &= fma(fma(sol[0], x, sol[1]), x, sol[2]) > 0.0 ? 1 : 0;
+            }
         }
+        pos = group_and(pos, S.L);
+        good = good && pos;
+        // the oldest point (m = H - 1) and the newest (m = 0), read from the lanes that own them
+        const int m_old = max(H - 1, 0);
+        const double y_old = S.y[(m_old / S.L) * 32 + (S.lane - S.l) + (m_old & (S.L - 1))];
+        const double y_new = S.y[S.lane - S.l];
+        if (good) {
+            pI[0] = sol[0]; pI[1] = sol[1]; pI[2] = sol[2];
+        } else {
+            const double z_old = 1.0 / (y_old - d0), z_new = 1.0 / (y_new - d0);
+            pI[0] = 0.0;
+            pI[1] = fmax(z_new - z_old, 0.0);
+            pI[2] = z_new;
+        }
+        pI[3] = d0;
     }
-    pos = group_and(pos, S.L);
-    good = good && pos;
-    // the oldest point (m = H - 1) and the newest (m = 0), read from the lanes that own them
-    const int m_old = max(H - 1, 0);
-    const double y_old = S.y[(m_old / S.L) * 32 + (S.lane - S.l) + (m_old & (S.L - 1))];
-    const double y_new = S.y[S.lane - S.l];
-    if (good) {
-        pI[0] = sol[0]; pI[1] = sol[1]; pI[2] = sol[2];
-    } else {
-        const double z_old = 1.0 / (y_old - d0), z_new = 1.0 / (y_new - d0);
-        pI[0] = 0.0;
-        pI[1] = fmax(z_new - z_old, 0.0);
-        pI[2] = z_new;
-    }
-    pI[3] = d0;
     // family II
     const double den = sw * swx2 - swx * swx;
     const double slope = (sw * sxu - swx * su) / den;
@@ -575,6 +586,59 @@ __device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span,
     pII[1] = fmax(-slope, 1e-8);
     pII[2] = d0;
     pII[3] = 0.0;
+}
+
+// Last epoch's end points of both families in this epoch's window coordinates.  The curves
+// are functions of the iteration index and the raw loss; with x0 = (k - K0)/span0, y0 = l/M0
+// then and x = (k - K)/span, y = l/M now, x0 = t + r x and y = sigma y0, where
+// t = (K - K0)/span0, r = span/span0, sigma = M0/M, and both families keep their form under
+// that substitution.  Clears `wmask` if the stored coordinates cannot be used.
+__device__ void carry_over(const FitArrays& fit, const JobArrays& job, int j, double span, double M, unsigned& wmask,
+                           double (&pI)[4], double (&pII)[4]) {
+    const double span0 = fit.warm_span[j], M0 = fit.warm_scale[j];
+    if (!(span0 > 0.0) || !(M0 > 0.0) || !finite_d(M0)) {
+        wmask = 0;
+        return;
+    }
+    const double* q = fit.warm_p + 8 * (size_t)j;
+    const double t = (double)(job.k_last[j] - fit.warm_k[j]) / span0;
+    const double r = span / span0, sigma = M0 / M;
+    if (wmask & 1u) {
+        const double a = q[0], b = q[1], c = q[2], d = q[3];
+        pI[0] = a * r * r / sigma;
+        pI[1] = (2.0 * a * t + b) * r / sigma;
+        pI[2] = ((a * t + b) * t + c) / sigma;
+        pI[3] = sigma * d;
+    }
+    if (wmask & 2u) {
+        pII[0] = q[4] - q[5] * t + log(sigma);
+        pII[1] = q[5] * r;
+        pII[2] = sigma * q[6];
+        pII[3] = 0.0;
+    }
+}
+
+// The second round of a warm start: the families whose carried-over point had no finite
+// residual (`redo`, per lane for its own family) take their first guesses and are swept again.
+__device__ __noinline__ void restart_from_first_guesses(const Lanes& S, int fam, int H, int k_all, double inv_span,
+                                                        double ymin, double ymax, bool fits, bool redo, double* pI,
+                                                        double* pII, SweepSums* sums) {
+    const int lane = S.lane;
+    const bool redoI = __shfl_sync(kFull, (int)redo, lane & ~1) != 0;
+    const bool redoII = __shfl_sync(kFull, (int)redo, lane | 1) != 0;
+    Moments mom;
+    double gI[4], gII[4], qI[4], qII[4];
+    first_guesses(S, H, k_all, inv_span, ymin, ymax, fits, redoI, redoII, mom, gI, gII);
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        qI[a] = redoI ? gI[a] : pI[a];
+        qII[a] = redoII ? gII[a] : pII[a];
+        pI[a] = qI[a];
+        pII[a] = qII[a];
+    }
+    SweepSums again;
+    sweep(S, fam, H, k_all, inv_span, qI, redoI, qII, redoII, again);
+    if (redo) *sums = again;
 }
 
 // Window-length classes, longest first: class c holds the jobs with h_lo[c] < H <= h_hi[c] and
@@ -587,10 +651,13 @@ struct FitClasses {
     int h_max;       // longest window
 };
 
+// kWarm: families may start from last epoch's parameters (a separate instantiation, so that the
+// plain one carries none of that code).
+template <bool kWarm>
 __global__ void __launch_bounds__(kMaxWarpsPerBlock * 32, 4)
 fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, const int32_t* __restrict__ order,
-           const int32_t* __restrict__ start, FitClasses cls, int lm_trials, int min_fit_points, unsigned int* queue,
-           long long* counters, int32_t* err_word) {
+           const int32_t* __restrict__ start, FitClasses cls, int lm_trials, int min_fit_points,
+           unsigned int* queue, long long* counters, int32_t* err_word) {
     extern __shared__ double smem[];
     __shared__ int slot_base[kMaxFitClasses + 1];
     double* wtab = smem;                                   // [h_max]
@@ -643,6 +710,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         double p_out[4] = {CUDART_NAN, CUDART_NAN, CUDART_NAN, CUDART_NAN};
         double S_out[2] = {CUDART_INF, CUDART_INF};
         int sweeps_out[2] = {0, 0};
+        int ended = 0;   // bit 0 / 1: family I / II ended with a finite residual
         const double span = (double)max(H - 1, 1);
         const bool fits = status == SLAQ_JOB_FITTED && H >= min_fit_points;   // this lane's job gets curves fitted
 
@@ -651,9 +719,41 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
             Moments mom;
             Family F;
             double pI[4], pII[4];      // the points the next sweep evaluates
-            first_guesses(S, H, k_all, inv_span, nz.ymin, nz.ymax, fits, mom, pI, pII);
+            // Starting points: the first guesses, or (kWarm) last epoch's parameters where the job
+            // has some; a carried-over point without a finite residual is dropped for the
+            // family's first guess in a second round.
+            int spent = 0;
             SweepSums sums;
-            sweep(S, fam, H, k_all, inv_span, pI, fits, pII, fits, sums);
+            if (!kWarm) {
+                first_guesses(S, H, k_all, inv_span, nz.ymin, nz.ymax, fits, fits, fits, mom, pI, pII);
+                sweep(S, fam, H, k_all, inv_span, pI, fits, pII, fits, sums);
+            } else {
+                unsigned wmask = fits ? fit.warm_mask[j] : 0u;
+                if (wmask) carry_over(fit, job, j, span, nz.M, wmask, pI, pII);
+                {
+                    double gI[4], gII[4];
+                    const bool needI = fits && !(wmask & 1u), needII = fits && !(wmask & 2u);
+                    first_guesses(S, H, k_all, inv_span, nz.ymin, nz.ymax, fits, needI, needII, mom, gI, gII);
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+                        if (needI) pI[a] = gI[a];
+                        if (needII) pII[a] = gII[a];
+                    }
+                }
+                sweep(S, fam, H, k_all, inv_span, pI, fits, pII, fits, sums);
+                const bool redo = fits && ((wmask >> fam) & 1u) && !sums.usable;
+                if (__any_sync(kFull, redo)) {   // rare: kept out of line, with its own copies of what it changes
+                    double tI[4], tII[4];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) tI[a] = pI[a], tII[a] = pII[a];
+                    SweepSums again = sums;
+                    restart_from_first_guesses(S, fam, H, k_all, inv_span, nz.ymin, nz.ymax, fits, redo, tI, tII, &again);
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) pI[a] = tI[a], pII[a] = tII[a];
+                    sums = again;
+                    spent = redo ? 1 : 0;
+                }
+            }
 #pragma unroll
             for (int a = 0; a < 4; ++a) F.p[a] = fam ? pII[a] : pI[a];
             F.ok = fits && sums.usable;
@@ -661,7 +761,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
             F.lambda = kLambda0;
             F.nu = 2.0;
             F.was_frozen = 0;
-            F.sweeps = fits ? 1 : 0;
+            F.sweeps = fits ? 1 + spent : 0;
             F.done = !F.ok;
             F.has_trial = false;
             F.predicted = 0.0;
@@ -699,6 +799,15 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
                 if (ok_I) S_out[0] = S_I;
                 if (ok_II) S_out[1] = S_II;
                 const bool okI = ok_I && finite_d(S_I), okII = ok_II && finite_d(S_II);
+                ended = (okI ? 1 : 0) | (okII ? 2 : 0);
+                if (S.l == 0 && ended) {   // what the next epoch may start from
+                    fit.k_fit[j] = job.k_last[j];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+                        fit.both[8 * (size_t)j + a] = pI[a];
+                        fit.both[8 * (size_t)j + 4 + a] = pII[a];
+                    }
+                }
                 if (okI && (!okII || S_I <= S_II)) {   // a tie goes to family I
                     family = 0;
 #pragma unroll
@@ -739,6 +848,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
                 n_fallback += 1;
             }
             fit.status[j] = status;
+            fit.mask[j] = (uint8_t)ended;
             fit.family[j] = (int8_t)family;
 #pragma unroll
             for (int a = 0; a < 4; ++a) fit.params[4 * (size_t)j + a] = p_out[a];
@@ -980,22 +1090,23 @@ int launch_fit(slaq_handle* h) {
         h->err = "fit kernel: a window does not fit in shared memory";
         return -1;
     }
-    cudaError_t e = cudaFuncSetAttribute(fit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const auto kernel = h->warm_start ? fit_kernel<true> : fit_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) {
         h->err = std::string("fit kernel shared memory: ") + cudaGetErrorString(e);
         return -1;
     }
-    cudaFuncSetAttribute(fit_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     int per_sm = 1;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fit_kernel, warps * 32, smem);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, warps * 32, smem);
     if (per_sm < 1) per_sm = 1;
     int blocks = h->sm_count * per_sm;
     const int needed = (J + warps - 1) / warps;   // at least one job per slot
     if (blocks > needed) blocks = needed;
     if (blocks < 1) blocks = 1;
-    fit_kernel<<<blocks, warps * 32, smem, st>>>(h->job, h->fit, h->wtab, h->scratch.order, h->scratch.start, cls,
-                                                h->lm_trials, h->min_fit_points, h->scratch.ticket + kFitQueueBase,
-                                                h->scratch.counters, h->err_word);
+    kernel<<<blocks, warps * 32, smem, st>>>(h->job, h->fit, h->wtab, h->scratch.order, h->scratch.start, cls,
+                                            h->lm_trials, h->min_fit_points, h->scratch.ticket + kFitQueueBase,
+                                            h->scratch.counters, h->err_word);
     ++launches;
     e = cudaGetLastError();
     if (e != cudaSuccess) {

@@ -43,6 +43,18 @@ struct FitArrays {
     int32_t* sweeps;     // [max_jobs][2]
     double* largest;     // M
     double* span;        // max(H-1, 1)
+    // Both families' end points of the last epoch, in that epoch's window coordinates
+    // (span, largest and k_fit say which), and the copy the next fit may start from.  A
+    // job's copy is refreshed when its history changes, so an epoch repeated without new
+    // losses starts from the same point and gives the same result.
+    double* both;        // [max_jobs][8]: family I (a, b, c, d), family II (alpha, beta, c, unused)
+    uint8_t* mask;       // bit 0 / 1: family I / II ended with a finite residual
+    int64_t* k_fit;      // index of the newest iteration at that fit
+    double* warm_p;      // [max_jobs][8]
+    uint8_t* warm_mask;
+    int64_t* warm_k;
+    double* warm_span;
+    double* warm_scale;
 };
 
 // Running state of the radix select.
@@ -87,6 +99,7 @@ struct slaq_handle {
     double gamma = 0.9;
     int32_t lm_trials = 20, min_fit_points = 4;
     size_t fit_slice_bytes = 16 * 1024;   // shared memory one warp of the fit kernel may use
+    bool warm_start = false;              // fits start from the last epoch's parameters where there are some
     cudaStream_t stream = nullptr;
     bool owns_ws = false;
     void* ws = nullptr;

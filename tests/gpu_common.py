@@ -21,8 +21,15 @@ def oracle_epoch(oracle, wl, total_cores=None, threads=0):
                            threads=threads)
 
 
-def compare_epoch(gpu_alloc, pred, ref, total_cores, cap, allow_unstable=0):
-    """Element-by-element comparison of one epoch.  Returns a dict of counts for reporting."""
+def compare_epoch(gpu_alloc, pred, ref, total_cores, cap, allow_unstable=0, loose=(1e-4, 1e-7), total_rtol=1e-9):
+    """Element-by-element comparison of one epoch.  Returns a dict of counts for reporting.
+
+    allow_unstable: how many jobs may miss the tolerance on R(n); those must still meet the
+    `loose` (relative, absolute) one.  Zero everywhere except where the fits of both sides run
+    freely over several epochs from their own earlier results, so that rounding differences
+    compound in the few jobs whose residual is flat along a direction.
+    total_rtol: tolerance on the sum of the predicted reductions at the allocation (the per-job
+    tolerance is R_RTOL; the sum of the cold path's fits agrees a thousand times better)."""
     status_g, status_c = pred["status"], ref["status"]
     np.testing.assert_array_equal(status_g, status_c)
     fitted = status_c == 0
@@ -43,6 +50,8 @@ def compare_epoch(gpu_alloc, pred, ref, total_cores, cap, allow_unstable=0):
     assert bad_jobs.size <= allow_unstable, (
         f"{bad_jobs.size} jobs exceed the tolerance on R(n): first {bad_jobs[:5]}, "
         f"worst {np.abs(Rg - Rc)[bad_jobs].max() if bad_jobs.size else 0}")
+    if bad_jobs.size:
+        np.testing.assert_allclose(Rg[bad_jobs], Rc[bad_jobs], rtol=loose[0], atol=loose[1])
     # allocation: equal except where the deciding gains lie within the band around the threshold
     ca = ref["alloc"]
     assert gpu_alloc.sum() == ca.sum()
@@ -61,8 +70,11 @@ def compare_epoch(gpu_alloc, pred, ref, total_cores, cap, allow_unstable=0):
                 f"job {j}: alloc {gpu_alloc[j]} vs {ca[j]} but gains {contested} are not near threshold {tau}")
     # predicted reduction at the allocation, and its total
     same = gpu_alloc == ca
+    same[bad_jobs] = False
+    same[fam_diff] = False
     np.testing.assert_allclose(pred["R"][same], ref["R"][same], rtol=R_RTOL, atol=R_ATOL)
     tot_c = ref["R"].sum()
-    assert abs(pred["R"].sum() - tot_c) <= 1e-9 * abs(tot_c) + 1e-9 * max(1, diff.size)
+    slack = np.abs(pred["R"] - ref["R"])[np.union1d(bad_jobs, fam_diff).astype(np.int64)].sum()
+    assert abs(pred["R"].sum() - tot_c) <= total_rtol * abs(tot_c) + 1e-9 * max(1, diff.size) + slack
     return dict(jobs=int(status_c.size), fitted=int(fitted.sum()), family_ties=int(fam_diff.size),
                 unstable=int(bad_jobs.size), alloc_diff=int(diff.size))
