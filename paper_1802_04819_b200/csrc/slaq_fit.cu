@@ -84,6 +84,12 @@ __device__ __forceinline__ double older_neighbour(const Lanes& S, int k) {
     return S.l + 1 < S.L ? S.y[k * 32 + S.lane + 1] : S.y[(k + 1) * 32 + S.lane - (S.L - 1)];
 }
 
+// One asynchronous copy of a double from global to shared memory (both 8-byte aligned).
+__device__ __forceinline__ void copy_async_8(double* dst_shared, const double* src) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(dst_shared);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(d), "l"(src) : "memory");
+}
+
 // Copy the job's window into the lane columns (ring storage: the newest loss sits just before
 // `head`).  Returns H, or 0 after flagging storage that cannot be right.
 __device__ int stage_window(const JobArrays& job, int j, int h_cap, const Lanes& S, int32_t* err_word) {
@@ -98,26 +104,15 @@ __device__ int stage_window(const JobArrays& job, int j, int h_cap, const Lanes&
     }
     int newest = job.head[j] - 1;
     if (newest < 0) newest += cap;
-    // four loads in flight per lane; the values are read once, so they bypass the caches' keep lists
+    // asynchronous 8-byte copies straight into the lane's column: all of a lane's points are in
+    // flight at once, and nothing passes through registers
     double* dst = S.y + S.lane;
-    int m = S.l;
-    for (; m + 3 * S.L < H; m += 4 * S.L, dst += 4 * 32) {
-        int p0 = newest - m, p1 = p0 - S.L, p2 = p1 - S.L, p3 = p2 - S.L;
-        p0 += p0 < 0 ? cap : 0;
-        p1 += p1 < 0 ? cap : 0;
-        p2 += p2 < 0 ? cap : 0;
-        p3 += p3 < 0 ? cap : 0;
-        const double v0 = __ldcs(row + p0), v1 = __ldcs(row + p1), v2 = __ldcs(row + p2), v3 = __ldcs(row + p3);
-        dst[0] = v0;
-        dst[32] = v1;
-        dst[64] = v2;
-        dst[96] = v3;
-    }
-    for (; m < H; m += S.L, dst += 32) {
+    for (int m = S.l; m < H; m += S.L, dst += 32) {
         int pos = newest - m;
         pos += pos < 0 ? cap : 0;
-        *dst = __ldcs(row + pos);
+        copy_async_8(dst, row + pos);
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");
     return H;
 }
 
