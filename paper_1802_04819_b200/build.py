@@ -20,6 +20,16 @@ def nvcc_command(verbose_ptxas: bool = False) -> list[str]:
     return cmd + [str(CSRC / s) for s in SOURCES]
 
 
+PROBE = PKG / "fp64_issue_probe"
+
+
+def build_probe() -> Path:
+    """Compile the stand-alone fp64 issue-rate probe (csrc/fp64_issue_probe.cu) next to the library."""
+    subprocess.run(["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+                    "-o", str(PROBE), str(CSRC / "fp64_issue_probe.cu")], check=True)
+    return PROBE
+
+
 def is_stale() -> bool:
     if not LIB.exists():
         return True
@@ -36,3 +46,4 @@ def build(force: bool = False, verbose_ptxas: bool = False) -> Path:
 
 if __name__ == "__main__":
     build(force=True, verbose_ptxas=True)
+    build_probe()

@@ -351,7 +351,7 @@ __device__ __forceinline__ bool finish_trial(Family& F, const double (&trial)[4]
 #pragma unroll
         for (int a = 0; a < 4; ++a) F.p[a] = trial[a];
         F.S = S_trial;
-        const double rho = F.predicted > 0.0 ? (S_before - S_trial) / F.predicted : 0.0;
+        const double rho = F.predicted > 0.0 ? (S_before - S_trial) * fast_rcp(F.predicted) : 0.0;
         const double c = 2.0 * rho - 1.0;
         F.lambda *= fmax(1.0 / 3.0, 1.0 - c * c * c);
         F.nu = 2.0;
