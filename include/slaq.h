@@ -62,8 +62,9 @@ enum {
     SLAQ_P_LM_TRIALS = 2,         /* Levenberg-Marquardt trials per family; default 20; 0 .. 1000 */
     SLAQ_P_MAX_CORES_PER_JOB = 3, /* cap on a_j; default 64; 1 .. what the handle was created for */
     SLAQ_P_MIN_FIT_POINTS = 4,    /* fewer stored points than this use linear extrapolation; default 4; >= 4 */
-    SLAQ_P_FIT_SLICE_BYTES = 5,   /* tuning: shared memory one warp of the fit kernel may use (8 KB..200 KB);
-                                     decides how many lanes share a job; results stay within rounding */
+    SLAQ_P_FIT_SLICE_BYTES = 5,   /* tuning: shared memory one warp of the fit kernel may use (8 KB..200 KB,
+                                     default 13,824: sixteen warps per SM); decides how many lanes share a
+                                     job; results stay within rounding */
     SLAQ_P_WARM_START = 6         /* 0 (default) or 1.  The scheduler refits every job at short intervals
                                      (Evaluation, "Scalability and efficiency"); with 1, a family starts from the
                                      parameters the job's last epoch ended with, carried into this epoch's window

@@ -8,9 +8,10 @@
 // (newest point x = 0, oldest x = -1); the family with the lower weighted residual wins.
 //
 // Work split.  Jobs are sorted by window length (counting sort, longest first) and cut into
-// length classes.  In class c a group of L lanes (L = 2, 4, .. 32, chosen so that a warp's
-// windows fit its shared-memory slice) owns one job, so a warp carries 32/L jobs.  One
-// persistent launch serves all classes from one work queue, longest windows first.  A lane
+// length classes.  In class c a group of L lanes (L = 2, 4, .. 32: the fewest lanes at which
+// the window fits the rows of a warp's shared-memory slice) owns one job, so a warp carries
+// 32/L jobs.  One persistent launch (one block of 16 warps per SM) serves all classes from
+// one work queue, longest windows first.  A lane
 // walks its job's points m = l, l + L, l + 2L, ... counted from the newest one; both families
 // are evaluated in the same sweep over the window; the partial sums of the normal equations
 // are reduced over the L lanes with shuffles; the even lanes of a group then run family I's
@@ -26,7 +27,7 @@ namespace slaq {
 
 namespace {
 
-constexpr int kMaxWarpsPerBlock = 4;
+constexpr int kMaxWarpsPerBlock = 16;          // one block per SM: its warps share one copy of the weight table
 constexpr size_t kSmemLimit = 226 * 1024;   // shared memory one block may use on sm_100, less the static part
 constexpr unsigned kFull = 0xffffffffu;
 constexpr double kLambda0 = 1e-3, kLambdaMin = 1e-5, kLambdaMax = 1e12;
@@ -649,7 +650,7 @@ struct FitClasses {
 // kWarm: families may start from last epoch's parameters (a separate instantiation, so that the
 // plain one carries none of that code).
 template <bool kWarm>
-__global__ void __launch_bounds__(kMaxWarpsPerBlock * 32, 4)
+__global__ void __launch_bounds__(kMaxWarpsPerBlock * 32, 1)
 fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, const int32_t* __restrict__ order,
            const int32_t* __restrict__ start, FitClasses cls, int lm_trials, int min_fit_points,
            unsigned int* queue, long long* counters, int32_t* err_word) {
@@ -1034,16 +1035,6 @@ size_t fit_smem_bytes(const FitClasses& c, int warps) {
     return sizeof(double) * ((size_t)c.h_max + (size_t)warps * ((size_t)(c.rows + 1) * 32 + kParked * 32));
 }
 
-// Lanes per job for windows up to h_hi points: the smallest group whose warp slice stays
-// within `budget` bytes of shared memory.
-int lanes_for(int h_hi, size_t budget) {
-    for (int L = 2; L <= 32; L <<= 1) {   // at least a pair: its lanes split the two families
-        const size_t slice = sizeof(double) * ((size_t)((h_hi + L - 1) / L + 1) * 32 + kParked * 32);
-        if (slice <= budget) return L;
-    }
-    return 32;
-}
-
 }  // namespace
 
 int launch_fit(slaq_handle* h) {
@@ -1061,15 +1052,20 @@ int launch_fit(slaq_handle* h) {
                                                                      h->scratch.order);
         launches += 3;
     }
-    // length classes, longest first: (max_hist/2, max_hist], (max_hist/4, max_hist/2], ... then (0, 64 or less]
+    // Length classes, longest first.  A warp's slice holds rows_cap rows of 32 points (what the
+    // slice budget leaves after the parked sums and the spare row, and at least what the longest
+    // window needs at 32 lanes); the class with L = 32, 16, .. 2 lanes per job takes the windows
+    // that would need more than rows_cap rows at L/2 lanes.
     FitClasses cls;
     cls.n = 0;
     cls.rows = 1;
     cls.h_max = Hmax;
-    for (int h_hi = Hmax; h_hi > 0;) {
-        int h_lo = h_hi > 64 ? (h_hi + 1) / 2 : 0;
-        if (cls.n == kMaxFitClasses - 1) h_lo = 0;
-        const int L = lanes_for(h_hi, h->fit_slice_bytes);
+    int rows_cap = (int)(h->fit_slice_bytes / (32 * sizeof(double))) - kParked - 1;
+    rows_cap = std::max(rows_cap, (Hmax + 31) / 32);
+    int h_hi = Hmax;
+    for (int L = 32; L >= 2 && h_hi > 0; L >>= 1) {
+        const int h_lo = L > 2 ? rows_cap * (L / 2) : 0;
+        if (h_lo >= h_hi) continue;
         cls.h_lo[cls.n] = h_lo;
         cls.h_hi[cls.n] = h_hi;
         cls.L[cls.n] = L;
