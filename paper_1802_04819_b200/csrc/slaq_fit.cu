@@ -31,7 +31,7 @@ constexpr int kMaxWarpsPerBlock = 16;          // one block per SM: its warps sh
 constexpr size_t kSmemLimit = 226 * 1024;   // shared memory one block may use on sm_100, less the static part
 constexpr unsigned kFull = 0xffffffffu;
 constexpr double kLambda0 = 1e-3, kLambdaMin = 1e-5, kLambdaMax = 1e12;
-constexpr int kParked = 12;                 // doubles per lane kept in shared memory between sweeps
+constexpr int kParked = 12;                 // doubles per job and family kept in shared memory between sweeps
 
 __device__ __forceinline__ bool finite_d(double v) { return fabs(v) <= 1.7976931348623157e308; }
 
@@ -75,9 +75,10 @@ __device__ __forceinline__ int warp_max_int(int v) {
 // every access of the sweeps is lane-private and free of bank conflicts.
 struct Lanes {
     double* y;         // [k_cap + 1][32]
-    double* park;      // [kParked][32]
+    double* park;      // this lane's family of its job in [kParked][2 * jobs per warp] (one column per job and family)
     const double* wtab;
     int lane, L, l;
+    __device__ __forceinline__ int park_stride() const { return 64 >> (__ffs(L) - 1); }   // 2 * (32 / L), L a power of two
 };
 
 // The window value at distance m + 1 from the newest point, seen from the lane that owns m.
@@ -466,25 +467,32 @@ __device__ __forceinline__ void sweep(const Lanes& S, int fam, int H, int k_all,
     out.usable = finite_d(chk) && (odd || feasible);
 }
 
-// The sums of the last accepted point live in the lane's shared-memory column between sweeps.
-__device__ __forceinline__ void park(const Lanes& S, const SweepSums& s) {
-    double* c = S.park + S.lane;
+// The sums of the last accepted point live in shared memory between sweeps, one column per job
+// and family: after the reduction every lane of a group's parity holds the same sums, so the
+// group's first two lanes write them for all.  Every lane of the warp calls this; `keep` says
+// whether the lane's family has new sums to park.
+__device__ __forceinline__ void park(const Lanes& S, const SweepSums& s, bool keep) {
+    if (keep && S.l < 2) {
+        const int n = S.park_stride();
 #pragma unroll
-    for (int k = 0; k < kParked; ++k) c[k * 32] = s.v[k];
+        for (int k = 0; k < kParked; ++k) S.park[k * n] = s.v[k];
+    }
+    __syncwarp();
 }
 
 // Normal equations A = sum w J J^T, g = sum w J r of the lane's family from the parked sums.
 __device__ __forceinline__ void normal_equations(const Lanes& S, int fam, double sw, Sym4& A, double (&g)[4]) {
-    const double* c = S.park + S.lane;
+    const double* c = S.park;
+    const int n = S.park_stride();
     if (fam == 0) {
-        A.a00 = c[4 * 32]; A.a01 = c[3 * 32]; A.a02 = c[2 * 32]; A.a11 = c[2 * 32]; A.a12 = c[1 * 32];
-        A.a22 = c[0 * 32];
-        A.a03 = -c[7 * 32]; A.a13 = -c[6 * 32]; A.a23 = -c[5 * 32]; A.a33 = sw;
-        g[0] = -c[10 * 32]; g[1] = -c[9 * 32]; g[2] = -c[8 * 32]; g[3] = c[11 * 32];
+        A.a00 = c[4 * n]; A.a01 = c[3 * n]; A.a02 = c[2 * n]; A.a11 = c[2 * n]; A.a12 = c[1 * n];
+        A.a22 = c[0];
+        A.a03 = -c[7 * n]; A.a13 = -c[6 * n]; A.a23 = -c[5 * n]; A.a33 = sw;
+        g[0] = -c[10 * n]; g[1] = -c[9 * n]; g[2] = -c[8 * n]; g[3] = c[11 * n];
     } else {
-        A.a00 = c[0 * 32]; A.a01 = -c[1 * 32]; A.a11 = c[2 * 32]; A.a02 = c[3 * 32]; A.a12 = -c[4 * 32]; A.a22 = sw;
+        A.a00 = c[0]; A.a01 = -c[1 * n]; A.a11 = c[2 * n]; A.a02 = c[3 * n]; A.a12 = -c[4 * n]; A.a22 = sw;
         A.a03 = 0.0; A.a13 = 0.0; A.a23 = 0.0; A.a33 = 1.0;
-        g[0] = c[5 * 32]; g[1] = -c[6 * 32]; g[2] = c[7 * 32]; g[3] = 0.0;
+        g[0] = c[5 * n]; g[1] = -c[6 * n]; g[2] = c[7 * n]; g[3] = 0.0;
     }
 }
 
@@ -645,6 +653,7 @@ struct FitClasses {
     int h_lo[kMaxFitClasses], h_hi[kMaxFitClasses], L[kMaxFitClasses];
     int rows;        // sweeps a lane makes at most, over all classes
     int h_max;       // longest window
+    int slice;       // doubles of shared memory per warp: parked sums, window rows, one spare row
 };
 
 // kWarm: families may start from last epoch's parameters (a separate instantiation, so that the
@@ -658,10 +667,8 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
     __shared__ int slot_base[kMaxFitClasses + 1];
     double* wtab = smem;                                   // [h_max]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const size_t per_warp = (size_t)(cls.rows + 1) * 32 + kParked * 32;   // one spare row for neighbour reads
+    double* const slice = smem + cls.h_max + (size_t)warp * cls.slice;   // this warp's: parked sums, then the window rows
     Lanes S;
-    S.y = smem + cls.h_max + warp * per_warp;
-    S.park = S.y + (size_t)(cls.rows + 1) * 32;
     S.wtab = wtab;
     S.lane = lane;
     for (int i = threadIdx.x; i < cls.h_max; i += blockDim.x) wtab[i] = g_wtab[i];
@@ -691,6 +698,8 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         S.L = L;
         S.l = lane & (L - 1);
         const int G = 32 / L, g = lane / L;
+        S.park = slice + 2 * g + (lane & 1);
+        S.y = slice + kParked * 2 * G;
         const int last = start[cls.h_lo[c]];
         const int base = start[h_hi] + (slot - slot_base[c]) * G;
         const int idx = base + g;
@@ -707,6 +716,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         double S_out[2] = {CUDART_INF, CUDART_INF};
         int sweeps_out[2] = {0, 0};
         int ended = 0;   // bit 0 / 1: family I / II ended with a finite residual
+        double both_out[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};   // both families' end points
         const double span = (double)max(H - 1, 1);
         const bool fits = status == SLAQ_JOB_FITTED && H >= min_fit_points;   // this lane's job gets curves fitted
 
@@ -761,7 +771,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
             F.done = !F.ok;
             F.has_trial = false;
             F.predicted = 0.0;
-            park(S, sums);
+            park(S, sums, true);
             for (int t = 0; t < lm_trials; ++t) {
                 if (!__any_sync(kFull, !F.done)) break;
                 double trial[4] = {0.0, 0.0, 0.0, 0.0};
@@ -779,7 +789,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
                     pII[a] = __shfl_sync(kFull, trial[a], oddl);
                 }
                 sweep(S, fam, H, k_all, inv_span, pI, (trying >> even) & 1u, pII, (trying >> oddl) & 1u, sums);
-                if (finish_trial(F, trial, sums.usable, sums.v[fam ? 8 : 12])) park(S, sums);
+                park(S, sums, finish_trial(F, trial, sums.usable, sums.v[fam ? 8 : 12]));
             }
             // both results of the job, in every lane
             const double S_I = __shfl_sync(kFull, F.S, even), S_II = __shfl_sync(kFull, F.S, oddl);
@@ -796,14 +806,8 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
                 if (ok_II) S_out[1] = S_II;
                 const bool okI = ok_I && finite_d(S_I), okII = ok_II && finite_d(S_II);
                 ended = (okI ? 1 : 0) | (okII ? 2 : 0);
-                if (S.l == 0 && ended) {   // what the next epoch may start from
-                    fit.k_fit[j] = job.k_last[j];
 #pragma unroll
-                    for (int a = 0; a < 4; ++a) {
-                        fit.both[8 * (size_t)j + a] = pI[a];
-                        fit.both[8 * (size_t)j + 4 + a] = pII[a];
-                    }
-                }
+                for (int a = 0; a < 4; ++a) both_out[a] = pI[a], both_out[4 + a] = pII[a];
                 if (okI && (!okII || S_I <= S_II)) {   // a tie goes to family I
                     family = 0;
 #pragma unroll
@@ -845,6 +849,11 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
             }
             fit.status[j] = status;
             fit.mask[j] = (uint8_t)ended;
+            if (ended) {   // what the next epoch may start from
+                fit.k_fit[j] = job.k_last[j];
+#pragma unroll
+                for (int a = 0; a < 8; ++a) fit.both[8 * (size_t)j + a] = both_out[a];
+            }
             fit.family[j] = (int8_t)family;
 #pragma unroll
             for (int a = 0; a < 4; ++a) fit.params[4 * (size_t)j + a] = p_out[a];
@@ -1032,7 +1041,7 @@ length_scatter_kernel(const int32_t* __restrict__ count, int max_jobs, int max_h
 }
 
 size_t fit_smem_bytes(const FitClasses& c, int warps) {
-    return sizeof(double) * ((size_t)c.h_max + (size_t)warps * ((size_t)(c.rows + 1) * 32 + kParked * 32));
+    return sizeof(double) * ((size_t)c.h_max + (size_t)warps * (size_t)c.slice);
 }
 
 }  // namespace
@@ -1052,19 +1061,21 @@ int launch_fit(slaq_handle* h) {
                                                                      h->scratch.order);
         launches += 3;
     }
-    // Length classes, longest first.  A warp's slice holds rows_cap rows of 32 points (what the
-    // slice budget leaves after the parked sums and the spare row, and at least what the longest
-    // window needs at 32 lanes); the class with L = 32, 16, .. 2 lanes per job takes the windows
-    // that would need more than rows_cap rows at L/2 lanes.
+    // Length classes, longest first.  A warp's slice holds the parked sums of its jobs (kParked
+    // doubles per job and family), the window rows of 32 points and one spare row; with L lanes
+    // per job that leaves rows_at(L) rows.  The class with L = 32, 16, .. 2 lanes per job takes
+    // the windows that do not fit at L/2 lanes.  The slice grows if the longest window does not
+    // fit at 32 lanes.
     FitClasses cls;
     cls.n = 0;
     cls.rows = 1;
     cls.h_max = Hmax;
-    int rows_cap = (int)(h->fit_slice_bytes / (32 * sizeof(double))) - kParked - 1;
-    rows_cap = std::max(rows_cap, (Hmax + 31) / 32);
+    cls.slice = (int)(h->fit_slice_bytes / sizeof(double));
+    cls.slice = std::max(cls.slice, kParked * 2 + ((Hmax + 31) / 32 + 1) * 32);
+    auto rows_at = [&](int L) { return (cls.slice - kParked * (64 / L)) / 32 - 1; };
     int h_hi = Hmax;
     for (int L = 32; L >= 2 && h_hi > 0; L >>= 1) {
-        const int h_lo = L > 2 ? rows_cap * (L / 2) : 0;
+        const int h_lo = L > 2 ? std::max(rows_at(L / 2), 0) * (L / 2) : 0;
         if (h_lo >= h_hi) continue;
         cls.h_lo[cls.n] = h_lo;
         cls.h_hi[cls.n] = h_hi;

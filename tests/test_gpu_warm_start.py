@@ -251,3 +251,31 @@ def test_replacing_a_history_forgets_its_fit(slaq, oracle_mod):
     got, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
     out = ref.schedule(wl.epoch_seconds, wl.total_cores)
     compare_epoch(got, sched.get_predictions(), out, wl.total_cores, wl.max_cores_per_job)
+
+
+@pytest.mark.parametrize("warm", [False, True])
+def test_the_fitted_curves_are_recorded_with_and_without_warm_start(slaq, oracle_mod, warm):
+    """After an epoch the scheduler state holds both families' end points, the iteration index they belong to
+    and the window's span and scale, whether or not the next fit will start from them: the recorded curve of
+    the winning family is the one the predictions were made from, bit for bit, and the record agrees with the
+    oracle's in which families ended with a finite residual."""
+    wl = make_workload(2, n_jobs=1200)
+    sched, ref = _pair(slaq, oracle_mod, wl, int(wl.max_hist), 20, warm=warm)
+    ids = np.arange(wl.n_jobs, dtype=np.int32)
+    sched.load_histories(ids, wl.offsets, wl.losses, wl.k_last)
+    ref.load_histories(ids, wl.offsets, wl.losses, wl.k_last)
+    sched.schedule(wl.epoch_seconds, wl.total_cores)
+    out = ref.schedule(wl.epoch_seconds, wl.total_cores)
+    st, pred = sched.get_fit_state(), sched.get_predictions(want_gain=False)
+    np.testing.assert_array_equal(st["valid"], out["mask"])
+    fitted = out["mask"] != 0
+    assert fitted.sum() > 1000
+    np.testing.assert_array_equal(st["K"][fitted], wl.k_last[fitted])
+    np.testing.assert_array_equal(st["span"][fitted], np.maximum(wl.hist_len[fitted] - 1, 1).astype(np.float64))
+    np.testing.assert_array_equal(st["M"][fitted], pred["M"][fitted])
+    for fam in (0, 1):
+        won = fitted & (pred["family"] == fam)
+        assert won.sum() > 50
+        width = 4 if fam == 0 else 3
+        np.testing.assert_array_equal(st["p"][won, 4 * fam:4 * fam + width], pred["params"][won, :width])
+    sched.close()
