@@ -65,7 +65,7 @@ enum {
     SLAQ_P_FIT_SLICE_BYTES = 5,   /* tuning: shared memory one warp of the fit kernel may use (8 KB..200 KB,
                                      default 13,824: sixteen warps per SM); decides how many lanes share a
                                      job; results stay within rounding */
-    SLAQ_P_WARM_START = 6         /* 0 (default) or 1.  The scheduler refits every job at short intervals
+    SLAQ_P_WARM_START = 6,        /* 0 (default) or 1.  The scheduler refits every job at short intervals
                                      (Evaluation, "Scalability and efficiency"); with 1, a family starts from the
                                      parameters the job's last epoch ended with, carried into this epoch's window
                                      coordinates, instead of from its linearised first guess (which it still uses
@@ -74,6 +74,12 @@ enum {
                                      slaq_schedule stays repeatable.  Together with a smaller SLAQ_P_LM_TRIALS
                                      this spreads a fit's iterations over the epochs.  The paper does not say how
                                      its fits are started. */
+    SLAQ_P_FIT_CLUSTER_JOBS = 7   /* tuning: with few active jobs the fit gives every job more lanes (up to a whole
+                                     warp), so that a small cluster still fills the GPU; the number of lanes is
+                                     chosen from the handle's active jobs.  A handle that holds one shard of a
+                                     larger cluster is told the cluster's number of active jobs here, so that
+                                     every shard makes the choice the undivided cluster would make and the
+                                     results agree bit for bit; 0 (default): the handle's own active jobs */
 };
 
 /* per-job status written by slaq_schedule (slaq_get_predictions, out_status) */

@@ -580,6 +580,10 @@ int slaq_set_param(slaq_t* h, int key, double value) {
             if (!(value == 0.0 || value == 1.0)) return fail(h, SLAQ_E_ARG, "warm start must be 0 or 1");
             h->warm_start = value != 0.0;
             return SLAQ_OK;
+        case SLAQ_P_FIT_CLUSTER_JOBS:
+            if (!(value >= 0.0 && value <= 1e15)) return fail(h, SLAQ_E_ARG, "cluster jobs must not be negative");
+            h->fit_cluster_jobs = (int64_t)value;
+            return SLAQ_OK;
         default:
             return fail(h, SLAQ_E_ARG, "unknown parameter key");
     }
@@ -594,6 +598,7 @@ int slaq_get_param(const slaq_t* h, int key, double* out_value) {
         case SLAQ_P_MIN_FIT_POINTS: *out_value = h->min_fit_points; return SLAQ_OK;
         case SLAQ_P_FIT_SLICE_BYTES: *out_value = (double)h->fit_slice_bytes; return SLAQ_OK;
         case SLAQ_P_WARM_START: *out_value = h->warm_start ? 1.0 : 0.0; return SLAQ_OK;
+        case SLAQ_P_FIT_CLUSTER_JOBS: *out_value = (double)h->fit_cluster_jobs; return SLAQ_OK;
         default: return SLAQ_E_ARG;
     }
 }

@@ -9,9 +9,10 @@
 //
 // Work split.  Jobs are sorted by window length (counting sort, longest first) and cut into
 // length classes.  In class c a group of L lanes (L = 2, 4, .. 32: the fewest lanes at which
-// the window fits the rows of a warp's shared-memory slice) owns one job, so a warp carries
-// 32/L jobs.  One persistent launch (one block of 16 warps per SM) serves all classes from
-// one work queue, longest windows first.  A lane
+// the window fits the rows of a warp's shared-memory slice) owns one job (so a warp carries
+// 32/L jobs; with few active jobs L is raised so that every warp of the GPU has work).  One
+// persistent launch (one block of 16 warps per SM) serves all classes from one work queue,
+// longest windows first.  A lane
 // walks its job's points m = l, l + L, l + 2L, ... counted from the newest one; both families
 // are evaluated in the same sweep over the window; the partial sums of the normal equations
 // are reduced over the L lanes with shuffles; the even lanes of a group then run family I's
@@ -1073,9 +1074,15 @@ int launch_fit(slaq_handle* h) {
     cls.slice = (int)(h->fit_slice_bytes / sizeof(double));
     cls.slice = std::max(cls.slice, kParked * 2 + ((Hmax + 31) / 32 + 1) * 32);
     auto rows_at = [&](int L) { return (cls.slice - kParked * (64 / L)) / 32 - 1; };
+    // With few active jobs every job gets more lanes, so that the warps of the GPU all have work:
+    // the fewest lanes at which the jobs fill about two slots per warp.
+    const long long jobs_for_lanes = h->fit_cluster_jobs > 0 ? (long long)h->fit_cluster_jobs : (long long)h->n_active;
+    const long long lanes_wanted = 64LL * h->sm_count * kMaxWarpsPerBlock;
+    int L_min = 2;
+    while (L_min < 32 && jobs_for_lanes * L_min < lanes_wanted) L_min <<= 1;
     int h_hi = Hmax;
-    for (int L = 32; L >= 2 && h_hi > 0; L >>= 1) {
-        const int h_lo = L > 2 ? std::max(rows_at(L / 2), 0) * (L / 2) : 0;
+    for (int L = 32; L >= L_min && h_hi > 0; L >>= 1) {
+        const int h_lo = L > L_min ? std::max(rows_at(L / 2), 0) * (L / 2) : 0;
         if (h_lo >= h_hi) continue;
         cls.h_lo[cls.n] = h_lo;
         cls.h_hi[cls.n] = h_hi;

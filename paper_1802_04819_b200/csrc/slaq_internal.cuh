@@ -100,6 +100,7 @@ struct slaq_handle {
     int32_t lm_trials = 20, min_fit_points = 4;
     size_t fit_slice_bytes = 13824;       // shared memory one warp of the fit kernel may use (parked sums, up to 52 rows of 32 points, a spare row)
     bool warm_start = false;              // fits start from the last epoch's parameters where there are some
+    int64_t fit_cluster_jobs = 0;         // active jobs the lanes per job are chosen for (0: this handle's own)
     cudaStream_t stream = nullptr;
     bool owns_ws = false;
     void* ws = nullptr;

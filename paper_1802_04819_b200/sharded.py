@@ -12,6 +12,8 @@ at the end one gather of each shard's number of threshold-equal gains.  Two ways
 
 from __future__ import annotations
 
+from .binding import P_FIT_CLUSTER_JOBS
+
 N_PASSES = 6
 N_BINS = 2048
 
@@ -76,6 +78,8 @@ def schedule_sharded(shards, exchange, epoch_seconds: float, total_cores: int):
     assert all(s.max_cores_per_job == cap for s in shards)
     n_jobs = exchange.sum_ints([s.get_active_count() for s in shards])[0]
     with_floor = total_cores >= n_jobs
+    for s in shards:                      # every shard fits with the lanes per job the undivided cluster would use
+        s.set_param(P_FIT_CLUSTER_JOBS, n_jobs)
     want = min(total_cores, n_jobs * cap) - (n_jobs if with_floor else 0)
     for s in shards:
         s.shard_predict(epoch_seconds, with_floor)

@@ -316,6 +316,19 @@ def test_lanes_per_job_do_not_change_results_beyond_rounding(slaq, oracle_mod, s
     compare_epoch(alloc, sched.get_predictions(), oracle_epoch(oracle_mod, wl), wl.total_cores, wl.max_cores_per_job)
 
 
+@pytest.mark.parametrize("cluster_jobs", [0, 3000, 40000, 10_000_000])
+def test_lanes_chosen_for_the_number_of_active_jobs_do_not_change_results_beyond_rounding(slaq, oracle_mod,
+                                                                                          cluster_jobs):
+    """With few active jobs a job gets up to a whole warp; a handle told that it is a shard of a large
+    cluster uses as few lanes as its windows allow.  Either way the epoch matches the oracle."""
+    wl = make_workload(3, n_jobs=1500)
+    sched = make_scheduler(wl, packed=True)
+    sched.set_param(slaq.binding.P_FIT_CLUSTER_JOBS, cluster_jobs)
+    assert sched.get_param(slaq.binding.P_FIT_CLUSTER_JOBS) == cluster_jobs
+    alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    compare_epoch(alloc, sched.get_predictions(), oracle_epoch(oracle_mod, wl), wl.total_cores, wl.max_cores_per_job)
+
+
 @pytest.mark.parametrize("gamma", [1.0, 0.5, 0.99])
 def test_other_weight_bases(slaq, oracle_mod, gamma):
     wl = make_workload(2, n_jobs=1200)
