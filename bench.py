@@ -35,8 +35,8 @@ WARM_TRIALS = 5   # trials per epoch of the warm-started loop reported beside th
 FLOP_SWEEP_I, FLOP_SWEEP_II, FLOP_SETUP = 40.0, 25.0, 40.0
 FP64_LANES_PER_SM = 64          # fp64 FMA lanes per SM on B200
 # DRAM bytes per stored loss moved by the fit kernel (ncu: dram__bytes_read.sum + dram__bytes_write.sum =
-# 165.34 MB + 12.64 MB on a 20,068,408-loss cut of this workload; traffic grows with the stored losses)
-NCU_FIT_DRAM_BYTES_PER_LOSS = (165.34e6 + 12.64e6) / 20_068_408
+# 165.72 MB + 13.70 MB on a 20,068,408-loss cut of this workload; traffic grows with the stored losses)
+NCU_FIT_DRAM_BYTES_PER_LOSS = (165.72e6 + 13.70e6) / 20_068_408
 
 
 from paper_1802_04819_b200.partition import max_over_ranks, partition_seed_offset, rank_info, whole_job_rate  # noqa: E402
