@@ -215,17 +215,20 @@ def run_gpu(args):
     # ---- end to end through the host-pointer calls: append one new loss per job, schedule, read the allocation ----
     rng = np.random.default_rng(99 + rank)
     pin = lambda n, dt: torch.empty(n, dtype=dt).pin_memory().numpy()   # noqa: E731
-    h_ids, h_loss, h_time = pin(J, torch.int32), pin(J, torch.float64), pin(J, torch.float64)
+    h_ids, h_time = pin(J, torch.int32), pin(J, torch.float64)
     h_alloc = pin(J, torch.int32)
     h_ids[:] = ids
     e2e_steps = max(1, min(args.steps, 10))
-    feeds = [next_losses(wl, s, rng) for s in range(2 * (args.warmup + e2e_steps))]
-    last = alloc_dev.astype(np.float64)
+    # every step's input (one new loss per job and the seconds its iteration took) waits in pinned host memory
+    feeds = []
+    for s in range(2 * (args.warmup + e2e_steps)):
+        buf = pin(J, torch.float64)
+        buf[:] = next_losses(wl, s, rng)
+        feeds.append(buf)
+    h_time[:] = wl.s + wl.w / np.maximum(alloc_dev.astype(np.float64), 1.0)
 
     def e2e_step(k):
-        h_loss[:] = feeds[k]
-        h_time[:] = wl.s + wl.w / np.maximum(last, 1.0)
-        sched.append_losses(h_ids, h_loss, h_time)
+        sched.append_losses(h_ids, feeds[k], h_time)
         sched.schedule(wl.epoch_seconds, wl.total_cores, out_alloc=h_alloc)
 
     for k in range(args.warmup):

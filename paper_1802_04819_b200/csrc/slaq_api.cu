@@ -335,20 +335,32 @@ int do_append(slaq_handle* h, int32_t n, const int32_t* ids, const double* losse
               const int32_t* cores) {
     if (!h) return SLAQ_E_ARG;
     if (n > 0 && !losses) return fail(h, SLAQ_E_ARG, "losses is null");
-    const int rc = check_ids(h, n, ids, true);
-    if (rc) return rc;
-    for (int32_t i = 0; i < n; ++i) {
-        if (!std::isfinite(losses[i])) return fail(h, SLAQ_E_NONFINITE, "a loss is not finite");
-        if (times && !std::isfinite(times[i])) return fail(h, SLAQ_E_NONFINITE, "an iteration time is not finite");
-        if (cores && cores[i] < 1) return fail(h, SLAQ_E_ARG, "cores_used must be at least 1");
+    if (const int dc = check_device(h)) return dc;
+    if (n < 0) return fail(h, SLAQ_E_ARG, "negative count");
+    if (n > 0 && !ids) return fail(h, SLAQ_E_ARG, "job_ids is null");
+    if (n > h->max_jobs) return fail(h, SLAQ_E_ARG, "more entries than job ids");
+    cudaStream_t st = h->stream;
+    // The copies into the staging arrays go first: from pinned memory they run while the host
+    // checks the arguments below.  Nothing reads the staging arrays unless the checks pass.
+    if (n > 0) {
+        CK(cudaMemcpyAsync(h->stage.ids, ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy job ids");
+        CK(cudaMemcpyAsync(h->stage.losses, losses, sizeof(double) * n, cudaMemcpyHostToDevice, st), "copy losses");
+        if (times)
+            CK(cudaMemcpyAsync(h->stage.times, times, sizeof(double) * n, cudaMemcpyHostToDevice, st), "copy times");
+        if (times && cores)
+            CK(cudaMemcpyAsync(h->stage.cores, cores, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy cores");
+    }
+    int bad = check_ids(h, n, ids, true);
+    for (int32_t i = 0; i < n && !bad; ++i) {
+        if (!std::isfinite(losses[i])) bad = fail(h, SLAQ_E_NONFINITE, "a loss is not finite");
+        else if (times && !std::isfinite(times[i])) bad = fail(h, SLAQ_E_NONFINITE, "an iteration time is not finite");
+        else if (cores && cores[i] < 1) bad = fail(h, SLAQ_E_ARG, "cores_used must be at least 1");
+    }
+    if (bad) {
+        cudaStreamSynchronize(st);   // the caller's buffers are free again; the state is untouched
+        return bad;
     }
     if (n == 0) return SLAQ_OK;
-    cudaStream_t st = h->stream;
-    CK(cudaMemcpyAsync(h->stage.ids, ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy job ids");
-    CK(cudaMemcpyAsync(h->stage.losses, losses, sizeof(double) * n, cudaMemcpyHostToDevice, st), "copy losses");
-    if (times) CK(cudaMemcpyAsync(h->stage.times, times, sizeof(double) * n, cudaMemcpyHostToDevice, st), "copy times");
-    if (times && cores)
-        CK(cudaMemcpyAsync(h->stage.cores, cores, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy cores");
     const int threads = 256;
     append_kernel<<<(n + threads - 1) / threads, threads, 0, st>>>(
         h->job, h->fit, h->max_jobs, n, h->stage.ids, h->stage.losses, times ? h->stage.times : nullptr,
