@@ -26,6 +26,19 @@ def test_every_declared_symbol_is_exported(lib):
     assert declared == set(slaq.EXPORTED_SYMBOLS)
 
 
+def test_binding_constants_match_the_header():
+    """Parameter keys, job states and warning codes are typed twice (C header, Python binding)."""
+    from paper_1802_04819_b200 import binding
+    header = (ROOT / "include" / "slaq.h").read_text()
+    values = {name: int(v) for name, v in re.findall(r"\b(SLAQ_[A-Z_]+)\s*=\s*(-?\d+)", header)}
+    keys = [n for n in values if n.startswith("SLAQ_P_")]
+    assert len(keys) >= 7
+    for name in keys:
+        assert getattr(binding, name[len("SLAQ_"):]) == values[name], name
+    for name in [n for n in values if n.startswith("SLAQ_JOB_") or n.startswith("SLAQ_W_")]:
+        assert getattr(binding, name[len("SLAQ_"):]) == values[name], name
+
+
 def test_workspace_size_is_host_arithmetic(lib):
     import paper_1802_04819_b200 as slaq
     small = slaq.workspace_bytes(8, 20, 16)

@@ -32,7 +32,7 @@ def _worker(rank, world, port, out):
 
 def test_two_ranks_partition_and_timing():
     world, port = 2, 29531 + os.getpid() % 400
-    manager = mp.Manager()
+    manager = mp.get_context("spawn").Manager()
     out = manager.dict()
     mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
     a, b = out[0], out[1]
@@ -61,7 +61,7 @@ def test_shard_exchange_over_a_process_group():
     """What the shards of one cluster exchange per epoch (sums of histograms and counts, gathered tie counts),
     over gloo on CPU; on GPUs the same calls run over NCCL."""
     world, port = 2, 29931 + os.getpid() % 400
-    out = mp.Manager().dict()
+    out = mp.get_context("spawn").Manager().dict()
     mp.spawn(_exchange_worker, args=(world, port, out), nprocs=world, join=True)
     for rank in range(world):
         assert out[rank]["total"] == [21]
