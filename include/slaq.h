@@ -74,12 +74,18 @@ enum {
                                      slaq_schedule stays repeatable.  Together with a smaller SLAQ_P_LM_TRIALS
                                      this spreads a fit's iterations over the epochs.  The paper does not say how
                                      its fits are started. */
-    SLAQ_P_FIT_CLUSTER_JOBS = 7   /* tuning: with few active jobs the fit gives every job more lanes (up to a whole
+    SLAQ_P_FIT_CLUSTER_JOBS = 7,  /* tuning: with few active jobs the fit gives every job more lanes (up to a whole
                                      warp), so that a small cluster still fills the GPU; the number of lanes is
                                      chosen from the handle's active jobs.  A handle that holds one shard of a
                                      larger cluster is told the cluster's number of active jobs here, so that
                                      every shard makes the choice the undivided cluster would make and the
                                      results agree bit for bit; 0 (default): the handle's own active jobs */
+    SLAQ_P_EPOCH_GRAPH = 8        /* 1: slaq_schedule / slaq_schedule_device replay the epoch's launches as one
+                                     CUDA graph once two calls in a row had the same arguments, parameters and
+                                     number of active jobs (an epoch of a small cluster is bound by its sixteen
+                                     launches); 0: always plain launches; -1 (default): graph for handles
+                                     created for at most 20,000 jobs.  Results are the same either way.  Not
+                                     used while the handle's stream is itself being captured. */
 };
 
 /* per-job status written by slaq_schedule (slaq_get_predictions, out_status) */
@@ -97,7 +103,7 @@ enum {
 /* Timings and counts of the last slaq_schedule / slaq_schedule_device call. */
 typedef struct slaq_stats {
     float ms_total;        /* device time of the whole epoch */
-    float ms_fit;          /* normalise + fit kernel */
+    float ms_fit;          /* normalise + fit kernel (the three stage times are 0 for an epoch replayed as a CUDA graph) */
     float ms_gain;         /* marginal-gain kernel (with the first selection histogram) */
     float ms_alloc;        /* threshold selection, per-job counts, allocation */
     int32_t launches;      /* kernels launched by the call */

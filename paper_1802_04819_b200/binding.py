@@ -12,6 +12,7 @@ from .build import LIB
 JOB_INACTIVE, JOB_FITTED, JOB_SHORT, JOB_NEW, JOB_FIT_FAILED, JOB_FLAT, JOB_NONFINITE, JOB_NO_TIME = -1, 0, 1, 2, 3, 4, 5, 6
 P_GAMMA, P_LM_TRIALS, P_MAX_CORES_PER_JOB, P_MIN_FIT_POINTS, P_FIT_SLICE_BYTES, P_WARM_START = 1, 2, 3, 4, 5, 6
 P_FIT_CLUSTER_JOBS = 7
+P_EPOCH_GRAPH = 8
 W_OVERSUBSCRIBED, W_UNDERFILLED = 1, 2
 
 EXPORTED_SYMBOLS = [

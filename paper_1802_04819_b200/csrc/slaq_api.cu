@@ -472,6 +472,43 @@ int do_load(slaq_handle* h, int32_t n, const int32_t* ids, const int64_t* offset
     return SLAQ_OK;
 }
 
+// The launches of one epoch, put on h->stream in order.  Returns the number of kernels or -1.
+// with_events: the stage boundaries are marked with the handle's events (left out of a captured
+// graph: events recorded by a graph cannot be timed).
+int enqueue_epoch(slaq_handle* h, double T, int64_t want, int floor_units, int32_t* d_out, bool only_allocate,
+                  bool with_events) {
+    cudaStream_t st = h->stream;
+    int launches = 0, k;
+    if (with_events && cudaEventRecord(h->ev[0], st) != cudaSuccess) return -1;
+    if (cudaMemsetAsync(h->scratch.hist, 0, h->scratch.zero_bytes, st) != cudaSuccess) return -1;
+    if (!only_allocate) {
+        if ((k = launch_fit(h)) < 0) return -1;
+        launches += k;
+    }
+    if (with_events && cudaEventRecord(h->ev[1], st) != cudaSuccess) return -1;
+    if (!only_allocate) {
+        if ((k = launch_gain(h, T, floor_units + 1)) < 0) return -1;
+        launches += k;
+    }
+    if (with_events && cudaEventRecord(h->ev[2], st) != cudaSuccess) return -1;
+    if ((k = launch_allocate(h, want, floor_units + 1, !only_allocate, d_out)) < 0) return -1;
+    launches += k;
+    if (with_events && cudaEventRecord(h->ev[3], st) != cudaSuccess) return -1;
+    return launches;
+}
+
+// Everything the epoch's launches depend on besides device data: a graph captured for one
+// key is replayed only for the same key.
+std::vector<long long> epoch_key(const slaq_handle* h, double T, int64_t want, int floor_units, const int32_t* d_out,
+                                 bool only_allocate) {
+    long long t_bits, g_bits;
+    std::memcpy(&t_bits, &T, sizeof t_bits);
+    std::memcpy(&g_bits, &h->gamma, sizeof g_bits);
+    return {t_bits, (long long)want, floor_units, (long long)(uintptr_t)d_out, only_allocate ? 1 : 0, h->n_active,
+            h->max_cores, h->lm_trials, h->min_fit_points, h->warm_start ? 1 : 0, (long long)h->fit_slice_bytes,
+            (long long)h->fit_cluster_jobs, g_bits};
+}
+
 int run_epoch(slaq_handle* h, double T, int64_t C, int32_t* d_out, bool only_allocate) {
     if (!only_allocate && !(T > 0.0 && std::isfinite(T))) return fail(h, SLAQ_E_ARG, "epoch_seconds must be positive");
     if (C < 0) return fail(h, SLAQ_E_ARG, "total_cores must not be negative");
@@ -483,22 +520,66 @@ int run_epoch(slaq_handle* h, double T, int64_t C, int32_t* d_out, bool only_all
     const int64_t usable = std::min<int64_t>(C, active * cap);
     const int64_t want = usable - active * floor_units;
     cudaStream_t st = h->stream;
-    int launches = 0, k;
-    CK(cudaMemsetAsync(h->scratch.hist, 0, h->scratch.zero_bytes, st), "clear scratch");
-    CK(cudaEventRecord(h->ev[0], st), "event");
-    if (!only_allocate) {
-        if ((k = launch_fit(h)) < 0) return SLAQ_E_CUDA;
-        launches += k;
+
+    bool graph_ok = h->epoch_graph == 1 || (h->epoch_graph < 0 && h->max_jobs <= kGraphAutoJobs);
+    if (graph_ok) {   // not while the caller captures this stream into a graph of its own
+        cudaStreamCaptureStatus status = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &status) != cudaSuccess || status != cudaStreamCaptureStatusNone) graph_ok = false;
+        if (!graph_ok) cudaGetLastError();
     }
-    CK(cudaEventRecord(h->ev[1], st), "event");
-    if (!only_allocate) {
-        if ((k = launch_gain(h, T, floor_units + 1)) < 0) return SLAQ_E_CUDA;
-        launches += k;
+    int launches = -1;
+    h->last_epoch_was_graph = false;
+    if (graph_ok) {
+        const std::vector<long long> key = epoch_key(h, T, want, floor_units, d_out, only_allocate);
+        if (h->graph_exec && key == h->graph_key) {
+            CK(cudaEventRecord(h->ev[0], st), "event");
+            CK(cudaGraphLaunch(h->graph_exec, st), "launch epoch graph");
+            CK(cudaEventRecord(h->ev[3], st), "event");
+            launches = h->graph_launches;
+            h->last_epoch_was_graph = true;
+        } else if (key == h->seen_key) {   // the second call in a row with this key: capture, then replay
+            if (!h->capture_stream)
+                CK(cudaStreamCreateWithFlags(&h->capture_stream, cudaStreamNonBlocking), "create capture stream");
+            CK(cudaStreamBeginCapture(h->capture_stream, cudaStreamCaptureModeRelaxed), "begin capture");
+            h->stream = h->capture_stream;
+            const int n = enqueue_epoch(h, T, want, floor_units, d_out, only_allocate, false);
+            h->stream = st;
+            cudaGraph_t graph = nullptr;
+            const cudaError_t e_end = cudaStreamEndCapture(h->capture_stream, &graph);
+            if (n >= 0 && e_end == cudaSuccess && graph) {
+                if (h->graph_exec) {
+                    cudaGraphExecDestroy(h->graph_exec);
+                    h->graph_exec = nullptr;
+                }
+                const cudaError_t e_inst = cudaGraphInstantiate(&h->graph_exec, graph, 0);
+                cudaGraphDestroy(graph);
+                if (e_inst == cudaSuccess) {
+                    h->graph_key = key;
+                    h->graph_launches = n;
+                    CK(cudaEventRecord(h->ev[0], st), "event");
+                    CK(cudaGraphLaunch(h->graph_exec, st), "launch epoch graph");
+                    CK(cudaEventRecord(h->ev[3], st), "event");
+                    launches = n;
+                    h->last_epoch_was_graph = true;
+                } else {
+                    h->graph_exec = nullptr;
+                    cudaGetLastError();
+                }
+            } else {
+                if (graph) cudaGraphDestroy(graph);
+                cudaGetLastError();
+                if (n < 0) return SLAQ_E_CUDA;
+            }
+        }
+        h->seen_key = key;
     }
-    CK(cudaEventRecord(h->ev[2], st), "event");
-    if ((k = launch_allocate(h, want, floor_units + 1, !only_allocate, d_out)) < 0) return SLAQ_E_CUDA;
-    launches += k;
-    CK(cudaEventRecord(h->ev[3], st), "event");
+    if (launches < 0) {
+        launches = enqueue_epoch(h, T, want, floor_units, d_out, only_allocate, true);
+        if (launches < 0) {
+            if (h->err.empty()) h->err = "an epoch launch failed";
+            return SLAQ_E_CUDA;
+        }
+    }
     h->have_epoch = true;
     h->last_launches = launches;
     h->last_cores = usable;
@@ -548,6 +629,8 @@ int slaq_destroy(slaq_t* h) {
     if (h->ws) cudaStreamSynchronize(h->stream);
     for (auto& ev : h->ev)
         if (ev) cudaEventDestroy(ev);
+    if (h->graph_exec) cudaGraphExecDestroy(h->graph_exec);
+    if (h->capture_stream) cudaStreamDestroy(h->capture_stream);
     if (h->packed_pool) cudaFree(h->packed_pool);
     if (h->owns_ws && h->ws) cudaFree(h->ws);
     delete h;
@@ -596,6 +679,10 @@ int slaq_set_param(slaq_t* h, int key, double value) {
             if (!(value >= 0.0 && value <= 1e15)) return fail(h, SLAQ_E_ARG, "cluster jobs must not be negative");
             h->fit_cluster_jobs = (int64_t)value;
             return SLAQ_OK;
+        case SLAQ_P_EPOCH_GRAPH:
+            if (!(value == -1.0 || value == 0.0 || value == 1.0)) return fail(h, SLAQ_E_ARG, "epoch graph must be -1, 0 or 1");
+            h->epoch_graph = (int)value;
+            return SLAQ_OK;
         default:
             return fail(h, SLAQ_E_ARG, "unknown parameter key");
     }
@@ -611,6 +698,7 @@ int slaq_get_param(const slaq_t* h, int key, double* out_value) {
         case SLAQ_P_FIT_SLICE_BYTES: *out_value = (double)h->fit_slice_bytes; return SLAQ_OK;
         case SLAQ_P_WARM_START: *out_value = h->warm_start ? 1.0 : 0.0; return SLAQ_OK;
         case SLAQ_P_FIT_CLUSTER_JOBS: *out_value = (double)h->fit_cluster_jobs; return SLAQ_OK;
+        case SLAQ_P_EPOCH_GRAPH: *out_value = (double)h->epoch_graph; return SLAQ_OK;
         default: return SLAQ_E_ARG;
     }
 }
@@ -730,6 +818,7 @@ int slaq_shard_predict(slaq_t* h, double epoch_seconds, int32_t with_floor) {
     cudaStream_t st = h->stream;
     int launches = 0, k;
     h->shard_first_unit = with_floor ? 2 : 1;
+    h->last_epoch_was_graph = false;
     CK(cudaMemsetAsync(h->scratch.hist, 0, h->scratch.zero_bytes, st), "clear scratch");
     CK(cudaEventRecord(h->ev[0], st), "event");
     if ((k = launch_fit(h)) < 0) return SLAQ_E_CUDA;
@@ -933,9 +1022,11 @@ int slaq_get_stats(slaq_t* h, slaq_stats* out) {
     CK(cudaMemcpyAsync(&sel, h->scratch.sel, sizeof sel, cudaMemcpyDeviceToHost, h->stream), "copy selection state");
     CK(cudaStreamSynchronize(h->stream), "copy statistics");
     CK(cudaEventElapsedTime(&out->ms_total, h->ev[0], h->ev[3]), "event time");
-    CK(cudaEventElapsedTime(&out->ms_fit, h->ev[0], h->ev[1]), "event time");
-    CK(cudaEventElapsedTime(&out->ms_gain, h->ev[1], h->ev[2]), "event time");
-    CK(cudaEventElapsedTime(&out->ms_alloc, h->ev[2], h->ev[3]), "event time");
+    if (!h->last_epoch_was_graph) {   // a replayed graph has no stage boundaries to time
+        CK(cudaEventElapsedTime(&out->ms_fit, h->ev[0], h->ev[1]), "event time");
+        CK(cudaEventElapsedTime(&out->ms_gain, h->ev[1], h->ev[2]), "event time");
+        CK(cudaEventElapsedTime(&out->ms_alloc, h->ev[2], h->ev[3]), "event time");
+    }
     out->launches = h->last_launches;
     out->active_jobs = h->n_active;
     out->points = counters[0];

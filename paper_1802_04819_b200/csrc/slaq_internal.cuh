@@ -19,6 +19,7 @@ constexpr int kRadixPasses = 6;       // 11 + 11 + 11 + 11 + 11 + 9 bits, most s
 constexpr int kMaxFitClasses = 8;     // window-length classes of the fit (one launch each)
 constexpr int kFitQueueBase = 8;      // ticket[kFitQueueBase + c]: work queue head of class c
 constexpr int kTickets = 16;
+constexpr int kGraphAutoJobs = 20000;  // handles up to this size replay the epoch as a CUDA graph unless told otherwise
 
 // Device-side state of one job, structure of arrays (index = job id).
 struct JobArrays {
@@ -129,6 +130,15 @@ struct slaq_handle {
     uint32_t stamp_epoch = 0;
     int32_t n_active = 0;
     int shard_first_unit = 2;         // set by slaq_shard_predict for the steps that follow
+    // The epoch as a CUDA graph: what the captured launches depended on, the instantiated graph,
+    // and the stream the capture runs on (the caller's stream may be the legacy default stream,
+    // which cannot capture).
+    int epoch_graph = -1;             // 0 never, 1 always, -1: for handles of at most kGraphAutoJobs jobs
+    std::vector<long long> graph_key, seen_key;
+    cudaGraphExec_t graph_exec = nullptr;
+    cudaStream_t capture_stream = nullptr;
+    int32_t graph_launches = 0;
+    bool last_epoch_was_graph = false;
     std::string err;
 };
 
