@@ -12,8 +12,8 @@
 // the window fits the rows of a warp's shared-memory slice) owns one job (so a warp carries
 // 32/L jobs; with few active jobs L is raised so that every warp of the GPU has work).  One
 // persistent launch (one block of 16 warps per SM) serves all classes from one work queue,
-// longest windows first.  A lane
-// walks its job's points m = l, l + L, l + 2L, ... counted from the newest one; both families
+// longest windows first.  A lane walks its job's points m = l, l + L, l + 2L, ... counted
+// from the newest one; both families
 // are evaluated in the same sweep over the window; the partial sums of the normal equations
 // are reduced over the L lanes with shuffles; the even lanes of a group then run family I's
 // solver step for the job and the odd lanes family II's.  All per-job control flow is per
