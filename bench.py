@@ -34,6 +34,9 @@ WARM_TRIALS = 5   # trials per epoch of the warm-started loop reported beside th
 # algorithmic fp64 work of the fit, per stored point: one sweep of family I, one of family II, set-up
 FLOP_SWEEP_I, FLOP_SWEEP_II, FLOP_SETUP = 40.0, 25.0, 40.0
 FP64_LANES_PER_SM = 64          # fp64 FMA lanes per SM on B200
+# The sweep of the fit issues 46 fp64 instructions per point: 92 cycles per warp row if each took 2, but the 15
+# fused multiply-adds on three different registers take 3 (measured with paper_1802_04819_b200/fp64_issue_probe)
+SWEEP_ISSUE_CYCLES_IDEAL, SWEEP_ISSUE_CYCLES_MEASURED_RATES = 92.0, 107.0
 # DRAM bytes per stored loss moved by the fit kernel (ncu: dram__bytes_read.sum + dram__bytes_write.sum =
 # 165.72 MB + 13.70 MB on a 20,068,408-loss cut of this workload; traffic grows with the stored losses)
 NCU_FIT_DRAM_BYTES_PER_LOSS = (165.72e6 + 13.70e6) / 20_068_408
@@ -297,6 +300,11 @@ def run_gpu(args):
                          "traffic": NCU_FIT_DRAM_BYTES_PER_LOSS * int(wl.offsets[-1]),
                          "traffic_note": "bytes per launch, scaled by stored losses from the ncu capture of a 40,000-job cut",
                          "algorithmic_flops_per_launch": fit_flops, "ms_per_launch": fit_ms_avg,
+                         "issue_bound_peak": peak_tflops * SWEEP_ISSUE_CYCLES_IDEAL / SWEEP_ISSUE_CYCLES_MEASURED_RATES,
+                         "frac_of_issue_bound": achieved / (peak_tflops * SWEEP_ISSUE_CYCLES_IDEAL
+                                                            / SWEEP_ISSUE_CYCLES_MEASURED_RATES),
+                         "issue_bound_note": "fp64 instructions on three different registers issue every 3 cycles, "
+                                             "not 2: what a loop of nothing but sweeps could reach",
                          "peak_is": f"{sm_count} SMs x {FP64_LANES_PER_SM} fp64 FMA lanes x 2 x {sm_max:.0f} MHz "
                                     f"(clock from MEASURED_PEAKS.json: {peak_kind})"},
         }
