@@ -252,6 +252,30 @@ def test_empty_scheduler_and_argument_errors(slaq):
         slaq.Scheduler(4, 100000, 4)                # window too long for one warp's shared memory
 
 
+def test_a_rejected_append_leaves_the_state_untouched(slaq):
+    """The library copies an append's arrays to the device while it checks them on the host; a batch that
+    fails a check (a value that is not finite, an id listed twice, an id out of range) must change nothing."""
+    wl = make_workload(1)
+    sched = make_scheduler(wl)
+    before, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    gains = sched.get_predictions()["gain"].copy()
+    ids = np.arange(wl.n_jobs, dtype=np.int32)
+    good = 0.9 * wl.losses[wl.offsets[1:] - 1]
+    for bad_ids, bad_losses, code in ((ids, np.where(ids == 77, np.inf, good), -3),
+                                      (np.where(ids == 5, 4, ids).astype(np.int32), good, -1),
+                                      (np.where(ids == 9, wl.n_jobs, ids).astype(np.int32), good, -2)):
+        with pytest.raises(slaq.SlaqError) as e:
+            sched.append_losses(bad_ids, bad_losses, np.ones(wl.n_jobs))
+        assert e.value.code == code
+        after, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+        np.testing.assert_array_equal(after, before)
+        np.testing.assert_array_equal(sched.get_predictions()["gain"].view(np.int64), gains.view(np.int64))
+    sched.append_losses(ids, good, np.ones(wl.n_jobs))        # and a clean batch is still taken
+    sched.schedule(wl.epoch_seconds, wl.total_cores)
+    assert not np.array_equal(sched.get_predictions()["gain"].view(np.int64), gains.view(np.int64))
+    sched.close()
+
+
 def test_caller_owned_workspace_and_stream(slaq, oracle_mod):
     import torch
     wl = make_workload(1)
