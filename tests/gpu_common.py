@@ -6,11 +6,13 @@ R_RTOL, R_ATOL = 1e-6, 1e-9          # predicted reductions: |gpu - cpu| <= 1e-6
 THRESHOLD_BAND = 1e-9                # allocations may differ where a deciding gain lies this close to the threshold
 
 
-def make_scheduler(wl, packed=False, max_hist=None, workspace=None):
+def make_scheduler(wl, packed=False, max_hist=None, workspace=None, m_seen=None):
+    """m_seen: the largest reduction seen that the handle is told (default: the workload's, which already
+    includes the stored window's own largest reduction)."""
     import paper_1802_04819_b200 as slaq
     sched = slaq.Scheduler(wl.n_jobs, max_hist or wl.max_hist, wl.max_cores_per_job, workspace=workspace)
     ids = np.arange(wl.n_jobs, dtype=np.int32)
-    sched.load_histories(ids, wl.offsets, wl.losses, wl.k_last, wl.m_seen, packed=packed)
+    sched.load_histories(ids, wl.offsets, wl.losses, wl.k_last, wl.m_seen if m_seen is None else m_seen, packed=packed)
     sched.set_time_model(ids, wl.s, wl.w)
     return sched
 

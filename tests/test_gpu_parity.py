@@ -19,13 +19,24 @@ def slaq():
 
 
 # ---------------------------------------------------------------- normalisation: bit-exact
-@pytest.mark.parametrize("cfg,n_jobs,packed", [(1, None, False), (2, None, True), (4, 3000, False)])
-def test_normalisation_is_bit_exact(slaq, oracle_mod, cfg, n_jobs, packed):
+@pytest.mark.parametrize("own_maximum", [False, True])
+@pytest.mark.parametrize("cfg,n_jobs,packed", [(1, None, False), (2, None, True), (4, 3000, False), (3, 2000, True)])
+def test_normalisation_is_bit_exact(slaq, oracle_mod, cfg, n_jobs, packed, own_maximum):
+    """own_maximum: both sides are told only the largest reduction BEFORE the stored window (nothing for a window
+    that starts at iteration 0), so the largest reduction inside the window is found by the kernel itself; the
+    workload's m_seen already contains it."""
     wl = make_workload(cfg, n_jobs=n_jobs)
-    sched = make_scheduler(wl, packed=packed)
+    seen = wl.m_past if own_maximum else wl.m_seen
+    if own_maximum:
+        assert (seen < wl.m_seen).any()          # the window's own maximum decides for some jobs
+    sched = make_scheduler(wl, packed=packed, m_seen=seen)
     ids = np.arange(wl.n_jobs)
     offsets, changes, levels, largest = sched.get_normalised(ids, capacity=int(wl.offsets[-1]))
-    M, dn, y = oracle_mod.normalise(wl.offsets, wl.losses, wl.m_seen)
+    M, dn, y = oracle_mod.normalise(wl.offsets, wl.losses, seen)
+    if own_maximum:                              # typed here: the window's largest one-step reduction joined with the past
+        for j in range(0, wl.n_jobs, max(1, wl.n_jobs // 200)):
+            h = wl.history(j)
+            assert largest[j] == max(seen[j], (h[:-1] - h[1:]).max())
     np.testing.assert_array_equal(offsets, wl.offsets)
     np.testing.assert_array_equal(largest, M)
     usable = np.repeat(M > 0, wl.hist_len)
@@ -371,6 +382,61 @@ def test_other_seeds(slaq, oracle_mod):
         alloc, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
         compare_epoch(alloc, sched.get_predictions(), oracle_epoch(oracle_mod, wl), wl.total_cores,
                       wl.max_cores_per_job)
+
+
+# ---------------------------------------------------------------- four or more points, yet no curve can be started
+@pytest.mark.parametrize("cluster_jobs", [0, 10_000_000])
+@pytest.mark.parametrize("packed", [False, True])
+def test_windows_without_a_usable_start_take_the_fallback(slaq, oracle_mod, packed, cluster_jobs):
+    """Both families fail at their first guess (levels that are integers near 2^53 a few units apart; or a flat
+    window scaled by a tiny largest-reduction-seen, whose squares overflow): the job is predicted from its weighted
+    mean normalised change, capped by its newest level.  The failing windows sit between ordinary ones, at
+    lengths of every class of lanes per job (cluster_jobs = 10^7: as few lanes per job as the window allows, so the
+    short ones share a warp with fifteen other jobs; 0: a whole warp each)."""
+    from workloads import make_unfittable_histories
+    lengths = [4, 5, 6, 9, 33, 64, 82, 83, 204, 205, 408, 409, 816, 817, 1000]
+    o1, l1, m1, drops = make_unfittable_histories(lengths, "staircase", seed=1)
+    o2, l2, m2, _ = make_unfittable_histories(lengths, "flat", seed=2)
+    wl = make_workload(3, hist_lengths=[7, 40, 90, 300, 600, 950] * 12)
+    n_bad = len(lengths)
+    # interleave: ordinary jobs first and last, the failing ones in the middle of the id range
+    half = wl.n_jobs // 2
+    pieces = [(wl.offsets[:half + 1], wl.losses[:wl.offsets[half]], wl.m_seen[:half]), (o1, l1, m1), (o2, l2, m2),
+              (wl.offsets[half:] - wl.offsets[half], wl.losses[wl.offsets[half]:], wl.m_seen[half:])]
+    H = np.concatenate([np.diff(o) for o, _, _ in pieces])
+    offsets = np.concatenate([[0], np.cumsum(H)]).astype(np.int64)
+    losses = np.concatenate([l for _, l, _ in pieces])
+    m_seen = np.concatenate([m for _, _, m in pieces])
+    J, cap, T = H.size, 16, 1.0
+    rng = np.random.default_rng(5)
+    s, w = rng.uniform(0.05, 0.5, J), rng.uniform(1.0, 100.0, J)
+    C = 4 * J
+    sched = slaq.Scheduler(J, 1000, cap)
+    ids = np.arange(J, dtype=np.int32)
+    sched.load_histories(ids, offsets, losses, H.astype(np.int64) - 1, m_seen, packed=packed)
+    sched.set_time_model(ids, s, w)
+    sched.set_param(slaq.binding.P_FIT_CLUSTER_JOBS, cluster_jobs)
+    alloc, rc = sched.schedule(T, C)
+    pred = sched.get_predictions()
+    ref = oracle_mod.schedule(offsets, losses, m_seen, s, w, T, C, cap)
+    compare_epoch(alloc, pred, ref, C, cap)
+    stair = np.arange(half, half + n_bad)
+    flat = np.arange(half + n_bad, half + 2 * n_bad)
+    assert (pred["status"][stair] == slaq.JOB_FIT_FAILED).all() and (pred["status"][flat] == slaq.JOB_FIT_FAILED).all()
+    assert (pred["family"][stair] == -1).all() and np.isinf(pred["S"][stair]).all()
+    ordinary = np.setdiff1d(ids, np.concatenate([stair, flat]))
+    assert (pred["status"][ordinary] == slaq.JOB_FITTED).all()
+    # expected from the rule itself: changes are 1 at the falls and 0 elsewhere, weights 0.9^(H-1-i)
+    n = np.arange(1, cap + 1)
+    for k, j in enumerate(stair):
+        i = np.arange(1, lengths[k])
+        weight = 0.9 ** (lengths[k] - 1 - i)
+        rho = (weight * np.isin(i, drops[k])).sum() / weight.sum()
+        R = rho * T * n / (s[j] * n + w[j])
+        np.testing.assert_allclose(np.cumsum(pred["gain"][j]), R, rtol=1e-12, atol=0)
+        assert pred["params"][j, 1] == losses[offsets[j + 1] - 1] / 2.0 ** -53      # the cap: the newest level
+    assert (pred["gain"][flat] == 0.0).all()
+    assert sched.get_stats().fallback_jobs == 2 * n_bad
 
 
 # ---------------------------------------------------------------- streaming: append -> schedule with the allocation fed back

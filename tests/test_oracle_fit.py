@@ -249,3 +249,48 @@ def test_short_histories_use_linear_extrapolation(oracle_mod):
     out = oracle_mod.predict(np.array([0, 3]), np.array([1.0, 2.0, 3.0]), None, s, w, T, cap)
     assert out["status"][0] == oracle_mod.ST_FLAT   # the loss never fell
     assert (out["gain"][0] == 0).all()
+
+
+def test_windows_on_which_no_family_can_start_use_the_mean_normalised_change(oracle_mod):
+    """Four or more points, yet neither family has a usable starting point: the prediction falls back to
+    the weighted mean normalised reduction per iteration (the rule for short windows), capped by the
+    newest normalised level.  The expected figures are typed from that rule, not taken from the oracle."""
+    from workloads import make_unfittable_histories
+    s, w, T, cap = 0.25, 6.0, 3.0, 8
+    n = np.arange(1, cap + 1)
+    m = T * n / (s * n + w)
+    lengths = [4, 5, 6, 9, 33, 64, 83, 205, 409, 817, 1000]
+    J = len(lengths)
+    # staircase: every fall is exactly the largest one, so the normalised changes are 1 at the falls and 0 elsewhere
+    offsets, losses, m_seen, drops = make_unfittable_histories(lengths, "staircase")
+    out = oracle_mod.predict(offsets, losses, m_seen, np.full(J, s), np.full(J, w), T, cap)
+    assert (out["status"] == oracle_mod.ST_FIT_FAILED).all()
+    assert (out["family"] == -1).all() and np.isinf(out["S"]).all()
+    np.testing.assert_array_equal(out["M"], np.full(J, 2.0 ** -53))
+    for j, H in enumerate(lengths):
+        i = np.arange(1, H)                          # the changes belong to iterations 1 .. H-1
+        weight = GAMMA ** (H - 1 - i)
+        change = np.isin(i, drops[j]).astype(float)
+        rho = (weight * change).sum() / weight.sum()
+        assert 0.0 < rho <= 1.0
+        R = rho * m                                  # far below the cap: the newest level is about 2^53
+        expect = np.diff(np.concatenate([[0.0], R]))
+        np.testing.assert_allclose(out["gain"][j], expect, rtol=1e-12, atol=0)
+    # flat windows under a tiny largest-reduction-seen: nothing ever fell inside the window, so no gain is predicted
+    offsets, losses, m_seen, _ = make_unfittable_histories(lengths, "flat")
+    out = oracle_mod.predict(offsets, losses, m_seen, np.full(J, s), np.full(J, w), T, cap)
+    assert (out["status"] == oracle_mod.ST_FIT_FAILED).all()
+    np.testing.assert_array_equal(out["M"], np.full(J, 1e-300))
+    assert (out["gain"] == 0.0).all()
+
+
+def test_the_cap_of_the_fallback_is_the_newest_normalised_level(oracle_mod):
+    # Three points falling 8 -> 4 -> 3: M = 4, newest level 3/4.  The weighted mean change is
+    # (0.9 * 1 + 1 * 0.25) / 1.9 per iteration; one core stays below the cap, two reach it.
+    s, w, T, cap = np.array([0.0]), np.array([1.0]), 1.0, 5
+    out = oracle_mod.predict(np.array([0, 3]), np.array([8.0, 4.0, 3.0]), None, s, w, T, cap)
+    rho = (0.9 * 1.0 + 0.25) / 1.9
+    R = np.minimum(rho * T * np.arange(1, cap + 1), 0.75)
+    expect = np.minimum.accumulate(np.maximum(np.diff(np.concatenate([[0.0], R])), 0.0))
+    assert R[-1] == 0.75 and R[0] < 0.75
+    np.testing.assert_allclose(out["gain"][0], expect, rtol=1e-13, atol=1e-16)

@@ -51,6 +51,11 @@ MUTATIONS = [
     ("warm start: stretch of the window inverted", "const double r = D.span / warm->span;",
      "const double r = warm->span / D.span;"),
     ("warm start: an unusable carried point is kept", "startedI = rI.ok;", "startedI = true;"),
+    ("fallback: mean change without the weights", "num += (long double)D.w[i] * dnorm;", "num += (long double)dnorm;"),
+    ("fallback: no cap at the newest level", "out.r_cap = D.y[H - 1] > 0.0 ? D.y[H - 1] : kInf;", "out.r_cap = kInf;"),
+    ("fallback: a window of four points or more without a fit predicts nothing",
+     "out.status = (H >= cfg.min_fit_points) ? ST_FIT_FAILED : ST_SHORT;",
+     "out.status = (H >= cfg.min_fit_points) ? ST_FLAT : ST_SHORT;"),
 ]
 
 PINS = [
@@ -69,6 +74,8 @@ PINS = [
     lambda m: [t_warm.test_carried_parameters_describe_the_same_curve(m, f) for f in (0, 1)],
     lambda m: t_warm.test_the_solver_never_ends_above_its_carried_starting_point(m),
     lambda m: t_warm.test_an_unusable_carried_point_falls_back_to_the_first_guess(m),
+    lambda m: t_fit.test_windows_on_which_no_family_can_start_use_the_mean_normalised_change(m),
+    lambda m: t_fit.test_the_cap_of_the_fallback_is_the_newest_normalised_level(m),
 ]
 
 

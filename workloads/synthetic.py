@@ -59,6 +59,8 @@ class Workload:
     family: np.ndarray         # int8 [J]; generating family (ground truth, tests only)
     params: np.ndarray         # float64 [J,4]; (a,b,c,d) or (mu,b0,c0,0) (ground truth, tests only)
     sigma: np.ndarray          # float64 [J]; noise level actually used
+    m_past: np.ndarray = field(default_factory=lambda: np.zeros(0))   # float64 [J]; largest one-step reduction
+                               # BEFORE the stored window only (-inf for a job whose window starts at iteration 0)
     clone_of: np.ndarray = field(default_factory=lambda: np.zeros(0, np.int64))  # int64 [J]; -1 or source id
 
     @property
@@ -215,7 +217,7 @@ def make_workload(cfg: int, n_jobs: int | None = None, seed_offset: int = 0, his
         cfg=cfg, n_jobs=J, total_cores=C, max_cores_per_job=cap, max_hist=int(max(spec["hmax"], H.max())),
         epoch_seconds=float(spec["T"]), offsets=offsets, losses=losses,
         k_last=k0 + H - 1, m_seen=m_seen, s=s, w=w, family=family, params=params,
-        sigma=sigma, clone_of=clone_of,
+        sigma=sigma, clone_of=clone_of, m_past=past,
     )
 
 
@@ -229,3 +231,42 @@ def make_time_samples(wl: Workload, n_samples: int, jobs: np.ndarray | None = No
     cores = np.tile(cyc[np.arange(n_samples) % 4][:, None], (1, jobs.size)).astype(np.int32)
     secs = wl.s[jobs][None, :] + wl.w[jobs][None, :] / cores
     return cores, secs
+
+
+def make_unfittable_histories(lengths, kind: str, seed: int = 0):
+    """Histories of at least four points on which neither curve family can be started.
+
+    kind "staircase": the loss sits just below 1 and falls by exactly one unit in the last place
+    (2^-53) at one to four randomly chosen iterations and stays put otherwise.  Scaled by its
+    largest one-step reduction such a window holds integers near 2^53 that span at most four
+    units, so an offset placed a tenth of that span below the smallest level rounds back onto it.
+    kind "flat": a constant loss; together with a tiny positive largest-reduction-seen (returned as
+    m_seen = 1e-300) the scaled levels are of the order 1e300 and their squares overflow.
+
+    Returns (offsets int64 [n+1], losses float64, m_seen float64 [n], drops: list of index arrays,
+    the iterations i >= 1 at which history j fell).  Only numbers are drawn here.
+    """
+    rng = np.random.default_rng(SEED_BASE + 7000 + seed)
+    lengths = np.asarray(lengths, dtype=np.int64)
+    assert lengths.min() >= 4
+    offsets = np.zeros(lengths.size + 1, dtype=np.int64)
+    np.cumsum(lengths, out=offsets[1:])
+    losses = np.empty(int(offsets[-1]))
+    m_seen = np.full(lengths.size, -np.inf)
+    drops = []
+    unit = 2.0 ** -53
+    for j, H in enumerate(lengths):
+        if kind == "staircase":
+            n_drops = int(rng.integers(1, 5))
+            where = np.sort(rng.choice(np.arange(1, H), size=min(n_drops, H - 1), replace=False))
+            fallen = np.zeros(H)
+            fallen[where] = 1.0
+            losses[offsets[j]:offsets[j + 1]] = 1.0 - np.cumsum(fallen) * unit   # exact: multiples of 2^-53 in [0.5, 1]
+        elif kind == "flat":
+            where = np.zeros(0, dtype=np.int64)
+            losses[offsets[j]:offsets[j + 1]] = rng.uniform(0.5, 4.0)
+            m_seen[j] = 1e-300
+        else:
+            raise ValueError(kind)
+        drops.append(where)
+    return offsets, losses, m_seen, drops
