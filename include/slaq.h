@@ -176,14 +176,17 @@ int slaq_append_losses_ex(slaq_t* h, int32_t n, const int32_t* job_ids, const do
  * is the iteration index of its newest loss; m_seen[i] (array may be NULL) the largest
  * one-step reduction of its earlier life, joined at scheduling time with the window's
  * own.  If a history is longer than max_hist only its newest max_hist points are kept.
- * Time sums and time models are left as they are.  Host pointers.
+ * Time sums, time models and current core counts of the listed jobs are left as they
+ * are.  Host pointers.
  * slaq_load_histories stores each job in its own max_hist-long ring, so later appends
  * extend the window up to max_hist.  slaq_load_histories_packed keeps the rows packed
  * back to back on the device exactly as given (one cudaMalloc of the total size, which
  * replaces any earlier packed load - jobs of an earlier packed load that are not listed
- * again become inactive): a job loaded this way keeps a window of the length it was loaded with,
- * later appends overwrite its oldest point.
- * Errors: SLAQ_E_ARG, SLAQ_E_RANGE, SLAQ_E_NONFINITE, SLAQ_E_NOMEM, SLAQ_E_CUDA.
+ * again lose their storage with it: they become inactive and forget everything, as after
+ * slaq_remove_jobs): a job loaded this way keeps a window of the length it was loaded
+ * with, later appends overwrite its oldest point.
+ * Errors: SLAQ_E_ARG, SLAQ_E_RANGE, SLAQ_E_NONFINITE, SLAQ_E_NOMEM (the handle is as it
+ * was before the call), SLAQ_E_CUDA.
  */
 int slaq_load_histories(slaq_t* h, int32_t n_jobs, const int32_t* job_ids, const int64_t* offsets,
                         const double* losses, const int64_t* k_last, const double* m_seen);

@@ -288,6 +288,27 @@ int check_device_errors(slaq_handle* h) {
     return SLAQ_OK;
 }
 
+// Device scratch for calls that move caller data of a size unknown at creation (a bulk load into
+// rings, the normalisation export): owned by the handle, grown when a call needs more, kept for
+// the next call, released by slaq_destroy.  The stream must be idle when it grows.
+int ensure_call_buffer(slaq_handle* h, size_t bytes, void** out) {
+    if (bytes > h->call_buf_bytes) {
+        CK(cudaStreamSynchronize(h->stream), "sync before growing the call buffer");
+        if (h->call_buf) cudaFree(h->call_buf);
+        h->call_buf = nullptr;
+        h->call_buf_bytes = 0;
+        const size_t want = (bytes + kAlign - 1) / kAlign * kAlign;
+        const cudaError_t e = cudaMalloc(&h->call_buf, want);
+        if (e != cudaSuccess) {
+            h->call_buf = nullptr;
+            return fail(h, SLAQ_E_NOMEM, std::string("cudaMalloc of the call buffer: ") + cudaGetErrorString(e));
+        }
+        h->call_buf_bytes = want;
+    }
+    *out = h->call_buf;
+    return SLAQ_OK;
+}
+
 int create_common(slaq_handle* h, int32_t max_jobs, int32_t max_hist, int32_t cap, void* ws, size_t bytes) {
     h->max_jobs = max_jobs;
     h->max_hist = max_hist;
@@ -397,45 +418,52 @@ int do_load(slaq_handle* h, int32_t n, const int32_t* ids, const int64_t* offset
                 return fail(h, SLAQ_E_NONFINITE, "m_seen must be a number below +infinity");
     cudaStream_t st = h->stream;
     double* d_src = nullptr;
+    double* old_pool = nullptr;
     if (packed) {
+        // The new pool is allocated before anything changes, so a failed allocation leaves the handle
+        // as it was.  Jobs of the old pool that are listed again are re-pointed by the load kernel and
+        // keep their time sums, time law and core count; those that are not listed lose their
+        // storage with the old pool and are reset to inactive.
+        double* new_pool = nullptr;
+        if (total > 0) {
+            const cudaError_t e = cudaMalloc(&new_pool, sizeof(double) * (size_t)total);
+            if (e != cudaSuccess)
+                return fail(h, SLAQ_E_NOMEM, std::string("cudaMalloc of the packed pool: ") + cudaGetErrorString(e));
+        }
         if (h->packed_pool) {
-            // jobs still stored in the old pool lose their storage with it: deactivate them first
-            std::vector<int32_t> stale;
+            std::vector<int32_t> gone;
             for (int32_t j = 0; j < h->max_jobs; ++j)
-                if (h->in_packed[j]) stale.push_back(j);
-            const int32_t m = (int32_t)stale.size();
+                if (h->in_packed[j] && h->stamp[j] != h->stamp_epoch) gone.push_back(j);   // check_ids stamped the listed ids
+            const int32_t m = (int32_t)gone.size();
             if (m > 0) {
-                CK(cudaMemcpyAsync(h->stage.ids, stale.data(), sizeof(int32_t) * m, cudaMemcpyHostToDevice, st),
-                   "copy job ids");
-                init_jobs_kernel<<<(m + 255) / 256, 256, 0, st>>>(h->job, h->fit, h->ring_pool, h->max_jobs, h->max_hist,
-                                                                  h->stage.ids, m, h->alloc, h->reduction);
-                CK(cudaGetLastError(), "release kernel");
-            }
-            CK(cudaStreamSynchronize(st), "sync before releasing the packed pool");
-            for (int32_t j : stale) {
-                h->in_packed[j] = 0;
-                if (h->active[j]) {
-                    h->active[j] = 0;
-                    h->n_active -= 1;
+                cudaError_t e = cudaMemcpyAsync(h->stage.ids, gone.data(), sizeof(int32_t) * m, cudaMemcpyHostToDevice, st);
+                if (e == cudaSuccess) {
+                    init_jobs_kernel<<<(m + 255) / 256, 256, 0, st>>>(h->job, h->fit, h->ring_pool, h->max_jobs,
+                                                                      h->max_hist, h->stage.ids, m, h->alloc, h->reduction);
+                    e = cudaGetLastError();
+                }
+                if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // `gone` is read by the copy until here
+                if (e != cudaSuccess) {
+                    cudaFree(new_pool);
+                    return cuda_fail(h, e, "release jobs of the earlier packed load");
+                }
+                for (int32_t j : gone) {
+                    h->in_packed[j] = 0;
+                    if (h->active[j]) {
+                        h->active[j] = 0;
+                        h->n_active -= 1;
+                    }
                 }
             }
-            CK(cudaFree(h->packed_pool), "cudaFree packed pool");
-            h->packed_pool = nullptr;
-            h->packed_len = 0;
+            old_pool = h->packed_pool;   // still referenced by the re-listed jobs until the load kernel has run
         }
-        if (total > 0) {
-            const cudaError_t e = cudaMalloc(&h->packed_pool, sizeof(double) * (size_t)total);
-            if (e != cudaSuccess) {
-                h->packed_pool = nullptr;
-                return fail(h, SLAQ_E_NOMEM, std::string("cudaMalloc of the packed pool: ") + cudaGetErrorString(e));
-            }
-            h->packed_len = (size_t)total;
-        }
-        d_src = h->packed_pool;
+        h->packed_pool = new_pool;
+        h->packed_len = (size_t)total;
+        d_src = new_pool;
     } else if (total > 0) {
-        const cudaError_t e = cudaMalloc(&d_src, sizeof(double) * (size_t)total);
-        if (e != cudaSuccess)
-            return fail(h, SLAQ_E_NOMEM, std::string("cudaMalloc of the load buffer: ") + cudaGetErrorString(e));
+        void* buf = nullptr;
+        if (const int rc_buf = ensure_call_buffer(h, sizeof(double) * (size_t)total, &buf)) return rc_buf;
+        d_src = static_cast<double*>(buf);
     }
     int status = SLAQ_OK;
     {
@@ -459,7 +487,7 @@ int do_load(slaq_handle* h, int32_t n, const int32_t* ids, const int64_t* offset
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // `rel` and the caller's buffers are free again
         if (e != cudaSuccess) status = cuda_fail(h, e, "bulk load");
     }
-    if (!packed && d_src) cudaFree(d_src);
+    if (old_pool) cudaFree(old_pool);   // the stream is idle: nothing points into the old pool any more
     if (status) return status;
     for (int32_t i = 0; i < n; ++i) {
         const bool now = offsets[i + 1] > offsets[i];
@@ -632,6 +660,7 @@ int slaq_destroy(slaq_t* h) {
     if (h->graph_exec) cudaGraphExecDestroy(h->graph_exec);
     if (h->capture_stream) cudaStreamDestroy(h->capture_stream);
     if (h->packed_pool) cudaFree(h->packed_pool);
+    if (h->call_buf) cudaFree(h->call_buf);
     if (h->owns_ws && h->ws) cudaFree(h->ws);
     delete h;
     return SLAQ_OK;
@@ -927,34 +956,30 @@ int slaq_get_normalised(slaq_t* h, int32_t n, const int32_t* job_ids, int64_t ca
     const int64_t total = offs[n];
     if ((out_changes || out_levels) && total > capacity) return fail(h, SLAQ_E_RANGE, "output capacity too small");
     if (out_offsets) std::memcpy(out_offsets, offs.data(), sizeof(int64_t) * (n + 1));
-    double *d_changes = nullptr, *d_levels = nullptr, *d_largest = nullptr;
+    // one handle-owned buffer: [n] largest, then [total] changes and [total] levels
+    void* buf = nullptr;
+    const size_t n_pad = ((size_t)n + 31) / 32 * 32;
+    if ((rc = ensure_call_buffer(h, sizeof(double) * (n_pad + 2 * (size_t)total), &buf))) return rc;
+    double* d_largest = static_cast<double*>(buf);
+    double* d_changes = total > 0 ? d_largest + n_pad : nullptr;
+    double* d_levels = total > 0 ? d_changes + total : nullptr;
     int status = SLAQ_OK;
-    cudaError_t e = cudaMalloc(&d_largest, sizeof(double) * n);
-    if (e == cudaSuccess && total > 0) e = cudaMalloc(&d_changes, sizeof(double) * (size_t)total);
-    if (e == cudaSuccess && total > 0) e = cudaMalloc(&d_levels, sizeof(double) * (size_t)total);
-    if (e != cudaSuccess) {
-        status = fail(h, SLAQ_E_NOMEM, std::string("cudaMalloc of the export buffers: ") + cudaGetErrorString(e));
-    } else {
-        e = cudaMemcpyAsync(h->stage.ids, job_ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st);
-        if (e == cudaSuccess)
-            e = cudaMemcpyAsync(h->stage.offsets, offs.data(), sizeof(int64_t) * (n + 1), cudaMemcpyHostToDevice, st);
-        if (e == cudaSuccess && launch_normalise_export(h, n, h->stage.offsets, d_changes, d_levels, d_largest) < 0)
-            status = SLAQ_E_CUDA;
-        if (e == cudaSuccess && status == SLAQ_OK) {
-            if (out_changes && total > 0)
-                e = cudaMemcpyAsync(out_changes, d_changes, sizeof(double) * (size_t)total, cudaMemcpyDeviceToHost, st);
-            if (e == cudaSuccess && out_levels && total > 0)
-                e = cudaMemcpyAsync(out_levels, d_levels, sizeof(double) * (size_t)total, cudaMemcpyDeviceToHost, st);
-            if (e == cudaSuccess && out_largest)
-                e = cudaMemcpyAsync(out_largest, d_largest, sizeof(double) * n, cudaMemcpyDeviceToHost, st);
-        }
-        const cudaError_t e2 = cudaStreamSynchronize(st);
-        if (e == cudaSuccess) e = e2;
-        if (e != cudaSuccess) status = cuda_fail(h, e, "normalised export");
+    cudaError_t e = cudaMemcpyAsync(h->stage.ids, job_ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(h->stage.offsets, offs.data(), sizeof(int64_t) * (n + 1), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && launch_normalise_export(h, n, h->stage.offsets, d_changes, d_levels, d_largest) < 0)
+        status = SLAQ_E_CUDA;
+    if (e == cudaSuccess && status == SLAQ_OK) {
+        if (out_changes && total > 0)
+            e = cudaMemcpyAsync(out_changes, d_changes, sizeof(double) * (size_t)total, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess && out_levels && total > 0)
+            e = cudaMemcpyAsync(out_levels, d_levels, sizeof(double) * (size_t)total, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess && out_largest)
+            e = cudaMemcpyAsync(out_largest, d_largest, sizeof(double) * n, cudaMemcpyDeviceToHost, st);
     }
-    cudaFree(d_changes);
-    cudaFree(d_levels);
-    cudaFree(d_largest);
+    const cudaError_t e2 = cudaStreamSynchronize(st);
+    if (e == cudaSuccess) e = e2;
+    if (e != cudaSuccess) status = cuda_fail(h, e, "normalised export");
     return status;
 }
 

@@ -109,6 +109,8 @@ struct slaq_handle {
     double* ring_pool = nullptr;      // [max_jobs][max_hist]
     double* packed_pool = nullptr;    // separate allocation made by slaq_load_histories_packed
     size_t packed_len = 0;
+    void* call_buf = nullptr;         // scratch of calls that move caller data of any size (grown on demand, kept)
+    size_t call_buf_bytes = 0;
     double* wtab = nullptr;           // gamma^m, m = 0..max_hist-1
     double wtab_gamma = -1.0;
     slaq::JobArrays job;

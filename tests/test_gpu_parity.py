@@ -384,6 +384,55 @@ def test_other_seeds(slaq, oracle_mod):
                       wl.max_cores_per_job)
 
 
+# ---------------------------------------------------------------- a packed load replaced by another
+def test_a_second_packed_load_keeps_time_laws_and_drops_unlisted_jobs(slaq, oracle_mod):
+    """Jobs listed again in a second packed load keep their time law, time sums and core count (a bulk load
+    replaces histories only); jobs of the first load that are not listed again become inactive."""
+    wl = make_workload(2, n_jobs=900)
+    J, cap = wl.n_jobs, wl.max_cores_per_job
+    ids = np.arange(J, dtype=np.int32)
+    sched = slaq.Scheduler(J, wl.max_hist, cap)
+    fixed = ids[: J // 2]                                    # a fixed law for the first half
+    sched.set_time_model(fixed, wl.s[fixed], wl.w[fixed])
+    sched.load_histories(ids, wl.offsets, wl.losses, wl.k_last, wl.m_seen, packed=True)
+    sampled = ids[J // 2:]                                   # time samples for the second half: 2 and then 4 cores
+    for n_cores in (2, 4):
+        k = wl.k_last[sampled] + (1 if n_cores == 2 else 2)
+        sched.append_losses(sampled, wl.losses[wl.offsets[sampled + 1] - 1] * 0.99,
+                            wl.s[sampled] + wl.w[sampled] / n_cores, np.full(sampled.size, n_cores, np.int32))
+    s_before, w_before = sched.get_time_model()
+    assert np.isfinite(s_before).all() and np.isfinite(w_before).all()
+    # second load: every third job is left out, the others get another seed's histories
+    other = make_workload(2, n_jobs=J, seed_offset=4)
+    keep = ids[ids % 3 != 0]
+    H = other.hist_len[keep]
+    off = np.concatenate([[0], np.cumsum(H)]).astype(np.int64)
+    ls = np.concatenate([other.history(j) for j in keep])
+    sched.load_histories(keep, off, ls, other.k_last[keep], other.m_seen[keep], packed=True)
+    assert sched.get_active_count() == keep.size
+    s_after, w_after = sched.get_time_model()
+    np.testing.assert_array_equal(s_after[keep], s_before[keep])
+    np.testing.assert_array_equal(w_after[keep], w_before[keep])
+    gone = ids[ids % 3 == 0]
+    assert np.isnan(s_after[gone]).all()
+    C = 4 * keep.size
+    alloc, rc = sched.schedule(wl.epoch_seconds, C)
+    pred = sched.get_predictions()
+    assert rc == 0 and (alloc[gone] == 0).all() and (pred["status"][gone] == slaq.JOB_INACTIVE).all()
+    assert (pred["status"][keep] != slaq.JOB_NO_TIME).all()
+    # oracle on the same state: all J ids, the dropped ones with empty histories
+    H_all = np.zeros(J, np.int64)
+    H_all[keep] = H
+    off_all = np.concatenate([[0], np.cumsum(H_all)]).astype(np.int64)
+    m_all = np.full(J, -np.inf)
+    m_all[keep] = other.m_seen[keep]
+    ref = oracle_mod.schedule(off_all, ls, m_all, s_before, w_before, wl.epoch_seconds, C, cap)
+    compare_epoch(alloc, pred, ref, C, cap)
+    # a third load into rings releases the packed pool's jobs that it lists, and later appends extend them
+    sched.load_histories(keep[:10], off[:11], ls[:off[10]], other.k_last[keep[:10]], other.m_seen[keep[:10]])
+    assert sched.get_active_count() == keep.size
+
+
 # ---------------------------------------------------------------- four or more points, yet no curve can be started
 @pytest.mark.parametrize("cluster_jobs", [0, 10_000_000])
 @pytest.mark.parametrize("packed", [False, True])
