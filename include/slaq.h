@@ -277,6 +277,17 @@ int slaq_allocate_only(slaq_t* h, int64_t total_cores, int32_t* out_alloc);
 int slaq_get_stats(slaq_t* h, slaq_stats* out);
 
 /*
+ * Diagnostic (the paper has no counterpart).  In a library built with -DSLAQ_PHASE_CLOCKS
+ * (paper_1802_04819_b200.build.build_variant("clocks")) the fit kernel adds up, over all its
+ * warps, the SM cycles a warp spent in each phase of the last epoch's fit; out_cycles (host,
+ * 6 entries) receives them: 0 staging and normalisation, 1 first guesses and the sweep at
+ * the starting points, 2 solver steps of the trials, 3 sweeps at the trial points with
+ * their reductions and accept/reject, 4 winner and record, 5 work queue and statistics.
+ * The ordinary library carries no clocks and reports zeros.
+ */
+int slaq_get_fit_phase_cycles(slaq_t* h, int64_t* out_cycles);
+
+/*
  * One cluster sharded over several GPUs.  The jobs of ONE cluster are split into contiguous
  * blocks of job ids, block r on GPU r (shard r: its own handle, local ids 0..max_jobs-1 in global
  * order), and all shards share the cluster's cores.  Normalise, fit and gains need no exchange.  The

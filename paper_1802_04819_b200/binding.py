@@ -7,7 +7,7 @@ from ctypes import POINTER, c_double, c_float, c_int, c_int8, c_int32, c_int64, 
 
 import numpy as np
 
-from .build import LIB
+from .build import LIB, variant_path
 
 JOB_INACTIVE, JOB_FITTED, JOB_SHORT, JOB_NEW, JOB_FIT_FAILED, JOB_FLAT, JOB_NONFINITE, JOB_NO_TIME = -1, 0, 1, 2, 3, 4, 5, 6
 P_GAMMA, P_LM_TRIALS, P_MAX_CORES_PER_JOB, P_MIN_FIT_POINTS, P_FIT_SLICE_BYTES, P_WARM_START = 1, 2, 3, 4, 5, 6
@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = [
     "slaq_load_histories_packed", "slaq_set_time_model", "slaq_remove_jobs", "slaq_schedule", "slaq_schedule_device",
     "slaq_get_predictions", "slaq_get_normalised", "slaq_get_time_model", "slaq_get_fit_state",
     "slaq_set_fit_state", "slaq_set_gains", "slaq_allocate_only",
-    "slaq_get_stats", "slaq_allocate_static", "slaq_get_active_count", "slaq_shard_predict", "slaq_shard_histogram",
+    "slaq_get_stats", "slaq_get_fit_phase_cycles", "slaq_allocate_static", "slaq_get_active_count", "slaq_shard_predict", "slaq_shard_histogram",
     "slaq_shard_pick", "slaq_shard_pass", "slaq_shard_count", "slaq_shard_finalise",
 ]
 
@@ -44,17 +44,18 @@ class SlaqError(RuntimeError):
         self.code = code
 
 
-_lib = None
+_libs = {}
 
 
-def load_library():
-    """Load libslaq.so (must have been built: ``python -m paper_1802_04819_b200.build``)."""
-    global _lib
-    if _lib is not None:
-        return _lib
-    if not LIB.exists():
-        raise FileNotFoundError(f"{LIB} is missing: build the CUDA library first (paper_1802_04819_b200.build())")
-    lib = ctypes.CDLL(str(LIB))
+def load_library(variant: str | None = None):
+    """Load libslaq.so (must have been built: ``python -m paper_1802_04819_b200.build``), or with
+    ``variant`` an instrumented build of the same sources (``build.build_variant(variant)``)."""
+    if variant in _libs:
+        return _libs[variant]
+    path = LIB if variant is None else variant_path(variant)
+    if not path.exists():
+        raise FileNotFoundError(f"{path} is missing: build the CUDA library first (paper_1802_04819_b200.build())")
+    lib = ctypes.CDLL(str(path))
     vp = c_void_p
     sig = {
         "slaq_create": (c_int, [c_int32, c_int32, POINTER(vp)]),
@@ -81,6 +82,7 @@ def load_library():
         "slaq_set_gains": (c_int, [vp, vp]),
         "slaq_allocate_only": (c_int, [vp, c_int64, vp]),
         "slaq_get_stats": (c_int, [vp, POINTER(Stats)]),
+        "slaq_get_fit_phase_cycles": (c_int, [vp, vp]),
         "slaq_allocate_static": (c_int, [vp, c_int32, c_int32, c_int64, vp, vp, vp]),
         "slaq_get_active_count": (c_int, [vp, POINTER(c_int32)]),
         "slaq_shard_predict": (c_int, [vp, c_double, c_int32]),
@@ -93,7 +95,7 @@ def load_library():
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
         fn.restype, fn.argtypes = res, args
-    _lib = lib
+    _libs[variant] = lib
     return lib
 
 
@@ -135,10 +137,12 @@ def _ptr(a):
 class Scheduler:
     """One scheduler handle.  Methods mirror the C calls of the same name (without ``slaq_``)."""
 
-    def __init__(self, max_jobs: int, max_hist: int, max_cores_per_job: int = 64, workspace=None, stream=None):
+    def __init__(self, max_jobs: int, max_hist: int, max_cores_per_job: int = 64, workspace=None, stream=None,
+                 variant: str | None = None):
         """``workspace``: optional torch uint8 CUDA tensor of at least ``workspace_bytes(...)`` bytes
-        (device memory owned by the caller); ``stream``: optional ``torch.cuda.Stream``."""
-        self._lib = load_library()
+        (device memory owned by the caller); ``stream``: optional ``torch.cuda.Stream``;
+        ``variant``: an instrumented build of the library (``build.VARIANTS``) instead of libslaq.so."""
+        self._lib = load_library(variant)
         self._h = c_void_p()
         self.max_jobs, self.max_hist, self.max_cores_per_job = int(max_jobs), int(max_hist), int(max_cores_per_job)
         self._workspace = workspace
@@ -305,6 +309,12 @@ class Scheduler:
     def shard_finalise(self, ties_before: int):
         out = np.empty(self.max_jobs, np.int32)
         self._check(self._lib.slaq_shard_finalise(self._h, int(ties_before), _ptr(out)))
+        return out
+
+    def get_fit_phase_cycles(self):
+        """SM cycles the fit kernel's warps spent per phase (zeros unless the "clocks" variant is loaded)."""
+        out = np.zeros(6, np.int64)
+        self._check(self._lib.slaq_get_fit_phase_cycles(self._h, _ptr(out)))
         return out
 
     def get_stats(self) -> Stats:

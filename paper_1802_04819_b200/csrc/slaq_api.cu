@@ -1037,6 +1037,16 @@ int slaq_set_fit_state(slaq_t* h, const double* params, const uint8_t* mask, con
     return SLAQ_OK;
 }
 
+int slaq_get_fit_phase_cycles(slaq_t* h, int64_t* out_cycles) {
+    if (!h || !out_cycles) return SLAQ_E_ARG;
+    if (!h->have_epoch) return fail(h, SLAQ_E_ARG, "no epoch has been scheduled yet");
+    long long counters[16];
+    CK(cudaMemcpyAsync(counters, h->scratch.counters, sizeof counters, cudaMemcpyDeviceToHost, h->stream), "copy counters");
+    CK(cudaStreamSynchronize(h->stream), "copy phase cycles");
+    for (int i = 0; i < 6; ++i) out_cycles[i] = counters[8 + i];
+    return SLAQ_OK;
+}
+
 int slaq_get_stats(slaq_t* h, slaq_stats* out) {
     if (!h || !out) return SLAQ_E_ARG;
     if (!h->have_epoch) return fail(h, SLAQ_E_ARG, "no epoch has been scheduled yet");

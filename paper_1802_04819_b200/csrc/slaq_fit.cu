@@ -29,6 +29,21 @@ namespace slaq {
 
 namespace {
 
+// Phase clocks (only in a library built with -DSLAQ_PHASE_CLOCKS): lane 0 of every warp adds up the
+// SM cycles it spends in each phase of the fit; the totals go to counters[8..13].
+#ifdef SLAQ_PHASE_CLOCKS
+#define SLAQ_PHASE_DECL long long ph_[6] = {0, 0, 0, 0, 0, 0}, ph_t_ = clock64()
+#define SLAQ_PHASE(i)                      \
+    do {                                   \
+        const long long now_ = clock64();  \
+        ph_[i] += now_ - ph_t_;            \
+        ph_t_ = now_;                      \
+    } while (0)
+#else
+#define SLAQ_PHASE_DECL
+#define SLAQ_PHASE(i)
+#endif
+
 constexpr int kMaxWarpsPerBlock = 16;          // one block per SM: its warps share one copy of the weight table
 constexpr size_t kSmemLimit = 226 * 1024;   // shared memory one block may use on sm_100, less the static part
 constexpr double kLambda0 = 1e-3, kLambdaMin = 1e-5, kLambdaMax = 1e12;
@@ -556,10 +571,12 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
 
     long long n_points = 0, n_sweep_points = 0;
     int n_fit = 0, n_sub = 0, n_exp = 0, n_fallback = 0;
+    SLAQ_PHASE_DECL;
     for (;;) {
         int slot = 0;
         if (lane == 0) slot = (int)atomicAdd(queue, 1u);
         slot = __shfl_sync(kFull, slot, 0);
+        SLAQ_PHASE(5);   // between jobs: statistics, record tail, queue
         if (slot >= slot_base[cls.n]) break;
         int c = 0;
         while (slot >= slot_base[c + 1]) ++c;
@@ -579,6 +596,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         __syncwarp();
         const double m_seen = j >= 0 ? job.m_seen[j] : -CUDART_INF;
         const Normalised nz = normalise_window(S, H, k_all, m_seen, min_fit_points, nullptr);
+        SLAQ_PHASE(0);   // staging and normalisation
 
         int status = nz.status, family = -1;
         double p_out[4] = {CUDART_NAN, CUDART_NAN, CUDART_NAN, CUDART_NAN};
@@ -641,6 +659,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
             F.has_trial = false;
             F.predicted = 0.0;
             park(S, sums, true);
+            SLAQ_PHASE(1);   // first guesses and the sweep at the starting points
             for (int t = 0; t < lm_trials; ++t) {
                 if (!__any_sync(kFull, !F.done)) break;
                 double trial[4] = {0.0, 0.0, 0.0, 0.0};
@@ -651,6 +670,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
                     prepare_trial(F, fam, A, gr, !F.done, mom.swy2, trial);
                 }
                 const unsigned trying = __ballot_sync(kFull, F.has_trial);
+                SLAQ_PHASE(2);   // solver step of a trial
                 if (!trying) continue;
 #pragma unroll
                 for (int a = 0; a < 4; ++a) {   // each lane of a pair fetches the other family's trial point
@@ -659,6 +679,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
                 }
                 sweep(S, fam, H, k_all, inv_span, pI, (trying >> even) & 1u, pII, (trying >> oddl) & 1u, sums);
                 park(S, sums, finish_trial(F, trial, sums.usable, sums.v[fam ? 8 : 12]));
+                SLAQ_PHASE(3);   // sweep at the trial points, reduction, accept or reject
             }
             // both results of the job, in every lane
             const double S_I = __shfl_sync(kFull, F.S, even), S_II = __shfl_sync(kFull, F.S, oddl);
@@ -734,6 +755,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
             fit.span[j] = span;
         }
         __syncwarp();
+        SLAQ_PHASE(4);   // winner, fallback, the job's record
     }
     // per-warp totals of the statistics
     for (int o = 16; o > 0; o >>= 1) {
@@ -752,6 +774,10 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         atomicAdd((unsigned long long*)&counters[4], (unsigned long long)n_exp);
         atomicAdd((unsigned long long*)&counters[5], (unsigned long long)n_fallback);
     }
+#ifdef SLAQ_PHASE_CLOCKS
+    if (lane == 0)
+        for (int i = 0; i < 6; ++i) atomicAdd((unsigned long long*)&counters[8 + i], (unsigned long long)ph_[i]);
+#endif
 }
 
 // Normalisation only, written out for inspection: same staging and scaling code as the fit,
