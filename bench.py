@@ -35,8 +35,9 @@ WARM_TRIALS = 5   # trials per epoch of the warm-started loop reported beside th
 FLOP_SWEEP_I, FLOP_SWEEP_II, FLOP_SETUP = 40.0, 25.0, 40.0
 FP64_LANES_PER_SM = 64          # fp64 FMA lanes per SM on B200
 # The sweep of the fit issues 46 fp64 instructions per point: 92 cycles per warp row if each took 2, but the 15
-# fused multiply-adds on three different registers take 3 (measured with paper_1802_04819_b200/fp64_issue_probe)
+# fused multiply-adds on three different registers take 3 (measured with bench_probes/fp64_issue_probe)
 SWEEP_ISSUE_CYCLES_IDEAL, SWEEP_ISSUE_CYCLES_MEASURED_RATES = 92.0, 107.0
+MIN_TIMED_SECONDS = 1.0   # the block of --steps steps is repeated until the timed region is at least this long
 # DRAM bytes per stored loss moved by the fit kernel (ncu: dram__bytes_read.sum + dram__bytes_write.sum =
 # 165.72 MB + 13.70 MB on a 20,068,408-loss cut of this workload; traffic grows with the stored losses)
 NCU_FIT_DRAM_BYTES_PER_LOSS = (165.72e6 + 13.70e6) / 20_068_408
@@ -106,6 +107,27 @@ def measured_peaks():
     if path.exists():
         return json.loads(path.read_text()), "measured"
     return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def measured_fp64_peak():
+    """Best fused multiply-add rate of the fp64 pipe on this GPU, measured now with bench_probes/fp64_issue_probe
+    (12 independent accumulators per thread, 16 warps per SM).  Returns (TFLOP/s, note) or (None, why)."""
+    exe = ROOT / "bench_probes" / "fp64_issue_probe"
+    try:
+        if not exe.exists():
+            sys.path.insert(0, str(ROOT / "bench_probes"))
+            import build as probe_build   # bench_probes/build.py
+            probe_build.build_probes()
+        out = subprocess.run([str(exe)], capture_output=True, text=True, timeout=120, check=True).stdout
+    except (OSError, subprocess.SubprocessError, ImportError) as err:
+        return None, f"fp64_issue_probe did not run: {err}"
+    best = 0.0
+    for row in out.splitlines():
+        cols = row.split()
+        if len(cols) == 4 and cols[0].startswith("fma"):
+            best = max(best, float(cols[3]))
+    return (best, "best fused multiply-add rate of bench_probes/fp64_issue_probe, run before the timed region") \
+        if best > 0 else (None, "fp64_issue_probe printed no rate")
 
 
 def host_threads() -> int:
@@ -197,21 +219,36 @@ def run_gpu(args):
     H = wl.hist_len.astype(np.float64)
     fit_flops = float((H[fitted] * (FLOP_SWEEP_I * pred["evals"][fitted, 0] + FLOP_SWEEP_II * pred["evals"][fitted, 1]
                                     + FLOP_SETUP)).sum())
+    fp64_peak_measured, fp64_peak_note = measured_fp64_peak() if rank == 0 else (None, "")
     barrier()
+    # The timed block is exactly --steps epochs between a barrier + synchronise on both sides.  It is repeated
+    # until the region lasts MIN_TIMED_SECONDS (a clock excursion then shows in the sampled clocks and in the
+    # spread of the blocks); the reported step time is the median block's.
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    fit_ms, stage_ms, launches = [], [], 0
+    fit_ms, stage_ms, launches, block_ms = [], [], 0, []
     t_from = time.perf_counter()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        sched.schedule_device(wl.epoch_seconds, wl.total_cores, d_alloc)
-        st = sched.get_stats()                 # reads the library's own per-stage CUDA events (same stream)
-        fit_ms.append(st.ms_fit)
-        stage_ms.append((st.ms_fit, st.ms_gain, st.ms_alloc))
-        launches += st.launches
-    ev1.record(stream)
-    barrier()
+    while True:
+        barrier()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            sched.schedule_device(wl.epoch_seconds, wl.total_cores, d_alloc)
+            st = sched.get_stats()                 # reads the library's own per-stage CUDA events (same stream)
+            fit_ms.append(st.ms_fit)
+            stage_ms.append((st.ms_fit, st.ms_gain, st.ms_alloc))
+            if not block_ms:
+                launches += st.launches            # kernels of one block of --steps steps
+        ev1.record(stream)
+        barrier()
+        block_ms.append(ev0.elapsed_time(ev1))
+        enough = time.perf_counter() - t_from >= MIN_TIMED_SECONDS
+        if world > 1:                              # every rank runs the same number of blocks
+            flag = torch.tensor([1.0 if enough else 0.0], device="cuda")
+            dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+            enough = bool(flag.item() > 0)
+        if enough or len(block_ms) >= 1000:
+            break
     clocks = sampler.stop(t_from, time.perf_counter())
-    ms_step = ev0.elapsed_time(ev1) / args.steps
+    ms_step = float(np.median(block_ms)) / args.steps
     alloc_dev = d_alloc.cpu().numpy()
     assert int(alloc_dev.sum()) == wl.total_cores
 
@@ -221,7 +258,7 @@ def run_gpu(args):
     h_ids, h_time = pin(J, torch.int32), pin(J, torch.float64)
     h_alloc = pin(J, torch.int32)
     h_ids[:] = ids
-    e2e_steps = max(1, min(args.steps, 10))
+    e2e_steps = max(1, args.steps)
     # every step's input (one new loss per job and the seconds its iteration took) waits in pinned host memory
     feeds = []
     for s in range(2 * (args.warmup + e2e_steps)):
@@ -284,6 +321,11 @@ def run_gpu(args):
                        "l2": f"inputs larger than L2 ({int(wl.offsets[-1]) * 8 / 1e6:.0f} MB of losses read per step)",
                        "parallelism": f"{world} independent cluster partition(s), one per GPU"},
             "clocks": clocks,
+            "timed_blocks": {"blocks": len(block_ms), "steps_per_block": args.steps, "ms_per_step_median": ms_step,
+                             "ms_per_step_min": float(np.min(block_ms)) / args.steps,
+                             "ms_per_step_max": float(np.max(block_ms)) / args.steps,
+                             "what": "the block of --steps epochs, repeated until the timed region lasts one second; "
+                                     "value and ms_per_step come from the median block"},
             "e2e": {"value": whole_job_rate(J, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": int(J * (4 + 8 + 8)), "d2h_bytes_per_step": int(J * 4 + 4),
                     "steps": e2e_steps,
@@ -306,7 +348,10 @@ def run_gpu(args):
                          "issue_bound_note": "fp64 instructions on three different registers issue every 3 cycles, "
                                              "not 2: what a loop of nothing but sweeps could reach",
                          "peak_is": f"{sm_count} SMs x {FP64_LANES_PER_SM} fp64 FMA lanes x 2 x {sm_max:.0f} MHz "
-                                    f"(clock from MEASURED_PEAKS.json: {peak_kind})"},
+                                    f"(clock from MEASURED_PEAKS.json: {peak_kind}; that file holds no fp64 figure)",
+                         "peak_measured": fp64_peak_measured,
+                         "frac_of_peak_measured": achieved / fp64_peak_measured if fp64_peak_measured else None,
+                         "peak_measured_is": fp64_peak_note},
         }
         if args.cpu_baseline:
             import oracle

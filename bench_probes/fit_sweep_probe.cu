@@ -100,9 +100,14 @@ int main(int argc, char** argv) {
     cudaEventCreate(&e1);
     printf("%d SMs, %d sweeps per warp, both families in every sweep\n", sm_count, n_sweeps);
     printf("%4s %5s %9s %22s %20s %14s\n", "L", "rows", "warps/SM", "cycles/warp row/SMSP", "of 92 (2-cycle issue)", "ms");
-    const int cases[][2] = {{2, 41}, {4, 51}, {8, 51}, {16, 51}, {32, 31}};
+    // rows a slice holds at L lanes per job: (slice - parked sums of its 32/L jobs) / 32 - 1 spare row, as in the library
+    const int cases[][2] = {{2, 41}, {4, 47}, {8, 50}, {16, 51}, {32, 31}};
     std::vector<long long> cyc(sm_count);
     for (const auto& c : cases) {
+        if (slaq::kParked * (64 / c[0]) + (c[1] + 1) * 32 > kSliceDoubles) {
+            fprintf(stderr, "fit_sweep_probe: %d rows at L = %d do not fit a slice\n", c[1], c[0]);
+            return 1;
+        }
         for (int warps = 4; warps <= kWarps; warps += 4) {
             double best_cycles = 1e300;
             float best_ms = 1e30f;
@@ -110,8 +115,9 @@ int main(int argc, char** argv) {
                 cudaEventRecord(e0);
                 sweep_loop_kernel<<<sm_count, kWarps * 32, smem>>>(d_tab, c[0], c[1], n_sweeps, warps, d_out, d_cycles);
                 cudaEventRecord(e1);
-                if (cudaDeviceSynchronize() != cudaSuccess) {
-                    fprintf(stderr, "fit_sweep_probe: kernel failed\n");
+                const cudaError_t err = cudaDeviceSynchronize();
+                if (err != cudaSuccess) {
+                    fprintf(stderr, "fit_sweep_probe: kernel failed: %s\n", cudaGetErrorString(err));
                     return 1;
                 }
                 float ms = 0.f;
