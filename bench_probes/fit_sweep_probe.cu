@@ -40,6 +40,10 @@ sweep_loop_kernel(const double* __restrict__ g_wtab, int L, int rows, int n_swee
     const int G = 32 / L;
     S.park = slice + 2 * (lane / L) + (lane & 1);
     S.y = slice + slaq::kParked * 2 * G;
+    S.slice = slice;
+    S.slice_len = kSliceDoubles;
+    S.wtab_len = kTable;
+    S.err_word = nullptr;
     const int H = rows * L;
     const double span = (double)(H - 1), inv_span = 1.0 / span;
     // a window that falls like 1/(a k^2 + b k + c) + d, newest point last, in normalised units

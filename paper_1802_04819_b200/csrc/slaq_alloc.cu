@@ -79,7 +79,8 @@ __device__ void pick_bin(const unsigned long long* hist, int pass, SelectState* 
 __global__ void __launch_bounds__(kSelectThreads)
 select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap,
                    int first_unit, int pass, unsigned long long* __restrict__ hist_all, SelectState* sel,
-                   unsigned int* ticket, int32_t* __restrict__ seg_lo, int32_t* __restrict__ seg_hi, int do_pick) {
+                   unsigned int* ticket, int32_t* __restrict__ seg_lo, int32_t* __restrict__ seg_hi, int do_pick,
+                   int32_t* err_word) {
     __shared__ unsigned int sh_hist[kRadixBins];
     __shared__ unsigned long long sh_scan[kSelectThreads + 1];
     __shared__ bool is_last;
@@ -103,6 +104,12 @@ select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ 
         if (live && pass > 1) {
             my_lo = seg_lo[mine];
             my_hi = seg_hi[mine];
+#ifdef SLAQ_DEBUG_BOUNDS
+            if (my_lo < first_unit - 1 || my_hi > cap || my_lo > my_hi) {   // not a segment of this row: skip it
+                if (err_word) atomicOr(err_word, kErrSegment);
+                my_lo = my_hi = first_unit - 1;
+            }
+#endif
         }
         unsigned todo = __ballot_sync(kFull, live && my_lo < my_hi);
         while (todo) {
@@ -115,12 +122,14 @@ select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ 
                 const int i = base + lane;
                 const bool in = i < hi;
                 unsigned long long key = 0;
-                if (in) key = keys[(size_t)j * cap + i];
+                if (in && index_ok((long long)j * cap + i, (long long)max_jobs * cap, kErrGain, err_word))
+                    key = keys[(size_t)j * cap + i];
                 const unsigned d_prev = (unsigned)(key >> prev_shift) & ((1u << prev_bits) - 1u);
                 const bool match = in && d_prev == prev_bin;
                 above += __popc(__ballot_sync(kFull, in && d_prev > prev_bin));
                 same += __popc(__ballot_sync(kFull, match));
-                if (match) atomicAdd(&sh_hist[(unsigned)(key >> shift) & ((1u << bits) - 1u)], 1u);
+                const unsigned bin = (unsigned)(key >> shift) & ((1u << bits) - 1u);
+                if (match && index_ok(bin, kRadixBins, kErrBin, err_word)) atomicAdd(&sh_hist[bin], 1u);
             }
             if (lane == r) {
                 my_lo = lo + above;
@@ -171,7 +180,7 @@ __global__ void init_select_kernel(SelectState* sel, long long want) {
 // Histogram of the first digit when the gain rows were not written by the gain kernel.
 __global__ void __launch_bounds__(kSelectThreads)
 first_hist_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap,
-                  int first_unit, unsigned long long* __restrict__ hist0) {
+                  int first_unit, unsigned long long* __restrict__ hist0, int32_t* err_word) {
     __shared__ unsigned int sh_hist[kRadixBins];
     for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) sh_hist[i] = 0;
     __syncthreads();
@@ -181,7 +190,8 @@ first_hist_kernel(const double* __restrict__ gain, const int32_t* __restrict__ c
     for (int j = blockIdx.x * (kSelectThreads / 32) + (threadIdx.x >> 5); j < max_jobs; j += warps_total) {
         if (count[j] <= 0) continue;
         for (int n = first_unit + lane; n <= cap; n += 32)
-            atomicAdd(&sh_hist[(unsigned)(keys[(size_t)j * cap + (n - 1)] >> (64 - kRadixBits))], 1u);
+            if (index_ok((long long)j * cap + (n - 1), (long long)max_jobs * cap, kErrGain, err_word))
+                atomicAdd(&sh_hist[(unsigned)(keys[(size_t)j * cap + (n - 1)] >> (64 - kRadixBits))], 1u);
     }
     __syncthreads();
     for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) {
@@ -197,7 +207,7 @@ first_hist_kernel(const double* __restrict__ gain, const int32_t* __restrict__ c
 __global__ void __launch_bounds__(256)
 count_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count, int max_jobs, int cap, int first_unit,
              const SelectState* __restrict__ sel, int32_t* __restrict__ gt, int32_t* __restrict__ eq,
-             long long* __restrict__ block_eq) {
+             long long* __restrict__ block_eq, int32_t* err_word) {
     __shared__ int sh_eq[8];
     const bool none_wanted = sel->done != 0;
     const unsigned long long tau = sel->prefix;
@@ -212,6 +222,12 @@ count_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count,
     if (live) {
         my_lo = gt[mine];    // segment [lo, hi) written by the last pass
         my_hi = eq[mine];
+#ifdef SLAQ_DEBUG_BOUNDS
+        if (my_lo < first_unit - 1 || my_hi > cap || my_lo > my_hi) {
+            if (err_word) atomicOr(err_word, kErrSegment);
+            my_lo = my_hi = first_unit - 1;
+        }
+#endif
     }
     int my_gt = live ? my_lo - (first_unit - 1) : 0, my_eq = 0;
     unsigned todo = __ballot_sync(kFull, live && my_lo < my_hi);
@@ -225,7 +241,8 @@ count_kernel(const double* __restrict__ gain, const int32_t* __restrict__ count,
             const int i = base + lane;
             const bool in = i < hi;
             unsigned long long key = 0;
-            if (in) key = keys[(size_t)j * cap + i];
+            if (in && index_ok((long long)j * cap + i, (long long)max_jobs * cap, kErrGain, err_word))
+                key = keys[(size_t)j * cap + i];
             const unsigned d = (unsigned)(key >> pass_shift(last)) & ((1u << pass_bits(last)) - 1u);
             above += __popc(__ballot_sync(kFull, in && d > last_bin));
             same += __popc(__ballot_sync(kFull, in && d == last_bin));
@@ -283,7 +300,7 @@ finalise_kernel(const double* __restrict__ gain, const int32_t* __restrict__ cou
                 const SelectState* __restrict__ sel, const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
                 const long long* __restrict__ block_prefix, int32_t* __restrict__ alloc, double* __restrict__ reduction,
                 int32_t* __restrict__ last_alloc, int32_t* __restrict__ out_alloc, long long* counters,
-                long long ties_before) {
+                long long ties_before, int32_t* err_word) {
     __shared__ long long sh_pre[kJobsPerBlock];
     __shared__ int sh_alloc[kJobsPerBlock];
     const int t = threadIdx.x;
@@ -307,6 +324,12 @@ finalise_kernel(const double* __restrict__ gain, const int32_t* __restrict__ cou
         take = take < 0 ? 0 : (take > my_eq ? my_eq : take);
         a = floor_units + gt[jt] + (int)take;
         ties_taken = take;
+#ifdef SLAQ_DEBUG_BOUNDS
+        if (a < 0 || a > cap) {   // an allocation outside 0..cap would read past the row below
+            if (err_word) atomicOr(err_word, kErrSegment);
+            a = a < 0 ? 0 : cap;
+        }
+#endif
     }
     sh_alloc[t] = a;
     if (jt < max_jobs) {
@@ -356,7 +379,8 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
     init_select_kernel<<<1, 1, 0, st>>>(h->scratch.sel, want);
     ++launches;
     if (!hist0_ready) {
-        first_hist_kernel<<<grid, kSelectThreads, 0, st>>>(h->gain, h->job.count, J, cap, first_unit, h->scratch.hist);
+        first_hist_kernel<<<grid, kSelectThreads, 0, st>>>(h->gain, h->job.count, J, cap, first_unit, h->scratch.hist,
+                                                          h->err_word);
         ++launches;
     }
     pick_first_kernel<<<1, kSelectThreads, 0, st>>>(h->scratch.hist, h->scratch.sel);
@@ -364,16 +388,16 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
     for (int pass = 1; pass < kRadixPasses; ++pass) {
         select_pass_kernel<<<grid, kSelectThreads, 0, st>>>(h->gain, h->job.count, J, cap, first_unit, pass,
                                                            h->scratch.hist, h->scratch.sel, h->scratch.ticket,
-                                                           h->scratch.gt, h->scratch.eq, 1);
+                                                           h->scratch.gt, h->scratch.eq, 1, h->err_word);
         ++launches;
     }
     const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
     count_kernel<<<blocks, 256, 0, st>>>(h->gain, h->job.count, J, cap, first_unit, h->scratch.sel, h->scratch.gt,
-                                         h->scratch.eq, h->scratch.block_eq);
+                                         h->scratch.eq, h->scratch.block_eq, h->err_word);
     scan_blocks_kernel<<<1, 1024, 0, st>>>(h->scratch.block_eq, blocks);
     finalise_kernel<<<blocks, 256, 0, st>>>(h->gain, h->job.count, J, cap, first_unit - 1, h->scratch.sel, h->scratch.gt,
                                             h->scratch.eq, h->scratch.block_eq, h->alloc, h->reduction,
-                                            h->job.last_alloc, d_out_alloc, h->scratch.counters, 0);
+                                            h->job.last_alloc, d_out_alloc, h->scratch.counters, 0, h->err_word);
     launches += 3;
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
@@ -413,7 +437,7 @@ int launch_shard_pass(slaq_handle* h, int pass, int first_unit) {
     if (grid > needed) grid = needed;
     select_pass_kernel<<<grid, kSelectThreads, 0, h->stream>>>(h->gain, h->job.count, J, h->max_cores, first_unit, pass,
                                                               h->scratch.hist, h->scratch.sel, h->scratch.ticket,
-                                                              h->scratch.gt, h->scratch.eq, 0);
+                                                              h->scratch.gt, h->scratch.eq, 0, h->err_word);
     return check_launch(h, "shard pass") ? -1 : 1;
 }
 
@@ -422,7 +446,7 @@ int launch_shard_count(slaq_handle* h, int first_unit, const long long** d_total
     const int J = h->max_jobs;
     const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
     count_kernel<<<blocks, 256, 0, h->stream>>>(h->gain, h->job.count, J, h->max_cores, first_unit, h->scratch.sel,
-                                                h->scratch.gt, h->scratch.eq, h->scratch.block_eq);
+                                                h->scratch.gt, h->scratch.eq, h->scratch.block_eq, h->err_word);
     scan_blocks_kernel<<<1, 1024, 0, h->stream>>>(h->scratch.block_eq, blocks);
     *d_total = h->scratch.block_eq + blocks;
     return check_launch(h, "shard count") ? -1 : 2;
@@ -434,7 +458,7 @@ int launch_shard_finalise(slaq_handle* h, int first_unit, long long ties_before,
     finalise_kernel<<<blocks, 256, 0, h->stream>>>(h->gain, h->job.count, J, h->max_cores, first_unit - 1, h->scratch.sel,
                                                    h->scratch.gt, h->scratch.eq, h->scratch.block_eq, h->alloc,
                                                    h->reduction, h->job.last_alloc, d_out_alloc, h->scratch.counters,
-                                                   ties_before);
+                                                   ties_before, h->err_word);
     return check_launch(h, "shard finalise") ? -1 : 1;
 }
 
@@ -518,18 +542,18 @@ extern "C" int slaq_allocate_static(const double* d_gain, int32_t n_jobs, int32_
     int grid = sm_count * 8;
     const int needed = (J + (kSelectThreads / 32) - 1) / (kSelectThreads / 32);
     if (grid > needed) grid = needed;
-    first_hist_kernel<<<grid, kSelectThreads, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, sc->hist);
+    first_hist_kernel<<<grid, kSelectThreads, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, sc->hist, nullptr);
     pick_first_kernel<<<1, kSelectThreads, 0, st>>>(sc->hist, &sc->sel);
     for (int pass = 1; pass < kRadixPasses; ++pass)
         select_pass_kernel<<<grid, kSelectThreads, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, pass,
-                                                           sc->hist, &sc->sel, sc->ticket, sc->gt, sc->eq, 1);
+                                                           sc->hist, &sc->sel, sc->ticket, sc->gt, sc->eq, 1, nullptr);
     const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
     count_kernel<<<blocks, 256, 0, st>>>(d_gain, sc->every_row_active, J, cap, first_unit, &sc->sel, sc->gt, sc->eq,
-                                         sc->block_eq);
+                                         sc->block_eq, nullptr);
     scan_blocks_kernel<<<1, 1024, 0, st>>>(sc->block_eq, blocks);
     finalise_kernel<<<blocks, 256, 0, st>>>(d_gain, sc->every_row_active, J, cap, floor_units, &sc->sel, sc->gt, sc->eq,
                                             sc->block_eq, d_out_alloc, d_out_reduction, sc->cores_now, nullptr,
-                                            sc->counters, 0);
+                                            sc->counters, 0, nullptr);
     if (cudaGetLastError() != cudaSuccess) return SLAQ_E_CUDA;
     if (total_cores < J) return SLAQ_W_OVERSUBSCRIBED;
     if (total_cores > (long long)J * cap) return SLAQ_W_UNDERFILLED;

@@ -86,6 +86,11 @@ size_t layout(slaq_handle* h, char* base, int32_t J, int32_t Hmax, int32_t cap) 
     int32_t* alloc = b.take<int32_t>(Js);
     double* reduction = b.take<double>(Js);
     int32_t* err_word = b.take<int32_t>(4);
+    job.max_jobs = J;
+    job.ring_lo = ring;
+    job.ring_hi = ring ? ring + Js * Hmax : nullptr;
+    job.packed_lo = job.packed_hi = nullptr;
+    job.err_word = err_word;
     if (h && base) {
         h->ring_pool = ring;
         h->wtab = wtab;
@@ -162,6 +167,16 @@ __global__ void append_kernel(JobArrays job, FitArrays fit, int max_jobs, int n,
     const int cap = job.cap[j];
     int head = job.head[j];
     const int count = job.count[j];
+#ifdef SLAQ_DEBUG_BOUNDS
+    {   // the ring lies inside one of the pools and the write position inside the ring
+        const bool in_ring = row >= job.ring_lo && row + cap <= job.ring_hi;
+        const bool in_packed = job.packed_lo && row >= job.packed_lo && row + cap <= job.packed_hi;
+        if (!(in_ring || in_packed) || head < 0 || head >= cap || count < 0 || count > cap) {
+            atomicOr(job.err_word, kErrStorage);
+            return;
+        }
+    }
+#endif
     if (count > 0) {
         const double prev = row[head == 0 ? cap - 1 : head - 1];
         const double seen = job.m_seen[j], drop = prev - loss;
@@ -217,7 +232,8 @@ __global__ void load_kernel(JobArrays job, FitArrays fit, double* ring, int max_
         row = const_cast<double*>(from);
         cap = (int)H;
     } else {
-        for (int i = lane; i < H; i += 32) row[i] = from[i];
+        for (int i = lane; i < H; i += 32)
+            if (index_ok((row - job.ring_lo) + i, job.ring_hi - job.ring_lo, kErrStorage, job.err_word)) row[i] = from[i];
     }
     if (lane == 0) {
         job.row[j] = row;
@@ -284,7 +300,17 @@ int check_device_errors(slaq_handle* h) {
     int32_t word = 0;
     CK(cudaMemcpyAsync(&word, h->err_word, sizeof word, cudaMemcpyDeviceToHost, h->stream), "read error word");
     CK(cudaStreamSynchronize(h->stream), "read error word");
-    if (word != 0) return fail(h, SLAQ_E_CUDA, "a kernel found inconsistent job storage (window longer than its ring)");
+    if (word != 0) {
+        std::string what = "a kernel found an inconsistency:";
+        if (word & kErrWindow) what += " a window longer than its ring;";
+        if (word & kErrStorage) what += " a position outside a job's storage;";
+        if (word & kErrShared) what += " an offset outside a shared-memory slice;";
+        if (word & kErrGain) what += " an entry outside the gain table;";
+        if (word & kErrSegment) what += " a candidate segment outside its row;";
+        if (word & kErrBin) what += " a histogram bin out of range;";
+        if (word & kErrJob) what += " a job id out of range;";
+        return fail(h, SLAQ_E_CUDA, what);
+    }
     return SLAQ_OK;
 }
 
@@ -459,6 +485,8 @@ int do_load(slaq_handle* h, int32_t n, const int32_t* ids, const int64_t* offset
         }
         h->packed_pool = new_pool;
         h->packed_len = (size_t)total;
+        h->job.packed_lo = new_pool;
+        h->job.packed_hi = new_pool ? new_pool + total : nullptr;
         d_src = new_pool;
     } else if (total > 0) {
         void* buf = nullptr;

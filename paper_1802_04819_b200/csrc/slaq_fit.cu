@@ -86,9 +86,20 @@ __device__ int stage_window(const JobArrays& job, int j, int h_cap, const Lanes&
     const int H = job.count[j];
     if (H <= 0) return 0;
     if (H > cap || H > h_cap || row == nullptr) {   // never expected: record and skip the job
-        if (S.l == 0) atomicOr(err_word, 1);
+        if (S.l == 0) atomicOr(err_word, kErrWindow);
         return 0;
     }
+#ifdef SLAQ_DEBUG_BOUNDS
+    {   // the ring lies inside one of the pools, and the write position inside the ring
+        const bool in_ring = row >= job.ring_lo && row + cap <= job.ring_hi;
+        const bool in_packed = job.packed_lo && row >= job.packed_lo && row + cap <= job.packed_hi;
+        const int head = job.head[j];
+        if (!(in_ring || in_packed) || head < 0 || head >= cap) {
+            if (S.l == 0) atomicOr(err_word, kErrStorage);
+            return 0;
+        }
+    }
+#endif
     int newest = job.head[j] - 1;
     if (newest < 0) newest += cap;
     // asynchronous 8-byte copies straight into the lane's column: all of a lane's points are in
@@ -97,7 +108,7 @@ __device__ int stage_window(const JobArrays& job, int j, int h_cap, const Lanes&
     for (int m = S.l; m < H; m += S.L, dst += 32) {
         int pos = newest - m;
         pos += pos < 0 ? cap : 0;
-        copy_async_8(dst, row + pos);
+        if (index_ok(pos, cap, kErrStorage, err_word) && S.holds(dst)) copy_async_8(dst, row + pos);
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     return H;
@@ -124,7 +135,7 @@ __device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double 
     for (int k = 0; k < k_all; ++k) {
         const int m = S.l + S.L * k;
         if (m < H) {
-            const double v = S.y[k * 32 + S.lane];
+            const double v = S.level(k);
             fin &= finite_d(v) ? 1 : 0;
             if (m + 1 < H) dmax = fmax(dmax, older_neighbour(S, k) - v);
         }
@@ -149,8 +160,8 @@ __device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double 
     for (int k = 0; k < k_all; ++k) {
         const int m = S.l + S.L * k;
         if (want_changes && m + 1 < H) {
-            const double change = __ddiv_rn(older_neighbour(S, k) - S.y[k * 32 + S.lane], M);
-            const double w = S.wtab[m];
+            const double change = __ddiv_rn(older_neighbour(S, k) - S.level(k), M);
+            const double w = S.weight(m);
             num = fma(w, change, num);
             den += w;
             if (changes_out) changes_out[H - 1 - m] = change;
@@ -165,8 +176,8 @@ __device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double 
     for (int k = 0; k < k_all; ++k) {
         const int m = S.l + S.L * k;
         if (usable && m < H) {
-            const double y = __ddiv_rn(S.y[k * 32 + S.lane], M);
-            S.y[k * 32 + S.lane] = y;
+            const double y = __ddiv_rn(S.level(k), M);
+            if (S.holds(S.y + k * 32 + S.lane)) S.y[k * 32 + S.lane] = y;
             lo = fmin(lo, y);
             hi = fmax(hi, y);
         }
@@ -184,8 +195,8 @@ __device__ double mean_change_of_levels(const Lanes& S, int H, int k_all) {
     for (int k = 0; k < k_all; ++k) {
         const int m = S.l + S.L * k;
         if (m + 1 < H) {
-            const double w = S.wtab[m];
-            num = fma(w, older_neighbour(S, k) - S.y[k * 32 + S.lane], num);
+            const double w = S.weight(m);
+            num = fma(w, older_neighbour(S, k) - S.level(k), num);
             den += w;
         }
     }
@@ -359,7 +370,8 @@ __device__ __forceinline__ void park(const Lanes& S, const SweepSums& s, bool ke
     if (keep && S.l < 2) {
         const int n = S.park_stride();
 #pragma unroll
-        for (int k = 0; k < kParked; ++k) S.park[k * n] = s.v[k];
+        for (int k = 0; k < kParked; ++k)
+            if (S.holds(S.park + k * n)) S.park[k * n] = s.v[k];
     }
     __syncwarp();
 }
@@ -368,6 +380,11 @@ __device__ __forceinline__ void park(const Lanes& S, const SweepSums& s, bool ke
 __device__ __forceinline__ void normal_equations(const Lanes& S, int fam, double sw, Sym4& A, double (&g)[4]) {
     const double* c = S.park;
     const int n = S.park_stride();
+    if (!S.holds(c) || !S.holds(c + (kParked - 1) * n)) {   // bounds build only: leave the system empty
+        A = Sym4{0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+        g[0] = g[1] = g[2] = g[3] = 0.0;
+        return;
+    }
     if (fam == 0) {
         A.a00 = c[4 * n]; A.a01 = c[3 * n]; A.a02 = c[2 * n]; A.a11 = c[2 * n]; A.a12 = c[1 * n];
         A.a22 = c[0];
@@ -400,8 +417,8 @@ __device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span,
         const int m = S.l + S.L * k;
         if (busy && m < H) {
             const double x = -md * inv_span;
-            const double w = S.wtab[m];
-            const double y = S.y[k * 32 + S.lane];
+            const double w = S.weight(m);
+            const double y = S.level(k);
             sw += w;
             swy2 = fma(w * y, y, swy2);
             if (any_guess) {
@@ -455,8 +472,9 @@ __device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span,
         good = good && pos;
         // the oldest point (m = H - 1) and the newest (m = 0), read from the lanes that own them
         const int m_old = max(H - 1, 0);
-        const double y_old = S.y[(m_old / S.L) * 32 + (S.lane - S.l) + (m_old & (S.L - 1))];
-        const double y_new = S.y[S.lane - S.l];
+        const double* at_old = S.y + (m_old / S.L) * 32 + (S.lane - S.l) + (m_old & (S.L - 1));
+        const double y_old = S.holds(at_old) ? *at_old : 0.0;
+        const double y_new = S.holds(S.y + S.lane - S.l) ? S.y[S.lane - S.l] : 0.0;
         if (good) {
             pI[0] = sol[0]; pI[1] = sol[1]; pI[2] = sol[2];
         } else {
@@ -555,6 +573,10 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
     Lanes S;
     S.wtab = wtab;
     S.lane = lane;
+    S.slice = slice;
+    S.slice_len = cls.slice;
+    S.wtab_len = cls.h_max;
+    S.err_word = err_word;
     for (int i = threadIdx.x; i < cls.h_max; i += blockDim.x) wtab[i] = g_wtab[i];
     if (threadIdx.x == 0) {   // queue slots of each class: one slot = one warp's worth of jobs
         int run = 0;
@@ -589,7 +611,8 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         const int last = start[cls.h_lo[c]];
         const int base = start[h_hi] + (slot - slot_base[c]) * G;
         const int idx = base + g;
-        const int j = idx < last ? order[idx] : -1;
+        int j = idx < last && index_ok(idx, job.max_jobs, kErrJob, err_word) ? order[idx] : -1;
+        if (j >= 0 && !index_ok(j, job.max_jobs, kErrJob, err_word)) j = -1;
         __syncwarp();
         const int H = stage_window(job, j, h_hi, S, err_word);
         const int k_all = warp_max_int((H + L - 1) / L);
@@ -722,7 +745,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
             p_out[1] = 1.0;   // at most the whole normalised loss
         } else if (status == SLAQ_JOB_FITTED && family < 0) {
             status = H >= min_fit_points ? SLAQ_JOB_FIT_FAILED : SLAQ_JOB_SHORT;
-            const double y_new = S.y[lane - S.l];
+            const double y_new = S.holds(S.y + lane - S.l) ? S.y[lane - S.l] : 0.0;
             p_out[0] = rho;
             p_out[1] = y_new > 0.0 ? y_new : CUDART_INF;
             p_out[2] = p_out[3] = CUDART_NAN;
@@ -792,6 +815,10 @@ normalise_export_kernel(JobArrays job, const int32_t* __restrict__ ids, const in
     const int k_cap = (max_hist + 31) / 32;
     Lanes S;
     S.y = smem + max_hist + (size_t)warp * (k_cap + 1) * 32;
+    S.slice = S.y;
+    S.slice_len = (k_cap + 1) * 32;
+    S.wtab_len = max_hist;
+    S.err_word = err_word;
     S.park = nullptr;
     S.wtab = wtab;
     S.lane = lane;
@@ -801,7 +828,8 @@ normalise_export_kernel(JobArrays job, const int32_t* __restrict__ ids, const in
     __syncthreads();
     const int slot = blockIdx.x * (blockDim.x >> 5) + warp;
     if (slot >= n) return;
-    const int j = ids[slot];
+    int j = ids[slot];
+    if (!index_ok(j, job.max_jobs, kErrJob, err_word)) j = -1;
     const int H = stage_window(job, j, max_hist, S, err_word);
     __syncwarp();
     if (H <= 0) {
@@ -819,7 +847,7 @@ normalise_export_kernel(JobArrays job, const int32_t* __restrict__ ids, const in
                 if (levels) levels[base + H - 1 - m] = CUDART_NAN;
                 if (changes) changes[base + H - 1 - m] = CUDART_NAN;
             } else if (levels) {
-                levels[base + H - 1 - m] = S.y[k * 32 + lane];
+                levels[base + H - 1 - m] = S.level(k);
             }
         }
     }
@@ -895,7 +923,7 @@ __global__ void __launch_bounds__(1024) length_scan_kernel(const int32_t* __rest
 // length with a single global atomic, and places its jobs inside those ranges.
 __global__ void __launch_bounds__(kSortThreads)
 length_scatter_kernel(const int32_t* __restrict__ count, int max_jobs, int max_hist, int32_t* cursor,
-                      int32_t* order) {
+                      int32_t* order, int32_t* err_word) {
     extern __shared__ int sh_sort[];    // [max_hist + 1] counts, then [max_hist + 1] next free position
     int* sh_count = sh_sort;
     int* sh_next = sh_sort + (max_hist + 1);
@@ -930,7 +958,8 @@ length_scatter_kernel(const int32_t* __restrict__ count, int max_jobs, int max_h
             int first = 0;
             if (lane == leader) first = atomicAdd(&sh_next[H], __popc(peers));
             first = __shfl_sync(peers, first, leader);
-            order[first + __popc(peers & ((1u << lane) - 1u))] = j;
+            const int at = first + __popc(peers & ((1u << lane) - 1u));
+            if (index_ok(at, max_jobs, kErrJob, err_word)) order[at] = j;
         }
     }
 }
@@ -953,7 +982,7 @@ int launch_fit(slaq_handle* h) {
         length_count_kernel<<<blocks, kSortThreads, one, st>>>(h->job.count, J, Hmax, h->scratch.bucket);
         length_scan_kernel<<<1, 1024, 0, st>>>(h->scratch.bucket, Hmax, h->scratch.start, h->scratch.cursor);
         length_scatter_kernel<<<blocks, kSortThreads, 2 * one, st>>>(h->job.count, J, Hmax, h->scratch.cursor,
-                                                                     h->scratch.order);
+                                                                     h->scratch.order, h->err_word);
         launches += 3;
     }
     // Length classes, longest first.  A warp's slice holds the parked sums of its jobs (kParked

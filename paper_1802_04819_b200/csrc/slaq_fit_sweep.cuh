@@ -6,6 +6,8 @@
 
 #include <math_constants.h>
 
+#include "slaq_bounds.cuh"
+
 namespace slaq {
 
 constexpr unsigned kFull = 0xffffffffu;
@@ -34,11 +36,26 @@ struct Lanes {
     const double* wtab;
     int lane, L, l;
     __device__ __forceinline__ int park_stride() const { return 64 >> (__ffs(L) - 1); }   // 2 * (32 / L), L a power of two
+    // extents, read by the bounds build only: the warp's slice [slice, slice + slice_len) and the weight table
+    const double* slice;
+    int slice_len, wtab_len;
+    int32_t* err_word;
+    __device__ __forceinline__ bool holds(const double* p) const {
+        return index_ok(p - slice, slice_len, kErrShared, err_word);
+    }
+    __device__ __forceinline__ double weight(int m) const {
+        return index_ok(m, wtab_len, kErrShared, err_word) ? wtab[m] : 0.0;
+    }
+    __device__ __forceinline__ double level(int k) const {   // the lane's point of row k
+        const double* p = y + k * 32 + lane;
+        return holds(p) ? *p : 0.0;
+    }
 };
 
 // The window value at distance m + 1 from the newest point, seen from the lane that owns m.
 __device__ __forceinline__ double older_neighbour(const Lanes& S, int k) {
-    return S.l + 1 < S.L ? S.y[k * 32 + S.lane + 1] : S.y[(k + 1) * 32 + S.lane - (S.L - 1)];
+    const double* p = S.l + 1 < S.L ? S.y + k * 32 + S.lane + 1 : S.y + (k + 1) * 32 + S.lane - (S.L - 1);
+    return S.holds(p) ? *p : 0.0;
 }
 
 // What a lane keeps of one sweep: the sums of ITS family over the whole window.
@@ -75,8 +92,8 @@ __device__ __forceinline__ void sweep(const Lanes& S, int fam, int H, int k_all,
     for (int k = 0, m = S.l; k < k_all; ++k, m += S.L, md += dL, yp += 32) {
         if (m < H) {
             const double x = -md * inv_span;
-            const double w = S.wtab[m];
-            const double y = *yp;
+            const double w = S.weight(m);
+            const double y = S.holds(yp) ? *yp : 0.0;
             const double x2 = x * x;
             if (doI) {
                 const double q = fma(fma(pI[0], x, pI[1]), x, pI[2]);

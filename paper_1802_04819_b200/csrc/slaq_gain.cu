@@ -140,13 +140,15 @@ gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int f
             g = fmin(g, carry);
             carry = __shfl_sync(kFull, g, 31);
             const bool counted = active && n <= cap && n >= first_unit;
-            if (n <= cap) gain[(size_t)j * cap + (n - 1)] = g;
+            if (n <= cap && index_ok((long long)j * cap + (n - 1), (long long)max_jobs * cap, kErrGain, job.err_word))
+                gain[(size_t)j * cap + (n - 1)] = g;
             const unsigned digit = (unsigned)((unsigned long long)__double_as_longlong(g) >> (64 - kRadixBits));
             // lanes with the same digit add once: a row is nearly constant in its top bits
             const unsigned live = __ballot_sync(kFull, counted);
             if (counted) {
                 const unsigned peers = __match_any_sync(live, digit);
-                if ((int)(__ffs(peers) - 1) == lane) atomicAdd(&sh_hist[digit], (unsigned)__popc(peers));
+                if ((int)(__ffs(peers) - 1) == lane && index_ok(digit, kRadixBins, kErrBin, job.err_word))
+                    atomicAdd(&sh_hist[digit], (unsigned)__popc(peers));
             }
         }
     }

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "slaq.h"
+#include "slaq_bounds.cuh"
 
 namespace slaq {
 
@@ -33,6 +34,13 @@ struct JobArrays {
     double* s_set;       // fixed time law (NaN: use the estimate)
     double* w_set;
     int32_t* last_alloc; // core count of the last epoch (1 before any)
+    // extents, read by the bounds build only
+    int32_t max_jobs;
+    const double* ring_lo;     // the ring pool [ring_lo, ring_hi)
+    const double* ring_hi;
+    const double* packed_lo;   // the packed pool (both null while there is none)
+    const double* packed_hi;
+    int32_t* err_word;
 };
 
 // What the fit leaves for the later stages, one entry per job.
