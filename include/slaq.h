@@ -51,7 +51,7 @@ enum {
     SLAQ_E_NONFINITE = -3,  /* a loss or time that is NaN or infinite */
     SLAQ_E_NOMEM = -4,      /* device or host allocation failed, or the given workspace is too small */
     SLAQ_E_CUDA = -5,       /* a CUDA call failed; the message holds its error string */
-    SLAQ_E_TIMEOUT = -6,    /* a bounded device-side wait ran out */
+    SLAQ_E_TIMEOUT = -6,    /* reserved: no kernel of this library waits on another, so nothing returns it */
     SLAQ_W_OVERSUBSCRIBED = 1, /* fewer cores than active jobs: no one-core floor, cores go to the best first units */
     SLAQ_W_UNDERFILLED = 2     /* more cores than active jobs x max_cores_per_job: every job is at its cap */
 };
@@ -121,15 +121,19 @@ typedef struct slaq_stats {
 
 /*
  * Create a scheduler for job ids 0..max_jobs-1, each keeping a window of its newest
- * max_hist losses (4 <= max_hist <= 6000) - the "history loss values" the fit uses.
+ * max_hist losses (4 <= max_hist <= 6000) - the loss history that the weighted fit of
+ * Design, "Predicting Quality Improvement" works on.
  * Allocates all device state with cudaMalloc on the current device:
  * slaq_workspace_bytes(max_jobs, max_hist, 64) bytes; up to 64 cores per job.
- * *out receives the handle.  Errors: SLAQ_E_ARG, SLAQ_E_NOMEM, SLAQ_E_CUDA.
+ * *out receives the handle.  The three calls slaq_create, slaq_append_losses and
+ * slaq_schedule are the inputs and the output of the problem statement (Design,
+ * "Scheduling Based on Quality Improvements": J jobs with their loss histories, the epoch
+ * T, the capacity C; a_j out).  Errors: SLAQ_E_ARG, SLAQ_E_NOMEM, SLAQ_E_CUDA.
  */
 int slaq_create(int32_t max_jobs, int32_t max_hist, slaq_t** out);
 
 /*
- * Same with an explicit cap on cores per job (1..1024).  dev_ws == NULL: the library
+ * Same with an explicit cap on cores per job (1..1024; the paper has no cap).  dev_ws == NULL: the library
  * allocates.  Otherwise the state lives inside device memory the caller owns (for
  * instance a torch tensor): dev_ws must be 256-byte aligned, hold at least
  * slaq_workspace_bytes(max_jobs, max_hist, max_cores_per_job) bytes and outlive the
@@ -137,17 +141,35 @@ int slaq_create(int32_t max_jobs, int32_t max_hist, slaq_t** out);
  */
 int slaq_create_in(void* dev_ws, size_t bytes, int32_t max_jobs, int32_t max_hist, int32_t max_cores_per_job,
                    slaq_t** out);
+/* Bytes slaq_create_in needs for these sizes (0 for sizes outside the limits).  Host arithmetic only. */
 size_t slaq_workspace_bytes(int32_t max_jobs, int32_t max_hist, int32_t max_cores_per_job);
 
-/* Release the handle and the device memory it allocated itself.  NULL is accepted. */
+/*
+ * Release the handle and the device memory it allocated itself (workspace, packed pool, call
+ * buffer).  NULL is accepted.  Housekeeping: the paper has no counterpart.
+ */
 int slaq_destroy(slaq_t* h);
 
-/* Message for the last non-zero status of h (handle-owned storage; valid until the next call on h). */
+/*
+ * Message for the last non-zero status of h (handle-owned storage; valid until the next call
+ * on h).  Housekeeping: the paper has no counterpart.
+ */
 const char* slaq_last_error(const slaq_t* h);
 
-/* cuda_stream is a cudaStream_t (NULL = default stream).  All later work of h runs on it. */
+/*
+ * cuda_stream is a cudaStream_t (NULL = default stream).  The call waits for the work already
+ * queued on the old stream; all later work of h runs on the new one.  Housekeeping: the paper
+ * has no counterpart.
+ */
 int slaq_set_stream(slaq_t* h, void* cuda_stream);
 
+/*
+ * Set / read one of the SLAQ_P_* parameters above.  The paper fixes none of them: it asks for
+ * an exponentially weighted fit (Design, "Predicting Quality Improvement") without naming the
+ * weight base, the solver or its trial count, and it has no cap on cores per job; the defaults
+ * are this library's readings.  Errors: SLAQ_E_ARG (unknown key, value outside the range given
+ * with the key), SLAQ_E_RANGE (more cores per job than the handle was created for).
+ */
 int slaq_set_param(slaq_t* h, int key, double value);
 int slaq_get_param(const slaq_t* h, int key, double* out_value);
 
@@ -156,8 +178,8 @@ int slaq_get_param(const slaq_t* h, int key, double* out_value);
  * iter_times[i] the wall seconds that iteration took.  A job id may appear at most once
  * per call.  The first loss activates the job (iteration index 0).  The call updates the
  * job's window (the oldest point is dropped once max_hist are stored), its iteration
- * index, the largest reduction l_{k-1} - l_k it has shown so far ("the largest change we
- * have seen so far", "Normalizing Quality Metrics"), and the sums of its iteration-time
+ * index, the largest reduction l_{k-1} - l_k it has shown so far (the denominator of the
+ * normalised change in Design, "Normalizing Quality Metrics"), and the sums of its iteration-time
  * law t(n) = s + w/n, the iteration being booked at the job's current core count: its
  * allocation from the last slaq_schedule, 1 before any.  iter_times may be NULL (no time
  * sample).  All pointers are host pointers, n entries each.
@@ -195,13 +217,19 @@ int slaq_load_histories_packed(slaq_t* h, int32_t n_jobs, const int32_t* job_ids
 
 /*
  * Fix the iteration-time law t(n) = s[i] + w[i]/n of the listed jobs (s >= 0 seconds,
- * w > 0 core-seconds), overriding the estimate from iter_times.  The paper leaves the
- * map from cores to progress open ("predict how much progress the job would achieve if
- * it was granted a certain amount of resources"); this law is the library's.  Host pointers.
+ * w > 0 core-seconds), overriding the estimate from iter_times.  The paper asks for a
+ * prediction of a job's progress under a given amount of resources (Design, second duty of
+ * the scheduler) without giving the map from cores to iterations; this law is the library's.
+ * Host pointers.  Errors: SLAQ_E_ARG (null, duplicate id, s < 0, w <= 0, not finite), SLAQ_E_RANGE.
  */
 int slaq_set_time_model(slaq_t* h, int32_t n, const int32_t* job_ids, const double* s, const double* w);
 
-/* Deactivate jobs and forget their state.  Host pointer. */
+/*
+ * Deactivate the listed jobs (finished or cancelled: they leave the set J of running jobs of
+ * Design, "Scheduling Based on Quality Improvements") and forget their histories, largest
+ * reduction, time sums, time law and fitted curves; a later append starts them anew at
+ * iteration 0.  Ids may repeat.  Host pointer.  Errors: SLAQ_E_ARG, SLAQ_E_RANGE.
+ */
 int slaq_remove_jobs(slaq_t* h, int32_t n, const int32_t* job_ids);
 
 /*
@@ -214,7 +242,10 @@ int slaq_remove_jobs(slaq_t* h, int32_t n, const int32_t* job_ids);
  * (SLAQ_E_ARG for T <= 0, C < 0 or null; SLAQ_E_CUDA).
  */
 int slaq_schedule(slaq_t* h, double epoch_seconds, int64_t total_cores, int32_t* out_alloc);
-/* Same, asynchronous on the handle's stream; d_out_alloc is a device pointer or NULL (result kept in the handle). */
+/*
+ * Same, asynchronous on the handle's stream; d_out_alloc is a device pointer (max_jobs entries) or
+ * NULL (the result stays in the handle: slaq_get_predictions, the next append's core counts).
+ */
 int slaq_schedule_device(slaq_t* h, double epoch_seconds, int64_t total_cores, int32_t* d_out_alloc);
 
 /*
@@ -243,7 +274,12 @@ int slaq_get_predictions(slaq_t* h, double* out_reduction, double* out_gain, int
 int slaq_get_normalised(slaq_t* h, int32_t n, const int32_t* job_ids, int64_t capacity, int64_t* out_offsets,
                         double* out_changes, double* out_levels, double* out_largest);
 
-/* Iteration-time law in use for every job (NaN where none yet).  Host pointers [max_jobs]. */
+/*
+ * Iteration-time law in use for every job: the fixed one where slaq_set_time_model gave one,
+ * else the least-squares estimate from the appended iteration times (NaN where a job has
+ * neither).  Host pointers [max_jobs].  The law itself is the library's (see
+ * slaq_set_time_model); the paper has no counterpart.
+ */
 int slaq_get_time_model(slaq_t* h, double* out_s, double* out_w);
 
 /*
@@ -267,14 +303,44 @@ int slaq_set_fit_state(slaq_t* h, const double* params, const uint8_t* mask, con
                        const double* scale);
 
 /*
- * Test hook for the allocation step alone: overwrite the gain rows (host,
+ * Test hook for the allocation step alone (the greedy loop of Design, "Scheduling Based on
+ * Quality Improvements", on gains the caller supplies): overwrite the gain rows (host,
  * max_jobs x max_cores_per_job, rows non-increasing, values >= +0) and allocate from
- * them with slaq_allocate_only, which runs only the greedy-equivalent selection.
+ * them with slaq_allocate_only, which runs only the greedy-equivalent selection and fills
+ * out_alloc (host, max_jobs) like slaq_schedule.
  */
 int slaq_set_gains(slaq_t* h, const double* gain);
 int slaq_allocate_only(slaq_t* h, int64_t total_cores, int32_t* out_alloc);
 
+/*
+ * Timings and counts of the last epoch (the struct above).  Diagnostic: the paper reports only
+ * the total time of a scheduling decision (Evaluation, "Scalability and efficiency").
+ * Errors: SLAQ_E_ARG (null, or no epoch has run yet), SLAQ_E_CUDA.
+ */
 int slaq_get_stats(slaq_t* h, slaq_stats* out);
+
+/*
+ * Checkpoint and resume (the paper has no counterpart: its scheduler lives inside a long-running
+ * driver).  slaq_export_state writes everything the handle knows about its jobs into one host
+ * blob: per job the stored window (oldest first), the index of its newest iteration, the largest
+ * reduction seen, the sums and the fixed value of its iteration-time law, its current core count,
+ * and both records of its fitted curves (what the last epoch ended with, what the next fit
+ * starts from).  Parameters (slaq_set_param) and the stream are not part of it.
+ * slaq_export_state_bytes gives the size the blob needs now; capacity below it: SLAQ_E_RANGE.
+ * slaq_import_state replaces the whole state of h by a blob's: h must have been created for the
+ * same max_jobs and for a max_hist of at least the blob's longest window (SLAQ_E_RANGE
+ * otherwise); windows are stored as rings of max_hist slots, also those that the exporting handle
+ * held packed (such a job kept the window length it was loaded with; after the import its window
+ * grows with later appends up to max_hist).  Apart from that, a handle that imported a blob
+ * schedules, appends and warm-starts bit for bit like the handle that exported it, given the same
+ * max_hist and parameters.  The blob is plain host memory in this machine's byte order, valid
+ * for this library version (SLAQ_E_ARG for anything else, or for sizes that disagree; the losses
+ * are checked as in slaq_load_histories).  On an error found while reading the blob's tables the
+ * handle is unchanged; after that point a failing import leaves it empty.
+ */
+int slaq_export_state_bytes(slaq_t* h, size_t* out_bytes);
+int slaq_export_state(slaq_t* h, void* out_blob, size_t capacity);
+int slaq_import_state(slaq_t* h, const void* blob, size_t bytes);
 
 /*
  * Diagnostic (the paper has no counterpart).  In a library built with -DSLAQ_PHASE_CLOCKS

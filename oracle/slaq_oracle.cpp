@@ -432,8 +432,8 @@ FitData make_fit_data(const double* loss, int64_t H, double M, double gamma) {
 }
 
 // ---------------------------------------------------------------------------------
-// Warm start ("short time intervals ... continued rebalancing", Evaluation,
-// "Scalability and efficiency"): a scheduler that refits every few seconds may start
+// Warm start (Evaluation, "Scalability and efficiency": the scheduler reruns every few
+// seconds and keeps rebalancing): a scheduler that refits that often may start
 // each family from the parameters it found last epoch instead of from the linearised
 // first guess.  The paper does not say how its fits are started; this is this
 // implementation's rule.  The fitted curve is a function of the iteration index k and

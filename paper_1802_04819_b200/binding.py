@@ -21,7 +21,8 @@ EXPORTED_SYMBOLS = [
     "slaq_load_histories_packed", "slaq_set_time_model", "slaq_remove_jobs", "slaq_schedule", "slaq_schedule_device",
     "slaq_get_predictions", "slaq_get_normalised", "slaq_get_time_model", "slaq_get_fit_state",
     "slaq_set_fit_state", "slaq_set_gains", "slaq_allocate_only",
-    "slaq_get_stats", "slaq_get_fit_phase_cycles", "slaq_allocate_static", "slaq_get_active_count", "slaq_shard_predict", "slaq_shard_histogram",
+    "slaq_get_stats", "slaq_get_fit_phase_cycles", "slaq_export_state_bytes", "slaq_export_state",
+    "slaq_import_state", "slaq_allocate_static", "slaq_get_active_count", "slaq_shard_predict", "slaq_shard_histogram",
     "slaq_shard_pick", "slaq_shard_pass", "slaq_shard_count", "slaq_shard_finalise",
 ]
 
@@ -83,6 +84,9 @@ def load_library(variant: str | None = None):
         "slaq_allocate_only": (c_int, [vp, c_int64, vp]),
         "slaq_get_stats": (c_int, [vp, POINTER(Stats)]),
         "slaq_get_fit_phase_cycles": (c_int, [vp, vp]),
+        "slaq_export_state_bytes": (c_int, [vp, POINTER(c_size_t)]),
+        "slaq_export_state": (c_int, [vp, vp, c_size_t]),
+        "slaq_import_state": (c_int, [vp, vp, c_size_t]),
         "slaq_allocate_static": (c_int, [vp, c_int32, c_int32, c_int64, vp, vp, vp]),
         "slaq_get_active_count": (c_int, [vp, POINTER(c_int32)]),
         "slaq_shard_predict": (c_int, [vp, c_double, c_int32]),
@@ -310,6 +314,18 @@ class Scheduler:
         out = np.empty(self.max_jobs, np.int32)
         self._check(self._lib.slaq_shard_finalise(self._h, int(ties_before), _ptr(out)))
         return out
+
+    def export_state(self) -> np.ndarray:
+        """The whole per-job state of the handle as one blob (uint8 array)."""
+        n = c_size_t()
+        self._check(self._lib.slaq_export_state_bytes(self._h, ctypes.byref(n)))
+        blob = np.zeros(n.value, np.uint8)
+        self._check(self._lib.slaq_export_state(self._h, _ptr(blob), blob.size))
+        return blob
+
+    def import_state(self, blob):
+        blob = np.ascontiguousarray(blob, dtype=np.uint8)
+        return self._check(self._lib.slaq_import_state(self._h, _ptr(blob), blob.size))
 
     def get_fit_phase_cycles(self):
         """SM cycles the fit kernel's warps spent per phase (zeros unless the "clocks" variant is loaded)."""

@@ -247,6 +247,23 @@ __global__ void load_kernel(JobArrays job, FitArrays fit, double* ring, int max_
     }
 }
 
+// Export: one warp per job copies its window, oldest point first, to out[offsets[j] ..].
+__global__ void export_windows_kernel(JobArrays job, int max_jobs, const int64_t* offsets, double* out) {
+    const int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (j >= max_jobs) return;
+    const int H = job.count[j], cap = job.cap[j];
+    if (H <= 0 || H > cap) return;
+    const double* row = job.row[j];
+    int oldest = job.head[j] - H;
+    if (oldest < 0) oldest += cap;
+    const int64_t base = offsets[j];
+    for (int i = lane; i < H; i += 32) {
+        int pos = oldest + i;
+        pos -= pos >= cap ? cap : 0;
+        if (index_ok(pos, cap, kErrStorage, job.err_word)) out[base + i] = row[pos];
+    }
+}
+
 __global__ void set_time_kernel(JobArrays job, int max_jobs, int n, const int32_t* ids, const double* s,
                                 const double* w) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -1062,6 +1079,209 @@ int slaq_set_fit_state(slaq_t* h, const double* params, const uint8_t* mask, con
     CK(cudaMemcpyAsync(h->fit.largest, scale, sizeof(double) * J, up, st), "copy fit scales");
     CK(cudaMemcpyAsync(h->fit.warm_scale, scale, sizeof(double) * J, up, st), "copy fit scales");
     CK(cudaStreamSynchronize(st), "copy fit state");
+    return SLAQ_OK;
+}
+
+// ---- the whole scheduler state as one host blob ----
+
+namespace {
+
+constexpr uint64_t kStateMagic = 0x51414c5345544154ull;   // "TATESLAQ" read as little-endian bytes
+constexpr uint32_t kStateVersion = 1;
+
+struct StateHeader {
+    uint64_t magic;
+    uint32_t version;
+    int32_t max_jobs;
+    int32_t max_hist;      // longest window in the blob
+    int32_t reserved;
+    int64_t total_points;
+    uint64_t bytes;        // size of the whole blob
+};
+
+// The per-job arrays of a blob, in order, each entry count given per job; all 8-byte aligned
+// because every block's size is a multiple of 8 (max_jobs is padded to a multiple of 8 entries).
+struct StateLayout {
+    size_t J8;             // max_jobs rounded up to a multiple of 8
+    size_t off_count, off_k_last, off_m_seen, off_tm, off_s_set, off_w_set, off_last_alloc;
+    size_t off_both, off_mask, off_k_fit, off_span, off_largest;
+    size_t off_warm_p, off_warm_mask, off_warm_k, off_warm_span, off_warm_scale;
+    size_t off_offsets, off_losses, bytes;
+};
+
+StateLayout state_layout(int32_t max_jobs, int64_t total_points) {
+    StateLayout L;
+    L.J8 = ((size_t)max_jobs + 7) / 8 * 8;
+    size_t o = sizeof(StateHeader);
+    auto take = [&](size_t bytes) { const size_t at = o; o += (bytes + 7) / 8 * 8; return at; };
+    L.off_count = take(4 * L.J8);
+    L.off_k_last = take(8 * L.J8);
+    L.off_m_seen = take(8 * L.J8);
+    L.off_tm = take(8 * 8 * (size_t)max_jobs);
+    L.off_s_set = take(8 * L.J8);
+    L.off_w_set = take(8 * L.J8);
+    L.off_last_alloc = take(4 * L.J8);
+    L.off_both = take(8 * 8 * L.J8);
+    L.off_mask = take(L.J8);
+    L.off_k_fit = take(8 * L.J8);
+    L.off_span = take(8 * L.J8);
+    L.off_largest = take(8 * L.J8);
+    L.off_warm_p = take(8 * 8 * L.J8);
+    L.off_warm_mask = take(L.J8);
+    L.off_warm_k = take(8 * L.J8);
+    L.off_warm_span = take(8 * L.J8);
+    L.off_warm_scale = take(8 * L.J8);
+    L.off_offsets = take(8 * ((size_t)max_jobs + 1));
+    L.off_losses = take(8 * (size_t)total_points);
+    L.bytes = o;
+    return L;
+}
+
+int read_counts(slaq_handle* h, std::vector<int32_t>& counts, int64_t* total, int32_t* longest) {
+    counts.resize((size_t)h->max_jobs);
+    CK(cudaMemcpyAsync(counts.data(), h->job.count, sizeof(int32_t) * counts.size(), cudaMemcpyDeviceToHost, h->stream),
+       "read window lengths");
+    CK(cudaStreamSynchronize(h->stream), "read window lengths");
+    *total = 0;
+    *longest = 0;
+    for (int32_t c : counts) {
+        *total += c > 0 ? c : 0;
+        *longest = std::max(*longest, c);
+    }
+    return SLAQ_OK;
+}
+
+}  // namespace
+
+int slaq_export_state_bytes(slaq_t* h, size_t* out_bytes) {
+    if (!h || !out_bytes) return SLAQ_E_ARG;
+    if (const int rc = check_device(h)) return rc;
+    std::vector<int32_t> counts;
+    int64_t total = 0;
+    int32_t longest = 0;
+    if (const int rc = read_counts(h, counts, &total, &longest)) return rc;
+    *out_bytes = state_layout(h->max_jobs, total).bytes;
+    return SLAQ_OK;
+}
+
+int slaq_export_state(slaq_t* h, void* out_blob, size_t capacity) {
+    if (!h || !out_blob) return SLAQ_E_ARG;
+    if (const int rc = check_device(h)) return rc;
+    std::vector<int32_t> counts;
+    int64_t total = 0;
+    int32_t longest = 0;
+    if (const int rc = read_counts(h, counts, &total, &longest)) return rc;
+    const StateLayout L = state_layout(h->max_jobs, total);
+    if (capacity < L.bytes) return fail(h, SLAQ_E_RANGE, "blob capacity below slaq_export_state_bytes()");
+    char* blob = static_cast<char*>(out_blob);
+    std::memset(blob, 0, L.bytes);
+    StateHeader hd{kStateMagic, kStateVersion, h->max_jobs, longest, 0, total, (uint64_t)L.bytes};
+    std::memcpy(blob, &hd, sizeof hd);
+    const size_t J = (size_t)h->max_jobs;
+    int64_t* offsets = reinterpret_cast<int64_t*>(blob + L.off_offsets);
+    offsets[0] = 0;
+    for (size_t j = 0; j < J; ++j) offsets[j + 1] = offsets[j] + (counts[j] > 0 ? counts[j] : 0);
+    cudaStream_t st = h->stream;
+    const cudaMemcpyKind down = cudaMemcpyDeviceToHost;
+    std::memcpy(blob + L.off_count, counts.data(), 4 * J);
+    CK(cudaMemcpyAsync(blob + L.off_k_last, h->job.k_last, 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_m_seen, h->job.m_seen, 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_tm, h->job.tm, 8 * 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_s_set, h->job.s_set, 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_w_set, h->job.w_set, 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_last_alloc, h->job.last_alloc, 4 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_both, h->fit.both, 8 * 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_mask, h->fit.mask, J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_k_fit, h->fit.k_fit, 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_span, h->fit.span, 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_largest, h->fit.largest, 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_warm_p, h->fit.warm_p, 8 * 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_warm_mask, h->fit.warm_mask, J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_warm_k, h->fit.warm_k, 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_warm_span, h->fit.warm_span, 8 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_warm_scale, h->fit.warm_scale, 8 * J, down, st), "export state");
+    if (total > 0) {
+        void* buf = nullptr;
+        if (const int rc = ensure_call_buffer(h, 8 * (size_t)total, &buf)) return rc;
+        CK(cudaMemcpyAsync(h->stage.offsets, offsets, 8 * (J + 1), cudaMemcpyHostToDevice, st), "export state");
+        const int threads = 256, warps = threads / 32;
+        export_windows_kernel<<<(h->max_jobs + warps - 1) / warps, threads, 0, st>>>(h->job, h->max_jobs, h->stage.offsets,
+                                                                                  static_cast<double*>(buf));
+        CK(cudaGetLastError(), "export kernel");
+        CK(cudaMemcpyAsync(blob + L.off_losses, buf, 8 * (size_t)total, down, st), "export state");
+    }
+    CK(cudaStreamSynchronize(st), "export state");
+    return SLAQ_OK;
+}
+
+int slaq_import_state(slaq_t* h, const void* blob_in, size_t bytes) {
+    if (!h || !blob_in) return SLAQ_E_ARG;
+    if (const int rc = check_device(h)) return rc;
+    const char* blob = static_cast<const char*>(blob_in);
+    StateHeader hd;
+    if (bytes < sizeof hd) return fail(h, SLAQ_E_ARG, "state blob shorter than its header");
+    std::memcpy(&hd, blob, sizeof hd);
+    if (hd.magic != kStateMagic || hd.version != kStateVersion) return fail(h, SLAQ_E_ARG, "not a state blob of this library version");
+    if (hd.max_jobs != h->max_jobs) return fail(h, SLAQ_E_RANGE, "state blob of a handle with another number of job ids");
+    if (hd.max_hist > h->max_hist) return fail(h, SLAQ_E_RANGE, "state blob holds windows longer than this handle's max_hist");
+    if (hd.total_points < 0) return fail(h, SLAQ_E_ARG, "state blob: negative point count");
+    const StateLayout L = state_layout(hd.max_jobs, hd.total_points);
+    if (hd.bytes != L.bytes || bytes < L.bytes) return fail(h, SLAQ_E_ARG, "state blob is truncated or its sizes disagree");
+    const size_t J = (size_t)h->max_jobs;
+    const int32_t* counts = reinterpret_cast<const int32_t*>(blob + L.off_count);
+    const int64_t* offsets = reinterpret_cast<const int64_t*>(blob + L.off_offsets);
+    const int64_t* k_last = reinterpret_cast<const int64_t*>(blob + L.off_k_last);
+    const double* m_seen = reinterpret_cast<const double*>(blob + L.off_m_seen);
+    const uint8_t* mask = reinterpret_cast<const uint8_t*>(blob + L.off_mask);
+    const uint8_t* warm_mask = reinterpret_cast<const uint8_t*>(blob + L.off_warm_mask);
+    if (offsets[0] != 0 || offsets[J] != hd.total_points) return fail(h, SLAQ_E_ARG, "state blob: offsets disagree with the point count");
+    for (size_t j = 0; j < J; ++j) {
+        const int64_t H = offsets[j + 1] - offsets[j];
+        if (H < 0 || H > h->max_hist || H != (counts[j] > 0 ? counts[j] : 0))
+            return fail(h, SLAQ_E_ARG, "state blob: a window length disagrees with its offsets");
+        if (std::isnan(m_seen[j]) || m_seen[j] == INFINITY) return fail(h, SLAQ_E_NONFINITE, "state blob: m_seen must be a number below +infinity");
+        if (mask[j] > 3 || warm_mask[j] > 3) return fail(h, SLAQ_E_ARG, "state blob: fit mask above 3");
+    }
+    // everything the handle holds goes; then the windows come in as a bulk load into rings (which checks the losses)
+    cudaStream_t st = h->stream;
+    {
+        const int threads = 256;
+        init_jobs_kernel<<<(h->max_jobs + threads - 1) / threads, threads, 0, st>>>(
+            h->job, h->fit, h->ring_pool, h->max_jobs, h->max_hist, nullptr, h->max_jobs, h->alloc, h->reduction);
+        CK(cudaGetLastError(), "import: reset kernel");
+        CK(cudaStreamSynchronize(st), "import: reset");
+        std::fill(h->active.begin(), h->active.end(), 0);
+        std::fill(h->in_packed.begin(), h->in_packed.end(), 0);
+        h->n_active = 0;
+        if (h->packed_pool) {
+            cudaFree(h->packed_pool);
+            h->packed_pool = nullptr;
+            h->packed_len = 0;
+            h->job.packed_lo = h->job.packed_hi = nullptr;
+        }
+        h->have_epoch = false;
+    }
+    std::vector<int32_t> ids(J);
+    for (size_t j = 0; j < J; ++j) ids[j] = (int32_t)j;
+    const int rc = do_load(h, h->max_jobs, ids.data(), offsets, reinterpret_cast<const double*>(blob + L.off_losses), k_last,
+                           m_seen, false);
+    if (rc) return rc;
+    const cudaMemcpyKind up = cudaMemcpyHostToDevice;
+    CK(cudaMemcpyAsync(h->job.tm, blob + L.off_tm, 8 * 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->job.s_set, blob + L.off_s_set, 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->job.w_set, blob + L.off_w_set, 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->job.last_alloc, blob + L.off_last_alloc, 4 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.both, blob + L.off_both, 8 * 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.mask, blob + L.off_mask, J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.k_fit, blob + L.off_k_fit, 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.span, blob + L.off_span, 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.largest, blob + L.off_largest, 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.warm_p, blob + L.off_warm_p, 8 * 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.warm_mask, blob + L.off_warm_mask, J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.warm_k, blob + L.off_warm_k, 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.warm_span, blob + L.off_warm_span, 8 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->fit.warm_scale, blob + L.off_warm_scale, 8 * J, up, st), "import state");
+    CK(cudaStreamSynchronize(st), "import state");
     return SLAQ_OK;
 }
 

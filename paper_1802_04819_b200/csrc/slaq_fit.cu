@@ -632,14 +632,14 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
 
         if (__any_sync(kFull, fits)) {
             const double inv_span = 1.0 / span;
-            Moments mom;
-            Family F;
-            double pI[4], pII[4];      // the points the next sweep evaluates
+            Moments mom = {0.0, 0.0};
+            Family F = {};
+            double pI[4] = {0.0, 0.0, 0.0, 0.0}, pII[4] = {0.0, 0.0, 0.0, 0.0};   // the points the next sweep evaluates
             // Starting points: the first guesses, or (kWarm) last epoch's parameters where the job
             // has some; a carried-over point without a finite residual is dropped for the
             // family's first guess in a second round.
             int spent = 0;
-            SweepSums sums;
+            SweepSums sums = {};
             if (!kWarm) {
                 first_guesses(S, H, k_all, inv_span, nz.ymin, nz.ymax, fits, fits, fits, mom, pI, pII);
                 sweep(S, fam, H, k_all, inv_span, pI, fits, pII, fits, sums);
