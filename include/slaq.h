@@ -80,12 +80,20 @@ enum {
                                      larger cluster is told the cluster's number of active jobs here, so that
                                      every shard makes the choice the undivided cluster would make and the
                                      results agree bit for bit; 0 (default): the handle's own active jobs */
-    SLAQ_P_EPOCH_GRAPH = 8        /* 1: slaq_schedule / slaq_schedule_device replay the epoch's launches as one
+    SLAQ_P_EPOCH_GRAPH = 8,       /* 1: slaq_schedule / slaq_schedule_device replay the epoch's launches as one
                                      CUDA graph once two calls in a row had the same arguments, parameters and
                                      number of active jobs (an epoch of a small cluster is bound by its sixteen
                                      launches); 0: always plain launches; -1 (default): graph for handles
                                      created for at most 20,000 jobs.  Results are the same either way.  Not
                                      used while the handle's stream is itself being captured. */
+    SLAQ_P_GAIN_ENVELOPE = 9      /* 0 (default) or 1.  The greedy loop is exact when every job's predicted reduction
+                                     R(n) is concave in its cores n, which a convex fitted curve gives.  Where a fit is
+                                     not convex ahead of the newest point (the paper assumes convex losses: footnotes of
+                                     "Predicting Quality Improvement"), the marginal gains may rise with n.  0: they
+                                     are made non-increasing by a running minimum (never predicts more than the curve).
+                                     1: they are replaced by the slopes of the upper concave envelope of the points
+                                     (n, R(n)), the smallest concave function nowhere below R, which keeps the curve's
+                                     whole drop at max_cores_per_job.  Rows of convex fits are the same either way. */
 };
 
 /* per-job status written by slaq_schedule (slaq_get_predictions, out_status) */
@@ -225,6 +233,17 @@ int slaq_load_histories_packed(slaq_t* h, int32_t n_jobs, const int32_t* job_ids
 int slaq_set_time_model(slaq_t* h, int32_t n, const int32_t* job_ids, const double* s, const double* w);
 
 /*
+ * Hints of the loss the listed jobs are expected to end at (Conclusion, "Non-convex optimization":
+ * users may tell the scheduler their target loss, from earlier trials or published results, so that
+ * it does not over-estimate what a job can still gain).  The paper gives no rule; the library's: a
+ * job is never predicted to fall below its target, i.e. its predicted reduction over the epoch is
+ * capped at max(newest loss - target, 0) in units of its largest reduction seen, for every core
+ * count.  targets[i] = NaN removes the hint; infinities are refused (SLAQ_E_NONFINITE).  Hints stay
+ * until replaced or the job is removed.  Host pointers.  Errors: SLAQ_E_ARG, SLAQ_E_RANGE.
+ */
+int slaq_set_target_loss(slaq_t* h, int32_t n, const int32_t* job_ids, const double* targets);
+
+/*
  * Deactivate the listed jobs (finished or cancelled: they leave the set J of running jobs of
  * Design, "Scheduling Based on Quality Improvements") and forget their histories, largest
  * reduction, time sums, time law and fitted curves; a later append starts them anew at
@@ -323,7 +342,7 @@ int slaq_get_stats(slaq_t* h, slaq_stats* out);
  * Checkpoint and resume (the paper has no counterpart: its scheduler lives inside a long-running
  * driver).  slaq_export_state writes everything the handle knows about its jobs into one host
  * blob: per job the stored window (oldest first), the index of its newest iteration, the largest
- * reduction seen, the sums and the fixed value of its iteration-time law, its current core count,
+ * reduction seen, the sums and the fixed value of its iteration-time law, its target-loss hint, its current core count,
  * and both records of its fitted curves (what the last epoch ended with, what the next fit
  * starts from).  Parameters (slaq_set_param) and the stream are not part of it.
  * slaq_export_state_bytes gives the size the blob needs now; capacity below it: SLAQ_E_RANGE.

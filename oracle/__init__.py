@@ -44,7 +44,9 @@ def _bind(lib):
     lib.oracle_predict.argtypes = [c_i64, vp, vp, vp, vp, vp, c_f64, c_i32, c_f64, c_i32, c_i32,
                                    vp, vp, vp, vp, vp, vp, vp]
     lib.oracle_predict_warm.argtypes = [c_i64, vp, vp, vp, vp, vp, c_f64, c_i32, c_f64, c_i32, c_i32,
-                                        vp, vp, vp, vp, vp, vp, vp] + [vp] * 8
+                                        vp, vp, vp, vp, vp, vp, vp] + [vp] * 8 + [c_i32, vp]
+    lib.oracle_envelope.argtypes = [c_i32, vp, vp]
+    lib.oracle_envelope.restype = None
     lib.oracle_carry.argtypes = [c_i32, vp, c_f64, c_f64, c_f64, vp]
     lib.oracle_carry.restype = None
     lib.oracle_allocate.argtypes = [c_i64, c_i32, vp, vp, c_i64, vp]
@@ -98,13 +100,15 @@ def normalise(offsets, losses, m_seen=None):
 
 
 def predict(offsets, losses, m_seen, s, w, epoch_seconds, cap, gamma=0.9, lm_trials=20, threads=0,
-            want_gain=True, k_last=None, warm=None):
+            want_gain=True, k_last=None, warm=None, envelope=False, target_loss=None):
     """Steps 1-3.  Returns a dict with family, params, S, status, evals, M, gain [J, cap], and both
     families' final parameters (`both` [J, 8], `mask`).
 
     warm: dict(valid uint8 [J], p [J, 8], K int64 [J], span [J], M [J]) from an earlier epoch; the
     families it covers start from those parameters carried into this epoch's coordinates
-    (k_last = index of each job's newest iteration now)."""
+    (k_last = index of each job's newest iteration now).
+    envelope: rows become the slopes of the upper concave envelope of R(n) instead of a running minimum.
+    target_loss: per job a loss below which nothing is predicted (NaN: no hint)."""
     lib = _load()
     offsets, losses = _i64(offsets), _f64(losses)
     J = offsets.size - 1
@@ -125,7 +129,17 @@ def predict(offsets, losses, m_seen, s, w, epoch_seconds, cap, gamma=0.9, lm_tri
                             float(gamma), int(lm_trials), int(threads), _p(out["family"]), _p(out["params"]),
                             _p(out["S"]), _p(out["status"]), _p(out["evals"]), _p(out["M"]), _p(out["gain"]),
                             _p(k_last) if warm is not None else None, _p(wv), _p(wp), _p(wK), _p(wS), _p(wM),
-                            _p(out["both"]), _p(out["mask"]))
+                            _p(out["both"]), _p(out["mask"]), int(bool(envelope)),
+                            None if target_loss is None else _p(_f64(target_loss)))
+    return out
+
+
+def envelope(R):
+    """Slopes of the upper concave envelope of the points (n, R[n]), n = 0..len(R)-1."""
+    lib = _load()
+    R = _f64(R)
+    out = np.empty(R.size - 1)
+    lib.oracle_envelope(R.size - 1, _p(R), _p(out))
     return out
 
 
@@ -171,10 +185,10 @@ def time_model(cnt, su, suu, st, sut, stn, umin, umax):
 
 
 def schedule(offsets, losses, m_seen, s, w, epoch_seconds, total_cores, cap, gamma=0.9, lm_trials=20, threads=0,
-             k_last=None, warm=None):
+             k_last=None, warm=None, envelope=False, target_loss=None):
     """One whole epoch on CSR histories.  Returns dict(alloc, R, gain, ...fit record)."""
     out = predict(offsets, losses, m_seen, s, w, epoch_seconds, cap, gamma, lm_trials, threads,
-                  k_last=k_last, warm=warm)
+                  k_last=k_last, warm=warm, envelope=envelope, target_loss=target_loss)
     active = (np.diff(_i64(offsets)) > 0)
     out["alloc"] = allocate(out["gain"], active, total_cores)
     out["R"] = reduction_at(out["gain"], out["alloc"])
@@ -232,6 +246,8 @@ class OracleScheduler:
         # A job's `warm` is refreshed from `fitted` when its history changes, so an epoch repeated
         # without new losses starts from the same point and gives the same result.
         self.warm_start = False
+        self.envelope = False                              # rows as slopes of the concave envelope of R(n)
+        self.target = np.full(max_jobs, np.nan)            # target-loss hints (NaN: none)
         self.fitted = self._no_fit(max_jobs)
         self.warm = self._no_fit(max_jobs)
 
@@ -282,8 +298,13 @@ class OracleScheduler:
         for i, j in enumerate(job_ids):
             self.s_set[j], self.w_set[j] = float(s[i]), float(w[i])
 
+    def set_target_loss(self, job_ids, targets):
+        for i, j in enumerate(job_ids):
+            self.target[j] = float(targets[i])
+
     def remove_jobs(self, job_ids):
         for j in job_ids:
+            self.target[j] = np.nan
             self.window[j].clear()
             self.k_last[j] = -1
             self.m_seen[j] = -np.inf
@@ -310,7 +331,8 @@ class OracleScheduler:
         s, w = self.time_model()
         out = schedule(offsets, losses, self.m_seen, s, w, epoch_seconds, total_cores, self.cap,
                        self.gamma, self.lm_trials, threads, k_last=self.k_last,
-                       warm=self.warm if self.warm_start else None)
+                       warm=self.warm if self.warm_start else None, envelope=self.envelope,
+                       target_loss=self.target if np.isfinite(self.target).any() else None)
         H = np.diff(offsets)
         self.fitted = dict(valid=out["mask"].copy(), p=out["both"].copy(), K=self.k_last.copy(),
                            span=np.maximum(H - 1, 1).astype(np.float64), M=out["M"].copy())

@@ -593,7 +593,38 @@ JobFit fit_job(const double* loss, int64_t H, double m_seen, const Settings& cfg
 // of the n-th core is g(n) = R(n) - R(n-1), evaluated in a form without cancellation,
 // clamped to +0 where it is not a positive finite number and forced non-increasing in n.
 // ---------------------------------------------------------------------------------
-void job_gains(const JobFit& fit, double s, double w, double T, int cap, double* g) {
+//
+// Two options, both off unless asked for:
+// envelope - where the fitted curve is not convex ahead of the newest point, R(n) is not concave
+//   and its differences may rise with n.  The default makes the row non-increasing with a running
+//   minimum.  With `envelope` the row becomes the slopes of the upper concave envelope of the
+//   points (n, R(n)), n = 0..cap, R(n) = sum of the clamped differences: the smallest concave
+//   function that is nowhere below R (the function a greedy, one-core-at-a-time allocation is
+//   exact for).
+// reduction_cap - a user's hint of the loss the job is expected to end at (Conclusion,
+//   "Non-convex optimization": hints of the target loss against over-estimated reductions).  The
+//   job cannot be predicted to fall below its target: with newest loss l and target tau the
+//   reduction is capped at max(l - tau, 0) / M, i.e. g(n) <- min(g(n), cap left after n-1 cores).
+void upper_concave_envelope(int cap, const double* R /* cap + 1 */, double* slopes /* cap */) {
+    std::vector<int> hull;   // indices of the envelope's vertices, left to right
+    for (int n = 0; n <= cap; ++n) {
+        while (hull.size() >= 2) {
+            const int a = hull[hull.size() - 2], b = hull.back();
+            // b lies on or below the chord a -> n: it is no vertex
+            if ((R[b] - R[a]) * (double)(n - b) <= (R[n] - R[b]) * (double)(b - a)) hull.pop_back();
+            else break;
+        }
+        hull.push_back(n);
+    }
+    for (size_t v = 1; v < hull.size(); ++v) {
+        const int a = hull[v - 1], b = hull[v];
+        const double slope = (R[b] - R[a]) / (double)(b - a);
+        for (int n = a + 1; n <= b; ++n) slopes[n - 1] = slope;
+    }
+}
+
+void job_gains(const JobFit& fit, double s, double w, double T, int cap, double* g, bool envelope = false,
+               double reduction_cap = kInf) {
     for (int n = 0; n < cap; ++n) g[n] = 0.0;
     const bool predicts = fit.status == ST_FITTED || fit.status == ST_SHORT || fit.status == ST_NEW ||
                           fit.status == ST_FIT_FAILED;
@@ -623,10 +654,27 @@ void job_gains(const JobFit& fit, double s, double w, double T, int cap, double*
             R_prev = R;
         }
         if (!(std::isfinite(gain) && gain > 0.0)) gain = 0.0;
-        if (n >= 2 && gain > g[n - 2]) gain = g[n - 2];
+        if (!envelope && n >= 2 && gain > g[n - 2]) gain = g[n - 2];
         g[n - 1] = gain;
         X_prev = X;
         den_prev = den;
+    }
+    if (envelope) {
+        bool rises = false;
+        for (int n = 1; n < cap; ++n) rises = rises || g[n] > g[n - 1];
+        if (rises) {   // a non-increasing row is its own envelope
+            std::vector<double> R(cap + 1, 0.0);
+            for (int n = 1; n <= cap; ++n) R[n] = R[n - 1] + g[n - 1];
+            upper_concave_envelope(cap, R.data(), g);
+        }
+    }
+    if (reduction_cap < kInf) {
+        double before = 0.0;   // uncapped reduction of the first n - 1 cores
+        for (int n = 1; n <= cap; ++n) {
+            const double left = reduction_cap - before;
+            before += g[n - 1];
+            g[n - 1] = left > 0.0 ? std::min(g[n - 1], left) : 0.0;
+        }
     }
 }
 
@@ -749,7 +797,7 @@ int oracle_predict_warm(int64_t n_jobs, const int64_t* offsets, const double* lo
                         double* out_S, int32_t* out_status, int32_t* out_evals, double* out_M, double* out_gain,
                         const int64_t* k_last, const uint8_t* warm_valid, const double* warm_p,
                         const int64_t* warm_K, const double* warm_span, const double* warm_M, double* out_both,
-                        uint8_t* out_mask) {
+                        uint8_t* out_mask, int32_t envelope, const double* target_loss) {
     Settings cfg;
     cfg.gamma = gamma;
     cfg.lm_trials = lm_trials;
@@ -785,7 +833,12 @@ int oracle_predict_warm(int64_t n_jobs, const int64_t* offsets, const double* lo
             out_evals[2 * j + 1] = fit.evals[1];
         }
         if (out_M) out_M[j] = fit.M;
-        if (out_gain) job_gains(fit, s[j], w[j], epoch_seconds, cap, out_gain + (int64_t)j * cap);
+        if (out_gain) {
+            double reduction_cap = kInf;   // a target-loss hint: nothing is gained below the target
+            if (target_loss && std::isfinite(target_loss[j]) && H >= 1 && fit.M > 0.0)
+                reduction_cap = std::max(losses[lo + H - 1] - target_loss[j], 0.0) / fit.M;
+            job_gains(fit, s[j], w[j], epoch_seconds, cap, out_gain + (int64_t)j * cap, envelope != 0, reduction_cap);
+        }
     }
     return 0;
 }
@@ -796,7 +849,7 @@ int oracle_predict(int64_t n_jobs, const int64_t* offsets, const double* losses,
                    double* out_S, int32_t* out_status, int32_t* out_evals, double* out_M, double* out_gain) {
     return oracle_predict_warm(n_jobs, offsets, losses, m_seen, s, w, epoch_seconds, cap, gamma, lm_trials, threads,
                                out_family, out_params, out_S, out_status, out_evals, out_M, out_gain, nullptr,
-                               nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+                               nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, nullptr);
 }
 
 // Step 4 alone on given gain rows.  Returns cores handed out.
@@ -822,6 +875,9 @@ void oracle_time_model(int64_t n_jobs, const double* cnt, const double* su, cons
 }
 
 // ---- hooks that exist only so tests can pin the pieces above ----
+
+// Slopes of the upper concave envelope of (n, R[n]), n = 0..cap.
+void oracle_envelope(int32_t cap, const double* R, double* out_slopes) { upper_concave_envelope(cap, R, out_slopes); }
 
 // Value and Jacobian of a family (0 sublinear, 1 exponential) at x.  Returns 0 if undefined there.
 int oracle_family_eval(int32_t family, const double* p, double x, double* f, double* jac) {

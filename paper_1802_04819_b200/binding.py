@@ -13,12 +13,14 @@ JOB_INACTIVE, JOB_FITTED, JOB_SHORT, JOB_NEW, JOB_FIT_FAILED, JOB_FLAT, JOB_NONF
 P_GAMMA, P_LM_TRIALS, P_MAX_CORES_PER_JOB, P_MIN_FIT_POINTS, P_FIT_SLICE_BYTES, P_WARM_START = 1, 2, 3, 4, 5, 6
 P_FIT_CLUSTER_JOBS = 7
 P_EPOCH_GRAPH = 8
+P_GAIN_ENVELOPE = 9
 W_OVERSUBSCRIBED, W_UNDERFILLED = 1, 2
 
 EXPORTED_SYMBOLS = [
     "slaq_create", "slaq_create_in", "slaq_workspace_bytes", "slaq_destroy", "slaq_last_error", "slaq_set_stream",
     "slaq_set_param", "slaq_get_param", "slaq_append_losses", "slaq_append_losses_ex", "slaq_load_histories",
-    "slaq_load_histories_packed", "slaq_set_time_model", "slaq_remove_jobs", "slaq_schedule", "slaq_schedule_device",
+    "slaq_load_histories_packed", "slaq_set_time_model", "slaq_set_target_loss", "slaq_remove_jobs", "slaq_schedule",
+    "slaq_schedule_device",
     "slaq_get_predictions", "slaq_get_normalised", "slaq_get_time_model", "slaq_get_fit_state",
     "slaq_set_fit_state", "slaq_set_gains", "slaq_allocate_only",
     "slaq_get_stats", "slaq_get_fit_phase_cycles", "slaq_export_state_bytes", "slaq_export_state",
@@ -72,6 +74,7 @@ def load_library(variant: str | None = None):
         "slaq_load_histories": (c_int, [vp, c_int32, vp, vp, vp, vp, vp]),
         "slaq_load_histories_packed": (c_int, [vp, c_int32, vp, vp, vp, vp, vp]),
         "slaq_set_time_model": (c_int, [vp, c_int32, vp, vp, vp]),
+        "slaq_set_target_loss": (c_int, [vp, c_int32, vp, vp]),
         "slaq_remove_jobs": (c_int, [vp, c_int32, vp]),
         "slaq_schedule": (c_int, [vp, c_double, c_int64, vp]),
         "slaq_schedule_device": (c_int, [vp, c_double, c_int64, vp]),
@@ -215,6 +218,10 @@ class Scheduler:
     def set_time_model(self, job_ids, s, w):
         ids, s, w = _arr(job_ids, np.int32), _arr(s, np.float64), _arr(w, np.float64)
         return self._check(self._lib.slaq_set_time_model(self._h, ids.size, _ptr(ids), _ptr(s), _ptr(w)))
+
+    def set_target_loss(self, job_ids, targets):
+        ids, t = _arr(job_ids, np.int32), _arr(targets, np.float64)
+        return self._check(self._lib.slaq_set_target_loss(self._h, ids.size, _ptr(ids), _ptr(t)))
 
     def remove_jobs(self, job_ids):
         ids = _arr(job_ids, np.int32)

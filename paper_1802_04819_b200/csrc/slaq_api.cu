@@ -44,6 +44,7 @@ size_t layout(slaq_handle* h, char* base, int32_t J, int32_t Hmax, int32_t cap) 
     job.s_set = b.take<double>(Js);
     job.w_set = b.take<double>(Js);
     job.last_alloc = b.take<int32_t>(Js);
+    job.target = b.take<double>(Js);
     FitArrays fit;
     fit.status = b.take<int32_t>(Js);
     fit.family = b.take<int8_t>(Js);
@@ -141,6 +142,7 @@ __global__ void init_jobs_kernel(JobArrays job, FitArrays fit, double* ring, int
     job.s_set[j] = CUDART_NAN;
     job.w_set[j] = CUDART_NAN;
     job.last_alloc[j] = 1;
+    job.target[j] = CUDART_NAN;
     fit.status[j] = SLAQ_JOB_INACTIVE;
     fit.family[j] = -1;
     for (int k = 0; k < 4; ++k) fit.params[4 * (size_t)j + k] = CUDART_NAN;
@@ -272,6 +274,14 @@ __global__ void set_time_kernel(JobArrays job, int max_jobs, int n, const int32_
     if (j < 0 || j >= max_jobs) return;
     job.s_set[j] = s[i];
     job.w_set[j] = w[i];
+}
+
+__global__ void set_target_kernel(JobArrays job, int max_jobs, int n, const int32_t* ids, const double* targets) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int j = ids[i];
+    if (j < 0 || j >= max_jobs) return;
+    job.target[j] = targets[i];
 }
 
 // Kernels and copies go to the current device: it must be the one the handle lives on.
@@ -579,7 +589,7 @@ std::vector<long long> epoch_key(const slaq_handle* h, double T, int64_t want, i
     std::memcpy(&g_bits, &h->gamma, sizeof g_bits);
     return {t_bits, (long long)want, floor_units, (long long)(uintptr_t)d_out, only_allocate ? 1 : 0, h->n_active,
             h->max_cores, h->lm_trials, h->min_fit_points, h->warm_start ? 1 : 0, (long long)h->fit_slice_bytes,
-            (long long)h->fit_cluster_jobs, g_bits};
+            (long long)h->fit_cluster_jobs, g_bits, h->gain_envelope ? 1 : 0};
 }
 
 int run_epoch(slaq_handle* h, double T, int64_t C, int32_t* d_out, bool only_allocate) {
@@ -757,6 +767,10 @@ int slaq_set_param(slaq_t* h, int key, double value) {
             if (!(value == -1.0 || value == 0.0 || value == 1.0)) return fail(h, SLAQ_E_ARG, "epoch graph must be -1, 0 or 1");
             h->epoch_graph = (int)value;
             return SLAQ_OK;
+        case SLAQ_P_GAIN_ENVELOPE:
+            if (!(value == 0.0 || value == 1.0)) return fail(h, SLAQ_E_ARG, "gain envelope must be 0 or 1");
+            h->gain_envelope = value != 0.0;
+            return SLAQ_OK;
         default:
             return fail(h, SLAQ_E_ARG, "unknown parameter key");
     }
@@ -773,6 +787,7 @@ int slaq_get_param(const slaq_t* h, int key, double* out_value) {
         case SLAQ_P_WARM_START: *out_value = h->warm_start ? 1.0 : 0.0; return SLAQ_OK;
         case SLAQ_P_FIT_CLUSTER_JOBS: *out_value = (double)h->fit_cluster_jobs; return SLAQ_OK;
         case SLAQ_P_EPOCH_GRAPH: *out_value = (double)h->epoch_graph; return SLAQ_OK;
+        case SLAQ_P_GAIN_ENVELOPE: *out_value = h->gain_envelope ? 1.0 : 0.0; return SLAQ_OK;
         default: return SLAQ_E_ARG;
     }
 }
@@ -814,6 +829,24 @@ int slaq_set_time_model(slaq_t* h, int32_t n, const int32_t* job_ids, const doub
                                                                     h->stage.times);
     CK(cudaGetLastError(), "time law kernel");
     CK(cudaStreamSynchronize(st), "time law");
+    return SLAQ_OK;
+}
+
+int slaq_set_target_loss(slaq_t* h, int32_t n, const int32_t* job_ids, const double* targets) {
+    if (!h) return SLAQ_E_ARG;
+    if (n > 0 && !targets) return fail(h, SLAQ_E_ARG, "targets is null");
+    const int rc = check_ids(h, n, job_ids, true);
+    if (rc) return rc;
+    for (int32_t i = 0; i < n; ++i)
+        if (std::isinf(targets[i])) return fail(h, SLAQ_E_NONFINITE, "a target loss must be a number, or NaN for none");
+    if (n == 0) return SLAQ_OK;
+    cudaStream_t st = h->stream;
+    CK(cudaMemcpyAsync(h->stage.ids, job_ids, sizeof(int32_t) * n, cudaMemcpyHostToDevice, st), "copy job ids");
+    CK(cudaMemcpyAsync(h->stage.losses, targets, sizeof(double) * n, cudaMemcpyHostToDevice, st), "copy targets");
+    const int threads = 256;
+    set_target_kernel<<<(n + threads - 1) / threads, threads, 0, st>>>(h->job, h->max_jobs, n, h->stage.ids, h->stage.losses);
+    CK(cudaGetLastError(), "target kernel");
+    CK(cudaStreamSynchronize(st), "targets");
     return SLAQ_OK;
 }
 
@@ -1103,7 +1136,7 @@ struct StateHeader {
 // because every block's size is a multiple of 8 (max_jobs is padded to a multiple of 8 entries).
 struct StateLayout {
     size_t J8;             // max_jobs rounded up to a multiple of 8
-    size_t off_count, off_k_last, off_m_seen, off_tm, off_s_set, off_w_set, off_last_alloc;
+    size_t off_count, off_k_last, off_m_seen, off_tm, off_s_set, off_w_set, off_last_alloc, off_target;
     size_t off_both, off_mask, off_k_fit, off_span, off_largest;
     size_t off_warm_p, off_warm_mask, off_warm_k, off_warm_span, off_warm_scale;
     size_t off_offsets, off_losses, bytes;
@@ -1121,6 +1154,7 @@ StateLayout state_layout(int32_t max_jobs, int64_t total_points) {
     L.off_s_set = take(8 * L.J8);
     L.off_w_set = take(8 * L.J8);
     L.off_last_alloc = take(4 * L.J8);
+    L.off_target = take(8 * L.J8);
     L.off_both = take(8 * 8 * L.J8);
     L.off_mask = take(L.J8);
     L.off_k_fit = take(8 * L.J8);
@@ -1190,6 +1224,7 @@ int slaq_export_state(slaq_t* h, void* out_blob, size_t capacity) {
     CK(cudaMemcpyAsync(blob + L.off_s_set, h->job.s_set, 8 * J, down, st), "export state");
     CK(cudaMemcpyAsync(blob + L.off_w_set, h->job.w_set, 8 * J, down, st), "export state");
     CK(cudaMemcpyAsync(blob + L.off_last_alloc, h->job.last_alloc, 4 * J, down, st), "export state");
+    CK(cudaMemcpyAsync(blob + L.off_target, h->job.target, 8 * J, down, st), "export state");
     CK(cudaMemcpyAsync(blob + L.off_both, h->fit.both, 8 * 8 * J, down, st), "export state");
     CK(cudaMemcpyAsync(blob + L.off_mask, h->fit.mask, J, down, st), "export state");
     CK(cudaMemcpyAsync(blob + L.off_k_fit, h->fit.k_fit, 8 * J, down, st), "export state");
@@ -1271,6 +1306,7 @@ int slaq_import_state(slaq_t* h, const void* blob_in, size_t bytes) {
     CK(cudaMemcpyAsync(h->job.s_set, blob + L.off_s_set, 8 * J, up, st), "import state");
     CK(cudaMemcpyAsync(h->job.w_set, blob + L.off_w_set, 8 * J, up, st), "import state");
     CK(cudaMemcpyAsync(h->job.last_alloc, blob + L.off_last_alloc, 4 * J, up, st), "import state");
+    CK(cudaMemcpyAsync(h->job.target, blob + L.off_target, 8 * J, up, st), "import state");
     CK(cudaMemcpyAsync(h->fit.both, blob + L.off_both, 8 * 8 * J, up, st), "import state");
     CK(cudaMemcpyAsync(h->fit.mask, blob + L.off_mask, J, up, st), "import state");
     CK(cudaMemcpyAsync(h->fit.k_fit, blob + L.off_k_fit, 8 * J, up, st), "import state");

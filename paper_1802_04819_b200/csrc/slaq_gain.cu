@@ -96,10 +96,41 @@ __device__ double raw_gain(const Curve& c, int n) {
     return (finite_d(gain) && gain > 0.0) ? gain : 0.0;
 }
 
+// Slopes of the upper concave envelope of the points (n, R(n)), n = 0..cap, written over the row
+// (row[n-1] holds the clamped difference R(n) - R(n-1) on entry).  One thread walks the row: a stack
+// of envelope vertices, a point leaving it when it lies on or below the chord from the vertex
+// before it to the new point.  Rows that need this are rare (the fit is not convex ahead).
+__device__ void envelope_of_row(double* row, int cap, unsigned short* stack) {
+    double run = 0.0;
+    for (int n = 1; n <= cap; ++n) {   // differences -> R(n) in place
+        run += row[n - 1];
+        row[n - 1] = run;
+    }
+    auto R = [&](int n) { return n == 0 ? 0.0 : row[n - 1]; };
+    int top = 0;
+    for (int n = 0; n <= cap; ++n) {
+        while (top >= 2) {
+            const int a = stack[top - 2], b = stack[top - 1];
+            if ((R(b) - R(a)) * (double)(n - b) <= (R(n) - R(b)) * (double)(b - a)) --top;
+            else break;
+        }
+        stack[top++] = (unsigned short)n;
+    }
+    // slopes, written from the right so that R(a) of each segment is still in place when it is read
+    for (int v = top - 1; v >= 1; --v) {
+        const int a = stack[v - 1], b = stack[v];
+        const double slope = (R(b) - R(a)) / (double)(b - a);
+        for (int n = b; n > a; --n) row[n - 1] = slope;
+    }
+}
+
+// options: bit 0 = rows become the slopes of the concave envelope of R(n) instead of a running minimum
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int first_unit, double* __restrict__ gain,
-            unsigned long long* __restrict__ hist0) {
+            unsigned long long* __restrict__ hist0, int options) {
     __shared__ unsigned int sh_hist[kRadixBins];
+    __shared__ unsigned short sh_stack[kWarpsPerBlock][kMaxCoresLimit + 1];
+    const bool envelope = (options & 1) != 0;
     for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) sh_hist[i] = 0;
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -125,6 +156,78 @@ gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int f
                 c.kind = status == SLAQ_JOB_FITTED ? (int)fit.family[j] : 2;
                 c.step_scale = T * c.w * c.inv_span;
             }
+        }
+        // A target-loss hint caps the predicted reduction at (newest loss - target) / M.
+        double reduction_cap = CUDART_INF;
+        if (c.kind != 3) {
+            const double target = job.target[j];
+            const double M = fit.largest[j];
+            if (finite_d(target) && M > 0.0) {
+                const int ring = job.cap[j];
+                int at = job.head[j] - 1;
+                at += at < 0 ? ring : 0;
+                const double newest = index_ok(at, ring, kErrStorage, job.err_word) ? job.row[j][at] : 0.0;
+                reduction_cap = __ddiv_rn(fmax(newest - target, 0.0), M);
+            }
+        }
+        if (envelope || reduction_cap < CUDART_INF) {
+            // General path (options in use): the row is completed in memory first, then read back for the cap
+            // and the histogram.
+            double* row = gain + (size_t)j * cap;
+            double prev = CUDART_INF, carry_min = CUDART_INF;
+            int rises = 0;
+            for (int base = 0; base < cap; base += 32) {
+                const int n = base + lane + 1;
+                double g = CUDART_INF;
+                if (n <= cap) g = c.kind == 3 ? 0.0 : raw_gain(c, n);
+                if (envelope) {
+                    double left = __shfl_up_sync(kFull, g, 1);
+                    if (lane == 0) left = prev;
+                    rises |= (n <= cap && g > left) ? 1 : 0;
+                    prev = __shfl_sync(kFull, g, 31);
+                } else {
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const double up = __shfl_up_sync(kFull, g, o);
+                        if (lane >= o) g = fmin(g, up);
+                    }
+                    g = fmin(g, carry_min);
+                    carry_min = __shfl_sync(kFull, g, 31);
+                }
+                if (n <= cap && index_ok((long long)j * cap + (n - 1), (long long)max_jobs * cap, kErrGain, job.err_word))
+                    row[n - 1] = g;
+            }
+            __syncwarp();
+            if (envelope && __any_sync(kFull, rises)) {
+                if (lane == 0) envelope_of_row(row, cap, sh_stack[warp]);
+                __syncwarp();
+            }
+            double before = 0.0;   // uncapped reduction of the cores before this chunk
+            for (int base = 0; base < cap; base += 32) {
+                const int n = base + lane + 1;
+                double g = n <= cap ? row[n - 1] : 0.0;
+                if (reduction_cap < CUDART_INF) {
+                    double incl = g;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const double up = __shfl_up_sync(kFull, incl, o);
+                        if (lane >= o) incl += up;
+                    }
+                    const double left = reduction_cap - (before + (incl - g));
+                    before += __shfl_sync(kFull, incl, 31);
+                    g = left > 0.0 ? fmin(g, left) : 0.0;
+                    if (n <= cap) row[n - 1] = g;
+                }
+                const bool counted = active && n <= cap && n >= first_unit;
+                const unsigned digit = (unsigned)((unsigned long long)__double_as_longlong(g) >> (64 - kRadixBits));
+                const unsigned live = __ballot_sync(kFull, counted);
+                if (counted) {
+                    const unsigned peers = __match_any_sync(live, digit);
+                    if ((int)(__ffs(peers) - 1) == lane && index_ok(digit, kRadixBins, kErrBin, job.err_word))
+                        atomicAdd(&sh_hist[digit], (unsigned)__popc(peers));
+                }
+            }
+            continue;
         }
         double carry = CUDART_INF;   // running minimum of the gains before this chunk
         for (int base = 0; base < cap; base += 32) {
@@ -175,7 +278,8 @@ int launch_gain(slaq_handle* h, double epoch_seconds, int first_unit) {
     const int needed = (h->max_jobs + kWarpsPerBlock - 1) / kWarpsPerBlock;
     if (blocks > needed) blocks = needed;
     gain_kernel<<<blocks, kWarpsPerBlock * 32, 0, h->stream>>>(h->job, h->fit, h->max_jobs, h->max_cores, epoch_seconds,
-                                                              first_unit, h->gain, h->scratch.hist);
+                                                              first_unit, h->gain, h->scratch.hist,
+                                                              h->gain_envelope ? 1 : 0);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         h->err = std::string("gain kernel launch: ") + cudaGetErrorString(e);

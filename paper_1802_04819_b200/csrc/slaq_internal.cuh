@@ -34,6 +34,7 @@ struct JobArrays {
     double* s_set;       // fixed time law (NaN: use the estimate)
     double* w_set;
     int32_t* last_alloc; // core count of the last epoch (1 before any)
+    double* target;      // hint of the loss the job will end at (NaN: none)
     // extents, read by the bounds build only
     int32_t max_jobs;
     const double* ring_lo;     // the ring pool [ring_lo, ring_hi)
@@ -109,6 +110,7 @@ struct slaq_handle {
     int32_t lm_trials = 20, min_fit_points = 4;
     size_t fit_slice_bytes = 13824;       // shared memory one warp of the fit kernel may use (parked sums, up to 52 rows of 32 points, a spare row)
     bool warm_start = false;              // fits start from the last epoch's parameters where there are some
+    bool gain_envelope = false;           // gain rows are slopes of the concave envelope of R(n), not a running minimum
     int64_t fit_cluster_jobs = 0;         // active jobs the lanes per job are chosen for (0: this handle's own)
     cudaStream_t stream = nullptr;
     bool owns_ws = false;

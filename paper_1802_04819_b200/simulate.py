@@ -38,14 +38,34 @@ def draw_trace(n_jobs=160, mean_gap=15.0, seed=0):
     return dict(arrive=arrive, family=family, params=params, s=s, w=w)
 
 
+def loss_groups(norm_loss):
+    """Positions (into `norm_loss`) of the quarter of the jobs with the highest normalised loss, of the next
+    quarter, and of the lower half - the three groups of the paper's allocation-by-loss-group figure."""
+    order = np.argsort(-np.asarray(norm_loss), kind="stable")
+    n = order.size
+    q = (n + 3) // 4
+    return order[:q], order[q:min(2 * q, n)], order[min(2 * q, n):]
+
+
 def run(trace, policy="slaq", total_cores=640, max_cores_per_job=64, epoch=3.0, horizon=800.0, max_hist=64,
-        sigma=0.01, target=0.99, seed=1):
+        sigma=0.01, target=0.99, seed=1, scheduler_factory=None, keep_allocations=False):
     """Simulate one policy ("slaq" or "fair").  Returns per-epoch average normalised loss of the running
-    jobs, and per job the time from arrival to 90 % and 95 % loss reduction (NaN if not reached)."""
-    import paper_1802_04819_b200 as slaq
+    jobs, per job the time from arrival to 90 % and 95 % loss reduction (NaN if not reached), and the share
+    of the handed-out cores that went to the running jobs' top quarter / next quarter / lower half by
+    normalised loss, averaged over the epochs with at least four running jobs.
+
+    scheduler_factory(max_jobs, max_hist, max_cores_per_job): what schedules under policy "slaq" (default:
+    this library's ``Scheduler``); it needs append_losses, schedule -> (alloc, status), remove_jobs and close.
+    keep_allocations: also return every epoch's allocation vector."""
     J = trace["arrive"].size
     rng = np.random.default_rng(seed)
-    sched = slaq.Scheduler(J, max_hist, max_cores_per_job) if policy == "slaq" else None
+    if policy != "slaq":
+        sched = None
+    elif scheduler_factory is not None:
+        sched = scheduler_factory(J, max_hist, max_cores_per_job)
+    else:
+        import paper_1802_04819_b200 as slaq
+        sched = slaq.Scheduler(J, max_hist, max_cores_per_job)
     fam, par, s, w = trace["family"], trace["params"], trace["s"], trace["w"]
     first = np.array([_curve(fam[j], par[j], 0.0) for j in range(J)])
     last = np.array([_curve(fam[j], par[j], 1e9) for j in range(J)])
@@ -55,6 +75,7 @@ def run(trace, policy="slaq", total_cores=640, max_cores_per_job=64, epoch=3.0, 
     state = np.zeros(J, dtype=np.int8)            # 0 not arrived, 1 running, 2 finished
     reached = {0.90: np.full(J, np.nan), 0.95: np.full(J, np.nan)}
     avg_loss, t = [], 0.0
+    shares, allocations = [], []
 
     def norm_loss(j):
         return (_curve(fam[j], par[j], float(k_done[j])) - last[j]) / (first[j] - last[j])
@@ -80,6 +101,12 @@ def run(trace, policy="slaq", total_cores=640, max_cores_per_job=64, epoch=3.0, 
                 for j in running[:max(0, extra)]:
                     if alloc[j] < max_cores_per_job:
                         alloc[j] += 1
+            if keep_allocations:
+                allocations.append(alloc.copy())
+            if running.size >= 4 and alloc[running].sum() > 0:
+                before = np.array([norm_loss(j) for j in running])
+                handed = float(alloc[running].sum())
+                shares.append([alloc[running][g].sum() / handed for g in loss_groups(before)])
             # run the epoch: iterations each job completes on its cores, reported one by one
             n = np.maximum(alloc[running], 0)
             per_iter = s[running] + w[running] / np.maximum(n, 1)
@@ -107,7 +134,13 @@ def run(trace, policy="slaq", total_cores=640, max_cores_per_job=64, epoch=3.0, 
         t += epoch
     if sched is not None:
         sched.close()
-    return dict(avg_loss=np.array(avg_loss), t90=reached[0.90], t95=reached[0.95], finished=int((state == 2).sum()))
+    share = np.mean(np.array(shares), axis=0) if shares else np.full(3, np.nan)
+    out = dict(avg_loss=np.array(avg_loss), t90=reached[0.90], t95=reached[0.95], finished=int((state == 2).sum()),
+               core_share_top_quarter=float(share[0]), core_share_next_quarter=float(share[1]),
+               core_share_lower_half=float(share[2]))
+    if keep_allocations:
+        out["allocations"] = allocations
+    return out
 
 
 def compare(n_jobs=160, horizon=800.0, total_cores=320, seed=1):
@@ -120,6 +153,9 @@ def compare(n_jobs=160, horizon=800.0, total_cores=320, seed=1):
         t90_slaq=float(np.nanmean(a["t90"])), t90_fair=float(np.nanmean(b["t90"])),
         t95_slaq=float(np.nanmean(a["t95"])), t95_fair=float(np.nanmean(b["t95"])),
         finished_slaq=a["finished"], finished_fair=b["finished"],
+        # share of the cores by loss group (the paper's cluster: 60 % to the top quarter, 22 % to the lower half)
+        core_share_top_quarter_slaq=a["core_share_top_quarter"], core_share_lower_half_slaq=a["core_share_lower_half"],
+        core_share_top_quarter_fair=b["core_share_top_quarter"], core_share_lower_half_fair=b["core_share_lower_half"],
     )
 
 

@@ -51,6 +51,10 @@ MUTATIONS = [
     ("warm start: stretch of the window inverted", "const double r = D.span / warm->span;",
      "const double r = warm->span / D.span;"),
     ("warm start: an unusable carried point is kept", "startedI = rI.ok;", "startedI = true;"),
+    ("envelope: chord test inverted", "<= (R[n] - R[b]) * (double)(b - a)) hull.pop_back();",
+     ">= (R[n] - R[b]) * (double)(b - a)) hull.pop_back();"),
+    ("target hint: every gain capped by the whole allowance", "const double left = reduction_cap - before;",
+     "const double left = reduction_cap;"),
     ("fallback: mean change without the weights", "num += (long double)D.w[i] * dnorm;", "num += (long double)dnorm;"),
     ("fallback: no cap at the newest level", "out.r_cap = D.y[H - 1] > 0.0 ? D.y[H - 1] : kInf;", "out.r_cap = kInf;"),
     ("fallback: a window of four points or more without a fit predicts nothing",
@@ -76,6 +80,8 @@ PINS = [
     lambda m: t_warm.test_an_unusable_carried_point_falls_back_to_the_first_guess(m),
     lambda m: t_fit.test_windows_on_which_no_family_can_start_use_the_mean_normalised_change(m),
     lambda m: t_fit.test_the_cap_of_the_fallback_is_the_newest_normalised_level(m),
+    lambda m: t_gains.test_concave_envelope_equals_its_definition(m),
+    lambda m: t_gains.test_target_loss_hint_caps_the_predicted_reduction(m),
 ]
 
 
