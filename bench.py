@@ -298,6 +298,49 @@ def run_gpu(args):
     warm_s = (time.perf_counter() - t0) / e2e_steps
     assert int(h_alloc.sum()) == wl.total_cores
 
+    # ---- one cluster sharded over several handles (the multi-GPU protocol: a histogram sum per radix pass and one
+    # exchange of tie counts).  With one GPU: the same 100,000 jobs as two shards of 50,000 on this GPU, sums done
+    # locally - the protocol's overhead against the single handle.  With N GPUs: the N partitions as ONE cluster of
+    # N x 100,000 jobs, one shard per rank, sums over NCCL.  Reported beside the headline, never instead of it. ----
+    sharded = None
+    try:
+        sched.set_param(slaq.binding.P_WARM_START, 0)
+        sched.set_param(slaq.binding.P_LM_TRIALS, 20)
+        reps = max(3, min(args.steps, 20))
+        if world == 1:
+            half = J // 2
+            shards = []
+            for lo, hi in ((0, half), (half, J)):
+                sh = slaq.Scheduler(hi - lo, wl.max_hist, cap, stream=stream)
+                sh.load_histories(np.arange(hi - lo, dtype=np.int32), wl.offsets[lo:hi + 1] - wl.offsets[lo],
+                                  wl.losses[wl.offsets[lo]:wl.offsets[hi]], wl.k_last[lo:hi], wl.m_seen[lo:hi],
+                                  packed=args.cfg == CFG)
+                sh.set_time_model(np.arange(hi - lo, dtype=np.int32), wl.s[lo:hi], wl.w[lo:hi])
+                shards.append(sh)
+            exchange, cluster_cores = slaq.LocalExchange(), wl.total_cores
+        else:
+            shards, exchange, cluster_cores = [sched], slaq.ProcessGroupExchange(), world * wl.total_cores
+        for _ in range(args.warmup):
+            parts = slaq.schedule_sharded(shards, exchange, wl.epoch_seconds, cluster_cores)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            parts = slaq.schedule_sharded(shards, exchange, wl.epoch_seconds, cluster_cores)
+        torch.cuda.synchronize()
+        shard_ms = (time.perf_counter() - t0) / reps * 1e3
+        handed = sum(int(p.sum()) for p in parts)
+        same = bool(world > 1 or np.array_equal(np.concatenate(parts), alloc_dev))
+        sharded = {"ms_per_epoch": max_over_ranks([shard_ms], device="cuda")[0], "shards": len(shards) * world,
+                   "jobs_in_the_cluster": J * world, "epochs_timed": reps, "cores_handed_out_by_this_rank": handed,
+                   "equals_single_handle": same if world == 1 else None,
+                   "what": "wall clock per epoch of schedule_sharded (host waits once, for the allocation); with one GPU "
+                           "two local shards of the benchmark's jobs, with N GPUs one shard per rank over NCCL"}
+        if world == 1:
+            for sh in shards:
+                sh.close()
+    except Exception as err:   # the headline must not depend on this leg
+        sharded = {"error": f"{type(err).__name__}: {err}"}
+
     ms_step, e2e_ms, warm_ms = max_over_ranks([ms_step, e2e_s * 1e3, warm_s * 1e3], device="cuda")
 
     if rank == 0:
@@ -335,6 +378,7 @@ def run_gpu(args):
                            "steps": e2e_steps,
                            "what": "the end-to-end loop with SLAQ_P_WARM_START = 1: every family starts from the "
                                    "curve it ended with last epoch and runs 5 trials instead of 20"},
+            "sharded_cluster": sharded,
             "gpu_launches": launches,
             "stage_ms": {"fit": float(stage[0]), "gain": float(stage[1]), "alloc": float(stage[2])},
             "roofline": {"bound": "alu", "kernel": "fit_kernel", "achieved": achieved, "peak": peak_tflops,

@@ -395,6 +395,11 @@ int slaq_get_fit_phase_cycles(slaq_t* h, int64_t* out_cycles);
  * d_hist is device memory of 2048 uint64 owned by the caller; out_alloc is a host array of max_jobs
  * entries.  The result equals slaq_schedule on one handle holding all jobs.  All calls are ordered on
  * the handle's stream; slaq_shard_count and slaq_shard_finalise return after the stream has finished.
+ * slaq_shard_count_device / slaq_shard_finalise_device are the same two steps without the host in
+ * between: the first leaves the shard's tie count in device memory of the caller (one int64,
+ * stream-ordered, no wait), the second reads ties_before from device memory (one int64 that the
+ * caller's collective left there, ordered on the handle's stream) - a whole sharded epoch then
+ * waits for the device once, when the allocation is copied out.
  */
 int slaq_get_active_count(slaq_t* h, int32_t* out_active);
 int slaq_shard_predict(slaq_t* h, double epoch_seconds, int32_t with_floor);
@@ -403,6 +408,8 @@ int slaq_shard_pick(slaq_t* h, int32_t pass, int64_t want);
 int slaq_shard_pass(slaq_t* h, int32_t pass);
 int slaq_shard_count(slaq_t* h, int64_t* out_local_ties);
 int slaq_shard_finalise(slaq_t* h, int64_t ties_before, int32_t* out_alloc);
+int slaq_shard_count_device(slaq_t* h, int64_t* d_out_local_ties);
+int slaq_shard_finalise_device(slaq_t* h, const int64_t* d_ties_before, int32_t* out_alloc);
 
 /*
  * The allocation step for callers that must not allocate device memory.  (The paper has

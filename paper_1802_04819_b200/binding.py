@@ -25,7 +25,8 @@ EXPORTED_SYMBOLS = [
     "slaq_set_fit_state", "slaq_set_gains", "slaq_allocate_only",
     "slaq_get_stats", "slaq_get_fit_phase_cycles", "slaq_export_state_bytes", "slaq_export_state",
     "slaq_import_state", "slaq_allocate_static", "slaq_get_active_count", "slaq_shard_predict", "slaq_shard_histogram",
-    "slaq_shard_pick", "slaq_shard_pass", "slaq_shard_count", "slaq_shard_finalise",
+    "slaq_shard_pick", "slaq_shard_pass", "slaq_shard_count", "slaq_shard_finalise", "slaq_shard_count_device",
+    "slaq_shard_finalise_device",
 ]
 
 
@@ -98,6 +99,8 @@ def load_library(variant: str | None = None):
         "slaq_shard_pass": (c_int, [vp, c_int32]),
         "slaq_shard_count": (c_int, [vp, POINTER(c_int64)]),
         "slaq_shard_finalise": (c_int, [vp, c_int64, vp]),
+        "slaq_shard_count_device": (c_int, [vp, vp]),
+        "slaq_shard_finalise_device": (c_int, [vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -338,6 +341,16 @@ class Scheduler:
         """SM cycles the fit kernel's warps spent per phase (zeros unless the "clocks" variant is loaded)."""
         out = np.zeros(6, np.int64)
         self._check(self._lib.slaq_get_fit_phase_cycles(self._h, _ptr(out)))
+        return out
+
+    def shard_count_device(self, d_ties):
+        """``d_ties``: torch int64 CUDA tensor of one entry that receives this shard's tie count (no host wait)."""
+        return self._check(self._lib.slaq_shard_count_device(self._h, c_void_p(d_ties.data_ptr())))
+
+    def shard_finalise_device(self, d_ties_before):
+        """``d_ties_before``: torch int64 CUDA tensor of one entry, ordered on the handle's stream."""
+        out = np.empty(self.max_jobs, np.int32)
+        self._check(self._lib.slaq_shard_finalise_device(self._h, c_void_p(d_ties_before.data_ptr()), _ptr(out)))
         return out
 
     def get_stats(self) -> Stats:

@@ -300,8 +300,9 @@ finalise_kernel(const double* __restrict__ gain, const int32_t* __restrict__ cou
                 const SelectState* __restrict__ sel, const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
                 const long long* __restrict__ block_prefix, int32_t* __restrict__ alloc, double* __restrict__ reduction,
                 int32_t* __restrict__ last_alloc, int32_t* __restrict__ out_alloc, long long* counters,
-                long long ties_before, int32_t* err_word) {
+                long long ties_before, const long long* __restrict__ d_ties_before, int32_t* err_word) {
     __shared__ long long sh_pre[kJobsPerBlock];
+    if (d_ties_before) ties_before += *d_ties_before;   // the count held by lower shards, left on the device by the caller
     __shared__ int sh_alloc[kJobsPerBlock];
     const int t = threadIdx.x;
     const int j0 = blockIdx.x * kJobsPerBlock;
@@ -397,7 +398,7 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
     scan_blocks_kernel<<<1, 1024, 0, st>>>(h->scratch.block_eq, blocks);
     finalise_kernel<<<blocks, 256, 0, st>>>(h->gain, h->job.count, J, cap, first_unit - 1, h->scratch.sel, h->scratch.gt,
                                             h->scratch.eq, h->scratch.block_eq, h->alloc, h->reduction,
-                                            h->job.last_alloc, d_out_alloc, h->scratch.counters, 0, h->err_word);
+                                            h->job.last_alloc, d_out_alloc, h->scratch.counters, 0, nullptr, h->err_word);
     launches += 3;
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
@@ -452,13 +453,14 @@ int launch_shard_count(slaq_handle* h, int first_unit, const long long** d_total
     return check_launch(h, "shard count") ? -1 : 2;
 }
 
-int launch_shard_finalise(slaq_handle* h, int first_unit, long long ties_before, int32_t* d_out_alloc) {
+int launch_shard_finalise(slaq_handle* h, int first_unit, long long ties_before, const long long* d_ties_before,
+                          int32_t* d_out_alloc) {
     const int J = h->max_jobs;
     const int blocks = (J + kJobsPerBlock - 1) / kJobsPerBlock;
     finalise_kernel<<<blocks, 256, 0, h->stream>>>(h->gain, h->job.count, J, h->max_cores, first_unit - 1, h->scratch.sel,
                                                    h->scratch.gt, h->scratch.eq, h->scratch.block_eq, h->alloc,
                                                    h->reduction, h->job.last_alloc, d_out_alloc, h->scratch.counters,
-                                                   ties_before, h->err_word);
+                                                   ties_before, d_ties_before, h->err_word);
     return check_launch(h, "shard finalise") ? -1 : 1;
 }
 
@@ -553,7 +555,7 @@ extern "C" int slaq_allocate_static(const double* d_gain, int32_t n_jobs, int32_
     scan_blocks_kernel<<<1, 1024, 0, st>>>(sc->block_eq, blocks);
     finalise_kernel<<<blocks, 256, 0, st>>>(d_gain, sc->every_row_active, J, cap, floor_units, &sc->sel, sc->gt, sc->eq,
                                             sc->block_eq, d_out_alloc, d_out_reduction, sc->cores_now, nullptr,
-                                            sc->counters, 0, nullptr);
+                                            sc->counters, 0, nullptr, nullptr);
     if (cudaGetLastError() != cudaSuccess) return SLAQ_E_CUDA;
     if (total_cores < J) return SLAQ_W_OVERSUBSCRIBED;
     if (total_cores > (long long)J * cap) return SLAQ_W_UNDERFILLED;

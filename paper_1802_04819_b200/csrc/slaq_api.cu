@@ -983,11 +983,33 @@ int slaq_shard_count(slaq_t* h, int64_t* out_local_ties) {
     return SLAQ_OK;
 }
 
+int slaq_shard_count_device(slaq_t* h, int64_t* d_out_local_ties) {
+    if (!h || !d_out_local_ties) return SLAQ_E_ARG;
+    const long long* d_total = nullptr;
+    const int k = launch_shard_count(h, h->shard_first_unit, &d_total);
+    if (k < 0) return SLAQ_E_CUDA;
+    h->last_launches += k;
+    CK(cudaMemcpyAsync(d_out_local_ties, d_total, sizeof(long long), cudaMemcpyDeviceToDevice, h->stream), "export tie count");
+    return SLAQ_OK;
+}
+
+int slaq_shard_finalise_device(slaq_t* h, const int64_t* d_ties_before, int32_t* out_alloc) {
+    if (!h) return SLAQ_E_ARG;
+    if (!out_alloc || !d_ties_before) return fail(h, SLAQ_E_ARG, "out_alloc or d_ties_before is null");
+    const int k = launch_shard_finalise(h, h->shard_first_unit, 0, reinterpret_cast<const long long*>(d_ties_before), nullptr);
+    if (k < 0) return SLAQ_E_CUDA;
+    h->last_launches += k;
+    CK(cudaEventRecord(h->ev[3], h->stream), "event");
+    CK(cudaMemcpyAsync(out_alloc, h->alloc, sizeof(int32_t) * (size_t)h->max_jobs, cudaMemcpyDeviceToHost, h->stream),
+       "copy allocation");
+    return check_device_errors(h);
+}
+
 int slaq_shard_finalise(slaq_t* h, int64_t ties_before, int32_t* out_alloc) {
     if (!h) return SLAQ_E_ARG;
     if (!out_alloc) return fail(h, SLAQ_E_ARG, "out_alloc is null");
     if (ties_before < 0) return fail(h, SLAQ_E_ARG, "ties_before must not be negative");
-    const int k = launch_shard_finalise(h, h->shard_first_unit, ties_before, nullptr);
+    const int k = launch_shard_finalise(h, h->shard_first_unit, ties_before, nullptr, nullptr);
     if (k < 0) return SLAQ_E_CUDA;
     h->last_launches += k;
     CK(cudaEventRecord(h->ev[3], h->stream), "event");

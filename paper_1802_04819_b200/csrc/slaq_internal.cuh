@@ -166,6 +166,7 @@ int launch_time_model(slaq_handle* h, double* d_s, double* d_w);
 int launch_shard_pick(slaq_handle* h, int pass, long long want);
 int launch_shard_pass(slaq_handle* h, int pass, int first_unit);
 int launch_shard_count(slaq_handle* h, int first_unit, const long long** d_total);
-int launch_shard_finalise(slaq_handle* h, int first_unit, long long ties_before, int32_t* d_out_alloc);
+int launch_shard_finalise(slaq_handle* h, int first_unit, long long ties_before, const long long* d_ties_before,
+                          int32_t* d_out_alloc);
 
 }  // namespace slaq

@@ -19,7 +19,9 @@ N_BINS = 2048
 
 
 class LocalExchange:
-    """All shards live in this process."""
+    """All shards live in this process, on the current CUDA device."""
+
+    device = "cuda"
 
     def sum_ints(self, values):
         total = sum(int(v) for v in values)
@@ -32,12 +34,12 @@ class LocalExchange:
         for b in buffers:
             b.copy_(total)
 
-    def gather_ints(self, values):
-        allv = [int(v) for v in values]
-        return [allv] * len(values)
-
-    def ranks(self, n_local):
-        return list(range(n_local))
+    def ties_before(self, ties):
+        """ties: one 1-entry int64 tensor per shard.  Returns per shard the sum over the shards before it."""
+        import torch
+        stacked = torch.cat(ties)
+        before = torch.cumsum(stacked, 0) - stacked
+        return [before[i:i + 1].contiguous() for i in range(len(ties))]
 
 
 class ProcessGroupExchange:
@@ -58,22 +60,30 @@ class ProcessGroupExchange:
         assert len(buffers) == 1
         self.dist.all_reduce(buffers[0], group=self.group)
 
-    def gather_ints(self, values):
+    def ties_before(self, ties):
         import torch
-        world = self.dist.get_world_size(self.group)
-        t = torch.tensor([int(values[0])], dtype=torch.int64, device=self.device)
-        out = [torch.zeros_like(t) for _ in range(world)]
-        self.dist.all_gather(out, t, group=self.group)
-        return [[int(o.item()) for o in out]]
-
-    def ranks(self, n_local):
-        return [self.dist.get_rank(self.group)]
+        assert len(ties) == 1
+        world, rank = self.dist.get_world_size(self.group), self.dist.get_rank(self.group)
+        out = [torch.zeros_like(ties[0]) for _ in range(world)]
+        self.dist.all_gather(out, ties[0], group=self.group)
+        return [torch.cat(out)[:rank].sum().reshape(1)]
 
 
 def schedule_sharded(shards, exchange, epoch_seconds: float, total_cores: int):
     """One epoch of one cluster whose jobs are split over ``shards`` (list of ``Scheduler``; one entry
-    per process with ``ProcessGroupExchange``).  Returns the list of per-shard allocations."""
+    per process with ``ProcessGroupExchange``).  Returns the list of per-shard allocations.
+
+    Every shard works on torch's current stream, on which torch orders its collectives as well: the
+    exchanges between the steps are stream-ordered, and the host waits for the device only twice, for
+    the cluster's job count before anything is queued and for the allocation at the end."""
     import torch
+    on_gpu = str(exchange.device).startswith("cuda")
+    if on_gpu:
+        stream = torch.cuda.current_stream()
+        for s in shards:
+            if getattr(s, "_sharded_stream", None) != stream.cuda_stream:
+                s.set_stream(stream)
+                s._sharded_stream = stream.cuda_stream
     cap = shards[0].max_cores_per_job
     assert all(s.max_cores_per_job == cap for s in shards)
     n_jobs = exchange.sum_ints([s.get_active_count() for s in shards])[0]
@@ -83,22 +93,19 @@ def schedule_sharded(shards, exchange, epoch_seconds: float, total_cores: int):
     want = min(total_cores, n_jobs * cap) - (n_jobs if with_floor else 0)
     for s in shards:
         s.shard_predict(epoch_seconds, with_floor)
-    buffers = [torch.zeros(N_BINS, dtype=torch.int64, device="cuda") for _ in shards]
+    buffers = [torch.zeros(N_BINS, dtype=torch.int64, device=exchange.device) for _ in shards]
     for p in range(N_PASSES):
         if p > 0:
             for s in shards:
                 s.shard_pass(p)
         for s, b in zip(shards, buffers):
             s.shard_histogram(p, b, import_it=False)
-        torch.cuda.synchronize()          # the library's stream and the collective's stream meet here
         exchange.sum_histograms(buffers)
-        torch.cuda.synchronize()
         for s, b in zip(shards, buffers):
             s.shard_histogram(p, b, import_it=True)
             s.shard_pick(p, want)
-    ties = [s.shard_count() for s in shards]
-    gathered = exchange.gather_ints(ties)
-    out = []
-    for s, all_ties, rank in zip(shards, gathered, exchange.ranks(len(shards))):
-        out.append(s.shard_finalise(sum(all_ties[:rank])))
-    return out
+    ties = [torch.zeros(1, dtype=torch.int64, device=exchange.device) for _ in shards]
+    for s, t in zip(shards, ties):
+        s.shard_count_device(t)
+    before = exchange.ties_before(ties)
+    return [s.shard_finalise_device(b) for s, b in zip(shards, before)]
