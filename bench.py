@@ -201,6 +201,8 @@ def run_gpu(args):
     sched = slaq.Scheduler(J, wl.max_hist, cap, stream=stream)
     sched.load_histories(ids, wl.offsets, wl.losses, wl.k_last, wl.m_seen, packed=args.cfg == CFG)   # config 4: rings
     sched.set_time_model(ids, wl.s, wl.w)
+    if args.selection is not None:
+        sched.set_param(slaq.binding.P_SELECTION, args.selection)
     d_alloc = torch.zeros(J, dtype=torch.int32, device="cuda")
 
     def barrier():
@@ -422,6 +424,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--cfg", type=int, default=CFG, choices=[2, 3, 4],
                     help="profiling aid: another workload generator (the reported line is then not the benchmark)")
+    ap.add_argument("--selection", type=int, default=None, choices=[0, 1],
+                    help="profiling aid: threshold selection over the gain table (0) or without a table (1)")
     ap.add_argument("--jobs", type=int, default=None,
                     help="profiling aid: a smaller cut of the same generator (the reported line is then not the benchmark)")
     args = ap.parse_args()

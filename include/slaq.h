@@ -86,7 +86,7 @@ enum {
                                      launches); 0: always plain launches; -1 (default): graph for handles
                                      created for at most 20,000 jobs.  Results are the same either way.  Not
                                      used while the handle's stream is itself being captured. */
-    SLAQ_P_GAIN_ENVELOPE = 9      /* 0 (default) or 1.  The greedy loop is exact when every job's predicted reduction
+    SLAQ_P_GAIN_ENVELOPE = 9,     /* 0 (default) or 1.  The greedy loop is exact when every job's predicted reduction
                                      R(n) is concave in its cores n, which a convex fitted curve gives.  Where a fit is
                                      not convex ahead of the newest point (the paper assumes convex losses: footnotes of
                                      "Predicting Quality Improvement"), the marginal gains may rise with n.  0: they
@@ -94,6 +94,15 @@ enum {
                                      1: they are replaced by the slopes of the upper concave envelope of the points
                                      (n, R(n)), the smallest concave function nowhere below R, which keeps the curve's
                                      whole drop at max_cores_per_job.  Rows of convex fits are the same either way. */
+    SLAQ_P_SELECTION = 10         /* How the greedy loop's threshold is found.  0: every job's gains for n = 1..max
+                                     are written to a table first and the selection reads the table.  1: no table -
+                                     a job's gains fall with n, so the selection finds what it needs of a row by
+                                     binary search over n with the gain in closed form, and evaluates only the gains
+                                     that share the threshold's leading digits (the effective gain of the n-th core is
+                                     then min(g(1), g(n)), which differs from the table's running minimum by rounding
+                                     at most).  Used for the plain prediction only: with SLAQ_P_GAIN_ENVELOPE, with
+                                     target-loss hints, and in the sharded steps the table is written.  The gain
+                                     rows that slaq_get_predictions returns are then written on request. */
 };
 
 /* per-job status written by slaq_schedule (slaq_get_predictions, out_status) */

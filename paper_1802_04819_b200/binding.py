@@ -14,6 +14,7 @@ P_GAMMA, P_LM_TRIALS, P_MAX_CORES_PER_JOB, P_MIN_FIT_POINTS, P_FIT_SLICE_BYTES, 
 P_FIT_CLUSTER_JOBS = 7
 P_EPOCH_GRAPH = 8
 P_GAIN_ENVELOPE = 9
+P_SELECTION = 10
 W_OVERSUBSCRIBED, W_UNDERFILLED = 1, 2
 
 EXPORTED_SYMBOLS = [

@@ -9,7 +9,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libslaq.so"
-SOURCES = ["slaq_api.cu", "slaq_fit.cu", "slaq_gain.cu", "slaq_alloc.cu"]
+SOURCES = ["slaq_api.cu", "slaq_fit.cu", "slaq_gain.cu", "slaq_alloc.cu", "slaq_select_free.cu"]
 
 
 # Instrumented builds of the same sources, each a library of its own beside libslaq.so.

@@ -408,6 +408,16 @@ int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_r
     return launches;
 }
 
+// The two small steps the table-free selection (slaq_select_free.cu) shares with this file.
+int launch_pick_first(slaq_handle* h) {
+    pick_first_kernel<<<1, kSelectThreads, 0, h->stream>>>(h->scratch.hist, h->scratch.sel);
+    return 1;
+}
+int launch_scan_blocks(slaq_handle* h, int blocks) {
+    scan_blocks_kernel<<<1, 1024, 0, h->stream>>>(h->scratch.block_eq, blocks);
+    return 1;
+}
+
 // ---- one cluster sharded over several GPUs: the same kernels, driven step by step so that the
 // histograms can be summed over the shards between the steps ----
 

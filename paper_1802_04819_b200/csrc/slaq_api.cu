@@ -390,6 +390,7 @@ int create_common(slaq_handle* h, int32_t max_jobs, int32_t max_hist, int32_t ca
     h->active.assign((size_t)max_jobs, 0);
     h->stamp.assign((size_t)max_jobs, 0u);
     h->in_packed.assign((size_t)max_jobs, 0);
+    h->hinted.assign((size_t)max_jobs, 0);
     for (auto& ev : h->ev) CK(cudaEventCreate(&ev), "cudaEventCreate");
     CK(cudaMemsetAsync(h->scratch.hist, 0, h->scratch.zero_bytes, h->stream), "clear scratch");
     CK(cudaMemsetAsync(h->err_word, 0, 16, h->stream), "clear error word");
@@ -502,6 +503,10 @@ int do_load(slaq_handle* h, int32_t n, const int32_t* ids, const int64_t* offset
                 }
                 for (int32_t j : gone) {
                     h->in_packed[j] = 0;
+                    if (h->hinted[j]) {
+                        h->hinted[j] = 0;
+                        h->n_hinted -= 1;
+                    }
                     if (h->active[j]) {
                         h->active[j] = 0;
                         h->n_active -= 1;
@@ -569,13 +574,20 @@ int enqueue_epoch(slaq_handle* h, double T, int64_t want, int floor_units, int32
         launches += k;
     }
     if (with_events && cudaEventRecord(h->ev[1], st) != cudaSuccess) return -1;
-    if (!only_allocate) {
+    // Without a table: only the plain prediction (no envelope, no target-loss hints) has gains in closed form.
+    const bool table_free = !only_allocate && h->selection == 1 && !h->gain_envelope && h->n_hinted == 0;
+    if (!only_allocate && !table_free) {
         if ((k = launch_gain(h, T, floor_units + 1)) < 0) return -1;
         launches += k;
     }
     if (with_events && cudaEventRecord(h->ev[2], st) != cudaSuccess) return -1;
-    if ((k = launch_allocate(h, want, floor_units + 1, !only_allocate, d_out)) < 0) return -1;
+    if (table_free) k = launch_allocate_free(h, T, want, floor_units + 1, d_out);
+    else k = launch_allocate(h, want, floor_units + 1, !only_allocate, d_out);
+    if (k < 0) return -1;
     launches += k;
+    h->gain_table_current = !table_free;
+    h->last_T = T;
+    h->last_first_unit = floor_units + 1;
     if (with_events && cudaEventRecord(h->ev[3], st) != cudaSuccess) return -1;
     return launches;
 }
@@ -589,7 +601,7 @@ std::vector<long long> epoch_key(const slaq_handle* h, double T, int64_t want, i
     std::memcpy(&g_bits, &h->gamma, sizeof g_bits);
     return {t_bits, (long long)want, floor_units, (long long)(uintptr_t)d_out, only_allocate ? 1 : 0, h->n_active,
             h->max_cores, h->lm_trials, h->min_fit_points, h->warm_start ? 1 : 0, (long long)h->fit_slice_bytes,
-            (long long)h->fit_cluster_jobs, g_bits, h->gain_envelope ? 1 : 0};
+            (long long)h->fit_cluster_jobs, g_bits, h->gain_envelope ? 1 : 0, h->selection, h->n_hinted};
 }
 
 int run_epoch(slaq_handle* h, double T, int64_t C, int32_t* d_out, bool only_allocate) {
@@ -771,6 +783,10 @@ int slaq_set_param(slaq_t* h, int key, double value) {
             if (!(value == 0.0 || value == 1.0)) return fail(h, SLAQ_E_ARG, "gain envelope must be 0 or 1");
             h->gain_envelope = value != 0.0;
             return SLAQ_OK;
+        case SLAQ_P_SELECTION:
+            if (!(value == 0.0 || value == 1.0)) return fail(h, SLAQ_E_ARG, "selection must be 0 or 1");
+            h->selection = (int)value;
+            return SLAQ_OK;
         default:
             return fail(h, SLAQ_E_ARG, "unknown parameter key");
     }
@@ -788,6 +804,7 @@ int slaq_get_param(const slaq_t* h, int key, double* out_value) {
         case SLAQ_P_FIT_CLUSTER_JOBS: *out_value = (double)h->fit_cluster_jobs; return SLAQ_OK;
         case SLAQ_P_EPOCH_GRAPH: *out_value = (double)h->epoch_graph; return SLAQ_OK;
         case SLAQ_P_GAIN_ENVELOPE: *out_value = h->gain_envelope ? 1.0 : 0.0; return SLAQ_OK;
+        case SLAQ_P_SELECTION: *out_value = (double)h->selection; return SLAQ_OK;
         default: return SLAQ_E_ARG;
     }
 }
@@ -847,6 +864,11 @@ int slaq_set_target_loss(slaq_t* h, int32_t n, const int32_t* job_ids, const dou
     set_target_kernel<<<(n + threads - 1) / threads, threads, 0, st>>>(h->job, h->max_jobs, n, h->stage.ids, h->stage.losses);
     CK(cudaGetLastError(), "target kernel");
     CK(cudaStreamSynchronize(st), "targets");
+    for (int32_t i = 0; i < n; ++i) {
+        const uint8_t now = std::isnan(targets[i]) ? 0 : 1;
+        h->n_hinted += (int32_t)now - (int32_t)h->hinted[job_ids[i]];
+        h->hinted[job_ids[i]] = now;
+    }
     return SLAQ_OK;
 }
 
@@ -864,6 +886,10 @@ int slaq_remove_jobs(slaq_t* h, int32_t n, const int32_t* job_ids) {
     CK(cudaStreamSynchronize(st), "remove");
     for (int32_t i = 0; i < n; ++i) {
         h->in_packed[job_ids[i]] = 0;
+        if (h->hinted[job_ids[i]]) {
+            h->hinted[job_ids[i]] = 0;
+            h->n_hinted -= 1;
+        }
         if (h->active[job_ids[i]]) {
             h->active[job_ids[i]] = 0;
             h->n_active -= 1;
@@ -1024,6 +1050,10 @@ int slaq_get_predictions(slaq_t* h, double* out_reduction, double* out_gain, int
     if (!h->have_epoch) return fail(h, SLAQ_E_ARG, "no epoch has been scheduled yet");
     const size_t J = (size_t)h->max_jobs;
     int rc = 0;
+    if (out_gain && !h->gain_table_current) {   // the last epoch ran without a table: write the rows now
+        if (launch_gain(h, h->last_T, h->last_first_unit) < 0) return SLAQ_E_CUDA;
+        h->gain_table_current = true;
+    }
     if ((rc = fetch(h, out_reduction, h->reduction, J, "copy reductions"))) return rc;
     if ((rc = fetch(h, out_gain, h->gain, J * h->max_cores, "copy gains"))) return rc;
     if ((rc = fetch(h, out_family, h->fit.family, J, "copy families"))) return rc;
@@ -1309,6 +1339,8 @@ int slaq_import_state(slaq_t* h, const void* blob_in, size_t bytes) {
         CK(cudaStreamSynchronize(st), "import: reset");
         std::fill(h->active.begin(), h->active.end(), 0);
         std::fill(h->in_packed.begin(), h->in_packed.end(), 0);
+        std::fill(h->hinted.begin(), h->hinted.end(), 0);
+        h->n_hinted = 0;
         h->n_active = 0;
         if (h->packed_pool) {
             cudaFree(h->packed_pool);
@@ -1329,6 +1361,14 @@ int slaq_import_state(slaq_t* h, const void* blob_in, size_t bytes) {
     CK(cudaMemcpyAsync(h->job.w_set, blob + L.off_w_set, 8 * J, up, st), "import state");
     CK(cudaMemcpyAsync(h->job.last_alloc, blob + L.off_last_alloc, 4 * J, up, st), "import state");
     CK(cudaMemcpyAsync(h->job.target, blob + L.off_target, 8 * J, up, st), "import state");
+    {
+        const double* target = reinterpret_cast<const double*>(blob + L.off_target);
+        for (size_t j = 0; j < J; ++j)
+            if (!std::isnan(target[j])) {
+                h->hinted[j] = 1;
+                h->n_hinted += 1;
+            }
+    }
     CK(cudaMemcpyAsync(h->fit.both, blob + L.off_both, 8 * 8 * J, up, st), "import state");
     CK(cudaMemcpyAsync(h->fit.mask, blob + L.off_mask, J, up, st), "import state");
     CK(cudaMemcpyAsync(h->fit.k_fit, blob + L.off_k_fit, 8 * J, up, st), "import state");

@@ -110,6 +110,12 @@ struct slaq_handle {
     int32_t lm_trials = 20, min_fit_points = 4;
     size_t fit_slice_bytes = 13824;       // shared memory one warp of the fit kernel may use (parked sums, up to 52 rows of 32 points, a spare row)
     bool warm_start = false;              // fits start from the last epoch's parameters where there are some
+    int selection = 0;                    // 0: selection over the written gain table, 1: gains evaluated on demand, no table
+    bool gain_table_current = false;      // h->gain holds the rows of the last epoch
+    double last_T = 0.0;                  // what the last epoch's gains were predicted for
+    int last_first_unit = 2;
+    std::vector<uint8_t> hinted;          // host mirror: job has a target-loss hint
+    int32_t n_hinted = 0;
     bool gain_envelope = false;           // gain rows are slopes of the concave envelope of R(n), not a running minimum
     int64_t fit_cluster_jobs = 0;         // active jobs the lanes per job are chosen for (0: this handle's own)
     cudaStream_t stream = nullptr;
@@ -160,6 +166,7 @@ namespace slaq {
 int launch_fit(slaq_handle* h);
 int launch_gain(slaq_handle* h, double epoch_seconds, int first_unit);
 int launch_allocate(slaq_handle* h, long long want, int first_unit, bool hist0_ready, int32_t* d_out_alloc);
+int launch_allocate_free(slaq_handle* h, double epoch_seconds, long long want, int first_unit, int32_t* d_out_alloc);
 int launch_normalise_export(slaq_handle* h, int32_t n, const int64_t* d_offsets, double* d_changes,
                             double* d_levels, double* d_largest);
 int launch_time_model(slaq_handle* h, double* d_s, double* d_w);
