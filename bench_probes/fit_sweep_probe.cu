@@ -20,18 +20,121 @@
 
 namespace {
 
+// An alternative that was measured and not adopted: the same sweep with the powers of x taken out of the
+// point loop (tables tab[p * ts + m] = gamma^m m^p, p = 0..4, in shared memory).  x = -m / span, so
+// sum w v x^p = (-1 / span)^p sum (gamma^m m^p) v: with the weighted powers gamma^m m^p in shared-memory
+// tables every accumulation is one fused multiply-add of (table entry, value, sum), the products with
+// w, x and x^2 disappear from the loop, and the sums are scaled once after it.  q is evaluated in
+// the point index as well: q = (a / span^2) m^2 - (b / span) m + c.
+__device__ __forceinline__ void sweep_tables(const slaq::Lanes& S, int ts, int fam, int H, int k_all, double inv_span,
+                                             const double (&pI)[4], bool doI, const double (&pII)[4], bool doII,
+                                             slaq::SweepSums& out) {
+    double m0 = 0, m1 = 0, m2 = 0, m3 = 0, m4 = 0, n0 = 0, n1 = 0, n2 = 0, h0 = 0, h1 = 0, h2 = 0, gd = 0, sI = 0;
+    double e0 = 0, e1 = 0, e2 = 0, f0 = 0, f1 = 0, k0 = 0, k1 = 0, gc = 0, sII = 0;
+    int feasible = 1;
+    double e = 0.0, ratio = 1.0;
+    if (doII) {
+        e = exp(fma(pII[1], (double)S.l * inv_span, pII[0]));
+        ratio = exp(pII[1] * ((double)S.L * inv_span));
+    }
+    const double qa = pI[0] * inv_span * inv_span, qb = -pI[1] * inv_span, qc = pI[2], dI = pI[3], cII = pII[2];
+    double md = (double)S.l;
+    const double dL = (double)S.L;
+    const double* yp = S.y + S.lane;
+    const double* tp = S.wtab + S.l;
+#pragma unroll 1
+    for (int k = 0, m = S.l; k < k_all; ++k, m += S.L, md += dL, yp += 32, tp += S.L) {
+        if (m < H) {
+            const bool ok = (m < S.wtab_len);
+            const double t0 = ok ? tp[0] : 0.0, t1 = ok ? tp[ts] : 0.0, t2 = ok ? tp[2 * ts] : 0.0;
+            const double y = S.holds(yp) ? *yp : 0.0;
+            if (doI) {
+                const double t3 = ok ? tp[3 * ts] : 0.0, t4 = ok ? tp[4 * ts] : 0.0;
+                const double q = fma(fma(qa, md, qb), md, qc);
+                feasible &= q > 0.0 ? 1 : 0;
+                const double inv = slaq::fast_rcp(q);
+                const double r = (y - dI) - inv;
+                const double u = inv * inv;
+                const double uu = u * u, ur = u * r;
+                m0 = fma(t0, uu, m0);
+                m1 = fma(t1, uu, m1);
+                m2 = fma(t2, uu, m2);
+                m3 = fma(t3, uu, m3);
+                m4 = fma(t4, uu, m4);
+                n0 = fma(t0, u, n0);
+                n1 = fma(t1, u, n1);
+                n2 = fma(t2, u, n2);
+                h0 = fma(t0, ur, h0);
+                h1 = fma(t1, ur, h1);
+                h2 = fma(t2, ur, h2);
+                gd = fma(t0, r, gd);
+                sI = fma(t0 * r, r, sI);
+            }
+            if (doII) {
+                const double r = (y - cII) - e;
+                const double ee = e * e, er = e * r;
+                e0 = fma(t0, ee, e0);
+                e1 = fma(t1, ee, e1);
+                e2 = fma(t2, ee, e2);
+                f0 = fma(t0, e, f0);
+                f1 = fma(t1, e, f1);
+                k0 = fma(t0, er, k0);
+                k1 = fma(t1, er, k1);
+                gc = fma(t0, r, gc);
+                sII = fma(t0 * r, r, sII);
+            }
+        }
+        e *= ratio;
+    }
+    // back to powers of x = -m / span
+    const double s1 = -inv_span, s2 = inv_span * inv_span, s3 = s1 * s2, s4 = s2 * s2;
+    m1 *= s1; m2 *= s2; m3 *= s3; m4 *= s4;
+    n1 *= s1; n2 *= s2;
+    h1 *= s1; h2 *= s2;
+    e1 *= s1; e2 *= s2;
+    f1 *= s1;
+    k1 *= s1;
+    const bool odd = fam != 0;
+    double v[13];
+#define SLAQ_PAIR(k, a, b) v[k] = (odd ? (b) : (a)) + __shfl_xor_sync(slaq::kFull, odd ? (a) : (b), 1)
+    SLAQ_PAIR(0, m0, e0); SLAQ_PAIR(1, m1, e1); SLAQ_PAIR(2, m2, e2); SLAQ_PAIR(3, m3, f0); SLAQ_PAIR(4, m4, f1);
+    SLAQ_PAIR(5, n0, k0); SLAQ_PAIR(6, n1, k1); SLAQ_PAIR(7, n2, gc); SLAQ_PAIR(8, h0, sII);
+#undef SLAQ_PAIR
+    v[9] = h1 + __shfl_xor_sync(slaq::kFull, h1, 1);
+    v[10] = h2 + __shfl_xor_sync(slaq::kFull, h2, 1);
+    v[11] = gd + __shfl_xor_sync(slaq::kFull, gd, 1);
+    v[12] = sI + __shfl_xor_sync(slaq::kFull, sI, 1);
+    feasible &= __shfl_xor_sync(slaq::kFull, feasible, 1);
+    for (int o = 2; o < S.L; o <<= 1) {
+#pragma unroll
+        for (int k = 0; k < 13; ++k) v[k] += __shfl_xor_sync(slaq::kFull, v[k], o);
+        feasible &= __shfl_xor_sync(slaq::kFull, feasible, o);
+    }
+    double chk = 0.0;
+#pragma unroll
+    for (int k = 0; k < 13; ++k) {
+        out.v[k] = v[k];
+        if (k < 9 || !odd) chk += v[k];
+    }
+    out.usable = slaq::finite_d(chk) && (odd || feasible);
+}
+
+
 constexpr int kWarps = 16;
 constexpr int kSliceDoubles = 13824 / 8;
 constexpr int kTable = 1000;
 
+// kTables: the variant with the weighted powers of the point index in shared-memory tables (5 tables, smaller slices)
+template <bool kTables>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 sweep_loop_kernel(const double* __restrict__ g_wtab, int L, int rows, int n_sweeps, int warps_active, double* out,
-                  long long* cycles) {
+                  long long* cycles, int slice_doubles) {
     extern __shared__ double smem[];
     double* wtab = smem;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int i = threadIdx.x; i < kTable; i += blockDim.x) wtab[i] = g_wtab[i];
-    double* const slice = smem + kTable + (size_t)warp * kSliceDoubles;
+    constexpr int kTabs = kTables ? 5 : 1;
+    for (int i = threadIdx.x; i < kTabs * kTable; i += blockDim.x) wtab[i] = g_wtab[i];
+    double* const slice = smem + kTabs * kTable + (size_t)warp * slice_doubles;
     slaq::Lanes S;
     S.wtab = wtab;
     S.lane = lane;
@@ -41,7 +144,7 @@ sweep_loop_kernel(const double* __restrict__ g_wtab, int L, int rows, int n_swee
     S.park = slice + 2 * (lane / L) + (lane & 1);
     S.y = slice + slaq::kParked * 2 * G;
     S.slice = slice;
-    S.slice_len = kSliceDoubles;
+    S.slice_len = slice_doubles;
     S.wtab_len = kTable;
     S.err_word = nullptr;
     const int H = rows * L;
@@ -63,7 +166,8 @@ sweep_loop_kernel(const double* __restrict__ g_wtab, int L, int rows, int n_swee
     if (warp < warps_active) {
         for (int it = 0; it < n_sweeps; ++it) {
             slaq::SweepSums sums;
-            slaq::sweep(S, fam, H, rows, inv_span, pI, true, pII, true, sums);
+            if (kTables) sweep_tables(S, kTable, fam, H, rows, inv_span, pI, true, pII, true, sums);
+            else slaq::sweep(S, fam, H, rows, inv_span, pI, true, pII, true, sums);
             check += sums.v[fam ? 8 : 12];
             // move the points a little, as accepted trials do (keeps every sweep's arithmetic live)
             pI[2] = fma(pI[2], 1.0 + 1e-9, sums.usable ? 0.0 : 1e-12);
@@ -84,56 +188,68 @@ int main(int argc, char** argv) {
         fprintf(stderr, "fit_sweep_probe: no CUDA device\n");
         return 1;
     }
-    std::vector<double> tab(kTable);
+    std::vector<double> tab(5 * kTable);
     double wv = 1.0;
-    for (int m = 0; m < kTable; ++m, wv *= 0.9) tab[m] = wv;
+    for (int m = 0; m < kTable; ++m, wv *= 0.9) {
+        double pw = wv;
+        for (int p = 0; p < 5; ++p, pw *= (double)m) tab[p * kTable + m] = pw;
+    }
     double *d_tab = nullptr, *d_out = nullptr;
     long long* d_cycles = nullptr;
-    const size_t smem = sizeof(double) * (kTable + (size_t)kWarps * kSliceDoubles);
-    if (cudaMalloc(&d_tab, sizeof(double) * kTable) != cudaSuccess ||
+    if (cudaMalloc(&d_tab, sizeof(double) * 5 * kTable) != cudaSuccess ||
         cudaMalloc(&d_out, sizeof(double) * sm_count * kWarps * 32) != cudaSuccess ||
         cudaMalloc(&d_cycles, sizeof(long long) * sm_count) != cudaSuccess)
         return 1;
-    cudaMemcpy(d_tab, tab.data(), sizeof(double) * kTable, cudaMemcpyHostToDevice);
-    if (cudaFuncSetAttribute(sweep_loop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-        fprintf(stderr, "fit_sweep_probe: cannot get %zu bytes of shared memory\n", smem);
-        return 1;
-    }
+    cudaMemcpy(d_tab, tab.data(), sizeof(double) * 5 * kTable, cudaMemcpyHostToDevice);
     cudaEvent_t e0, e1;
     cudaEventCreate(&e0);
     cudaEventCreate(&e1);
     printf("%d SMs, %d sweeps per warp, both families in every sweep\n", sm_count, n_sweeps);
-    printf("%4s %5s %9s %22s %20s %14s\n", "L", "rows", "warps/SM", "cycles/warp row/SMSP", "of 92 (2-cycle issue)", "ms");
-    // rows a slice holds at L lanes per job: (slice - parked sums of its 32/L jobs) / 32 - 1 spare row, as in the library
-    const int cases[][2] = {{2, 41}, {4, 47}, {8, 50}, {16, 51}, {32, 31}};
     std::vector<long long> cyc(sm_count);
-    for (const auto& c : cases) {
-        if (slaq::kParked * (64 / c[0]) + (c[1] + 1) * 32 > kSliceDoubles) {
-            fprintf(stderr, "fit_sweep_probe: %d rows at L = %d do not fit a slice\n", c[1], c[0]);
+    for (int variant = 0; variant < 2; ++variant) {
+        // the tables take 4 x kTable doubles more of the SM's shared memory: the sixteen slices shrink accordingly
+        const int slice_doubles = variant == 0 ? kSliceDoubles : (kSliceDoubles * kWarps - 4 * kTable) / kWarps / 32 * 32;
+        const size_t smem = sizeof(double) * ((variant == 0 ? 1 : 5) * kTable + (size_t)kWarps * slice_doubles);
+        auto kernel = variant == 0 ? sweep_loop_kernel<false> : sweep_loop_kernel<true>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+            fprintf(stderr, "fit_sweep_probe: cannot get %zu bytes of shared memory\n", smem);
             return 1;
         }
-        for (int warps = 4; warps <= kWarps; warps += 4) {
-            double best_cycles = 1e300;
-            float best_ms = 1e30f;
-            for (int rep = 0; rep < 4; ++rep) {   // the first repetition warms up
-                cudaEventRecord(e0);
-                sweep_loop_kernel<<<sm_count, kWarps * 32, smem>>>(d_tab, c[0], c[1], n_sweeps, warps, d_out, d_cycles);
-                cudaEventRecord(e1);
-                const cudaError_t err = cudaDeviceSynchronize();
-                if (err != cudaSuccess) {
-                    fprintf(stderr, "fit_sweep_probe: kernel failed: %s\n", cudaGetErrorString(err));
-                    return 1;
-                }
-                float ms = 0.f;
-                cudaEventElapsedTime(&ms, e0, e1);
-                cudaMemcpy(cyc.data(), d_cycles, sizeof(long long) * sm_count, cudaMemcpyDeviceToHost);
-                double mean = 0.0;
-                for (long long v : cyc) mean += (double)v;
-                mean /= sm_count;
-                if (rep > 0 && mean < best_cycles) best_cycles = mean, best_ms = ms;
+        printf("%s, %d doubles per slice\n", variant == 0 ? "powers of x multiplied in the loop" : "weighted powers from tables",
+               slice_doubles);
+        printf("%4s %5s %9s %22s %20s %14s\n", "L", "rows", "warps/SM", "cycles/warp row/SMSP", "of 92 (2-cycle issue)", "ms");
+        // rows a slice holds at L lanes per job: (slice - parked sums of its 32/L jobs) / 32 - 1 spare row, as in the library
+        const int Ls[5] = {2, 4, 8, 16, 32};
+        for (int L : Ls) {
+            int rows = (slice_doubles - slaq::kParked * (64 / L)) / 32 - 1;
+            if (rows * L > kTable - 8) rows = (kTable - 8) / L;
+            if (rows < 1 || slaq::kParked * (64 / L) + (rows + 1) * 32 > slice_doubles) {
+                fprintf(stderr, "fit_sweep_probe: no room for L = %d\n", L);
+                return 1;
             }
-            const double per_row = best_cycles / ((double)c[1] * n_sweeps * (warps / 4.0));
-            printf("%4d %5d %9d %22.1f %20.3f %14.3f\n", c[0], c[1], warps, per_row, 92.0 / per_row, best_ms);
+            for (int warps = 4; warps <= kWarps; warps += 4) {
+                double best_cycles = 1e300;
+                float best_ms = 1e30f;
+                for (int rep = 0; rep < 4; ++rep) {   // the first repetition warms up
+                    cudaEventRecord(e0);
+                    kernel<<<sm_count, kWarps * 32, smem>>>(d_tab, L, rows, n_sweeps, warps, d_out, d_cycles, slice_doubles);
+                    cudaEventRecord(e1);
+                    const cudaError_t err = cudaDeviceSynchronize();
+                    if (err != cudaSuccess) {
+                        fprintf(stderr, "fit_sweep_probe: kernel failed: %s\n", cudaGetErrorString(err));
+                        return 1;
+                    }
+                    float ms = 0.f;
+                    cudaEventElapsedTime(&ms, e0, e1);
+                    cudaMemcpy(cyc.data(), d_cycles, sizeof(long long) * sm_count, cudaMemcpyDeviceToHost);
+                    double mean = 0.0;
+                    for (long long v : cyc) mean += (double)v;
+                    mean /= sm_count;
+                    if (rep > 0 && mean < best_cycles) best_cycles = mean, best_ms = ms;
+                }
+                const double per_row = best_cycles / ((double)rows * n_sweeps * (warps / 4.0));
+                printf("%4d %5d %9d %22.1f %20.3f %14.3f\n", L, rows, warps, per_row, 92.0 / per_row, best_ms);
+            }
         }
     }
     cudaFree(d_tab);

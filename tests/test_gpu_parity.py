@@ -488,6 +488,63 @@ def test_windows_without_a_usable_start_take_the_fallback(slaq, oracle_mod, pack
     assert sched.get_stats().fallback_jobs == 2 * n_bad
 
 
+def _oracle_spread(oracle_mod, wl, j, cap, n_trials=24):
+    """How far the oracle's own R(n) of job j moves when its losses are perturbed by 1e-13 relative: per n the
+    largest distance from the unperturbed result.  Zero to rounding for a fit that has finished; large where the
+    twenty trials end on a path-dependent point."""
+    h = wl.history(j)
+    off = np.array([0, h.size])
+    one = lambda a: np.array([a[j]])     # noqa: E731
+    base = np.cumsum(oracle_mod.predict(off, h, one(wl.m_seen), one(wl.s), one(wl.w), wl.epoch_seconds, cap)["gain"][0])
+    rng = np.random.default_rng(1000 + j)
+    spread = np.zeros_like(base)
+    for _ in range(n_trials):
+        hp = h * (1.0 + 1e-13 * rng.standard_normal(h.size))
+        R = np.cumsum(oracle_mod.predict(off, hp, one(wl.m_seen), one(wl.s), one(wl.w), wl.epoch_seconds, cap)["gain"][0])
+        spread = np.maximum(spread, np.abs(R - base))
+    return spread
+
+
+def test_unseen_cuts_survey(slaq, oracle_mod):
+    """Cuts and seeds no other test uses, 100,000 jobs in all: how often does a job miss the tolerance on R(n), and
+    why.  Twenty solver trials do not finish every fit.  Where the residual is nearly flat along a direction
+    (converged jobs of config 4: sixty-four points of noise around a level), the end point of the unfinished
+    iteration depends on rounding, for the oracle too: perturbing such a job's losses by 1e-13 moves the ORACLE'S
+    OWN prediction by more than the tolerance.  Measured over 333,000 jobs of 40 unseen cuts: 5 jobs outside the
+    tolerance (by factors 1.005 to 15.8), all in config 4, each within the oracle's own spread under that
+    perturbation.  Asserted: every miss is explained that way (within 4 spreads), and there is at most one per
+    25,000 jobs."""
+    total, misses = 0, []
+    for cfg, sizes in ((4, (9000, 23000, 31000)), (3, (2500, 6500)), (2, (2000, 3000)), (1, (160,))):
+        for n in sizes:
+            for seed in (5, 6) if n < 20000 else (5,):
+                wl = make_workload(cfg, n_jobs=n, seed_offset=seed)
+                cap = wl.max_cores_per_job
+                sched = make_scheduler(wl, packed=cfg == 3)
+                sched.schedule(wl.epoch_seconds, wl.total_cores)
+                pred = sched.get_predictions()
+                ref = oracle_mod.predict(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, cap)
+                np.testing.assert_array_equal(pred["status"], ref["status"])
+                Rg, Rc = np.cumsum(pred["gain"], axis=1), np.cumsum(ref["gain"], axis=1)
+                tol = 1e-6 * np.abs(Rc) + 1e-9
+                width = (np.abs(Rg - Rc) / tol).max(axis=1)
+                tied = pred["family"] != ref["family"]
+                for j in np.nonzero(tied)[0]:
+                    S = ref["S"][j]
+                    assert abs(S[0] - S[1]) <= 1e-9 * max(abs(S[0]), abs(S[1]))
+                for j in np.nonzero((width > 1.0) & ~tied)[0]:
+                    spread = _oracle_spread(oracle_mod, wl, j, cap)
+                    assert (np.abs(Rg[j] - Rc[j]) <= 4.0 * spread + tol[j]).all(), (
+                        f"config {cfg}, {n} jobs, seed {seed}, job {j}: {width[j]:.2f} tolerances off, and the oracle's "
+                        f"own result is stable ({(spread / tol[j]).max():.2f} tolerances under perturbation)")
+                    misses.append((cfg, n, seed, int(j), float(width[j]), float((spread / tol[j]).max())))
+                total += wl.n_jobs
+                sched.close()
+    print(f"survey: {total} jobs, misses (config, jobs, seed, job, tolerances off, oracle's own spread): {misses}")
+    assert total >= 100_000
+    assert len(misses) <= total // 25_000
+
+
 # ---------------------------------------------------------------- streaming: append -> schedule with the allocation fed back
 def test_streaming_epochs_with_allocation_feedback(slaq, oracle_mod):
     """Several epochs in a row: each job runs as many iterations as its allocation allows in the epoch, reports
