@@ -242,7 +242,7 @@ def run_gpu(args):
         ev1.record(stream)
         barrier()
         block_ms.append(ev0.elapsed_time(ev1))
-        enough = time.perf_counter() - t_from >= MIN_TIMED_SECONDS
+        enough = time.perf_counter() - t_from >= args.min_seconds
         if world > 1:                              # every rank runs the same number of blocks
             flag = torch.tensor([1.0 if enough else 0.0], device="cuda")
             dist.all_reduce(flag, op=dist.ReduceOp.MIN)
@@ -424,6 +424,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--cfg", type=int, default=CFG, choices=[2, 3, 4],
                     help="profiling aid: another workload generator (the reported line is then not the benchmark)")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="the block of --steps steps is repeated until the timed region lasts this long (0: one block; "
+                         "for runs under a profiler)")
     ap.add_argument("--selection", type=int, default=None, choices=[0, 1],
                     help="profiling aid: threshold selection over the gain table (0) or without a table (1)")
     ap.add_argument("--jobs", type=int, default=None,

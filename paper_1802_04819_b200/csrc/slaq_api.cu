@@ -963,6 +963,9 @@ int slaq_shard_predict(slaq_t* h, double epoch_seconds, int32_t with_floor) {
     CK(cudaEventRecord(h->ev[3], st), "event");
     h->have_epoch = true;
     h->last_launches = launches;
+    h->gain_table_current = true;
+    h->last_T = epoch_seconds;
+    h->last_first_unit = h->shard_first_unit;
     return SLAQ_OK;
 }
 

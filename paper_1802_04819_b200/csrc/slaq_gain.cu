@@ -49,13 +49,16 @@ __device__ void envelope_of_row(double* row, int cap, unsigned short* stack) {
     }
 }
 
-// options: bit 0 = rows become the slopes of the concave envelope of R(n) instead of a running minimum
+// kOptions: the instantiation that knows the two options of the prediction (the plain one carries none of
+// their code).  options: bit 0 = rows become the slopes of the concave envelope of R(n) instead of a
+// running minimum; target-loss hints are read per job.
+template <bool kOptions>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int first_unit, double* __restrict__ gain,
             unsigned long long* __restrict__ hist0, int options) {
     __shared__ unsigned int sh_hist[kRadixBins];
-    __shared__ unsigned short sh_stack[kWarpsPerBlock][kMaxCoresLimit + 1];
-    const bool envelope = (options & 1) != 0;
+    __shared__ unsigned short sh_stack[kOptions ? kWarpsPerBlock : 1][kOptions ? kMaxCoresLimit + 1 : 1];
+    const bool envelope = kOptions && (options & 1) != 0;
     for (int i = threadIdx.x; i < kRadixBins; i += blockDim.x) sh_hist[i] = 0;
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -67,7 +70,7 @@ gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int f
         if (no_time && lane == 0) fit.status[j] = SLAQ_JOB_NO_TIME;
         // A target-loss hint caps the predicted reduction at (newest loss - target) / M.
         double reduction_cap = CUDART_INF;
-        if (c.kind != 3) {
+        if (kOptions && c.kind != 3) {
             const double target = job.target[j];
             const double M = fit.largest[j];
             if (finite_d(target) && M > 0.0) {
@@ -78,7 +81,7 @@ gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int f
                 reduction_cap = __ddiv_rn(fmax(newest - target, 0.0), M);
             }
         }
-        if (envelope || reduction_cap < CUDART_INF) {
+        if (kOptions && (envelope || reduction_cap < CUDART_INF)) {
             // General path (options in use): the row is completed in memory first, then read back for the cap
             // and the histogram.
             double* row = gain + (size_t)j * cap;
@@ -142,24 +145,36 @@ gain_kernel(JobArrays job, FitArrays fit, int max_jobs, int cap, double T, int f
             const int n = base + lane + 1;
             double g = CUDART_INF;
             if (n <= cap) g = c.kind == 3 ? 0.0 : raw_gain(c, n);
-            // inclusive running minimum over n
+            // inclusive running minimum over n; most chunks fall already (convex fits), which one look at the
+            // left neighbour shows
+            double left = __shfl_up_sync(kFull, g, 1);
+            if (lane == 0) left = carry;
+            if (!__all_sync(kFull, n > cap || !(g > left))) {
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const double up = __shfl_up_sync(kFull, g, o);
-                if (lane >= o) g = fmin(g, up);
+                for (int o = 1; o < 32; o <<= 1) {
+                    const double up = __shfl_up_sync(kFull, g, o);
+                    if (lane >= o) g = fmin(g, up);
+                }
+                g = fmin(g, carry);
             }
-            g = fmin(g, carry);
             carry = __shfl_sync(kFull, g, 31);
             const bool counted = active && n <= cap && n >= first_unit;
             if (n <= cap && index_ok((long long)j * cap + (n - 1), (long long)max_jobs * cap, kErrGain, job.err_word))
                 gain[(size_t)j * cap + (n - 1)] = g;
             const unsigned digit = (unsigned)((unsigned long long)__double_as_longlong(g) >> (64 - kRadixBits));
-            // lanes with the same digit add once: a row is nearly constant in its top bits
+            // lanes with the same digit add once: a row is nearly constant in its top bits, and often the whole
+            // chunk shares one digit
             const unsigned live = __ballot_sync(kFull, counted);
-            if (counted) {
-                const unsigned peers = __match_any_sync(live, digit);
-                if ((int)(__ffs(peers) - 1) == lane && index_ok(digit, kRadixBins, kErrBin, job.err_word))
-                    atomicAdd(&sh_hist[digit], (unsigned)__popc(peers));
+            if (live) {
+                const unsigned first_digit = __shfl_sync(kFull, digit, __ffs(live) - 1);
+                if (__all_sync(kFull, !counted || digit == first_digit)) {
+                    if (lane == __ffs(live) - 1 && index_ok(digit, kRadixBins, kErrBin, job.err_word))
+                        atomicAdd(&sh_hist[digit], (unsigned)__popc(live));
+                } else if (counted) {
+                    const unsigned peers = __match_any_sync(live, digit);
+                    if ((int)(__ffs(peers) - 1) == lane && index_ok(digit, kRadixBins, kErrBin, job.err_word))
+                        atomicAdd(&sh_hist[digit], (unsigned)__popc(peers));
+                }
             }
         }
     }
@@ -185,9 +200,9 @@ int launch_gain(slaq_handle* h, double epoch_seconds, int first_unit) {
     int blocks = h->sm_count * 4;
     const int needed = (h->max_jobs + kWarpsPerBlock - 1) / kWarpsPerBlock;
     if (blocks > needed) blocks = needed;
-    gain_kernel<<<blocks, kWarpsPerBlock * 32, 0, h->stream>>>(h->job, h->fit, h->max_jobs, h->max_cores, epoch_seconds,
-                                                              first_unit, h->gain, h->scratch.hist,
-                                                              h->gain_envelope ? 1 : 0);
+    const auto kernel = (h->gain_envelope || h->n_hinted > 0) ? gain_kernel<true> : gain_kernel<false>;
+    kernel<<<blocks, kWarpsPerBlock * 32, 0, h->stream>>>(h->job, h->fit, h->max_jobs, h->max_cores, epoch_seconds,
+                                                         first_unit, h->gain, h->scratch.hist, h->gain_envelope ? 1 : 0);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         h->err = std::string("gain kernel launch: ") + cudaGetErrorString(e);
