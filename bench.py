@@ -117,7 +117,7 @@ def measured_fp64_peak():
     try:
         if not exe.exists():
             sys.path.insert(0, str(ROOT / "bench_probes"))
-            import build as probe_build   # bench_probes/build.py
+            import build_probes as probe_build   # bench_probes/build_probes.py
             probe_build.build_probes()
         out = subprocess.run([str(exe)], capture_output=True, text=True, timeout=120, check=True).stdout
     except (OSError, subprocess.SubprocessError, ImportError) as err:

@@ -1,6 +1,6 @@
 """Compile the stand-alone measurement programs that back the roofline figures (sm_100a, nvcc).
 
-    python bench_probes/build.py
+    python bench_probes/build_probes.py
 
 fp64_issue_probe   issue rate of the fp64 pipe by operand pattern (the roofline's denominator)
 fit_sweep_probe    the fit kernel's sweep function in a loop of its own (what the instruction mix allows)
