@@ -117,3 +117,30 @@ def test_options_that_need_the_table_still_get_it(slaq, oracle_mod):
     ref = oracle_mod.schedule(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, wl.total_cores,
                               wl.max_cores_per_job, target_loss=target)
     compare_epoch(alloc, sched.get_predictions(), ref, wl.total_cores, wl.max_cores_per_job, allow_unstable=1)
+
+
+@pytest.mark.parametrize("cap", [1, 2, 33, 1024])
+def test_extreme_caps_with_every_way_of_predicting(slaq, oracle_mod, cap):
+    """One core per job at most, two, a row that is one entry longer than a warp step, and the largest cap the
+    library takes: table and table-free selection, envelope rows and target hints against the oracle."""
+    wl = make_workload(4, n_jobs=600)
+    J = wl.n_jobs
+    newest = wl.losses[wl.offsets[1:] - 1]
+    target = np.full(J, np.nan)
+    target[::3] = newest[::3] * 0.9995
+    for C in (J // 2, J, 3 * J, J * cap):
+        for selection, envelope, hints in ((0, 0, False), (1, 0, False), (0, 1, False), (0, 0, True), (1, 1, True)):
+            sched = slaq.Scheduler(J, wl.max_hist, cap)
+            ids = np.arange(J, dtype=np.int32)
+            sched.load_histories(ids, wl.offsets, wl.losses, wl.k_last, wl.m_seen)
+            sched.set_time_model(ids, wl.s, wl.w)
+            sched.set_param(slaq.binding.P_SELECTION, selection)
+            sched.set_param(slaq.binding.P_GAIN_ENVELOPE, envelope)
+            if hints:
+                sched.set_target_loss(ids[::3], target[::3])
+            alloc, rc = sched.schedule(wl.epoch_seconds, C)
+            ref = oracle_mod.schedule(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, C, cap,
+                                      envelope=bool(envelope), target_loss=target if hints else None)
+            compare_epoch(alloc, sched.get_predictions(), ref, C, cap)
+            assert alloc.sum() == min(C, J * cap) and alloc.max() <= cap
+            sched.close()
