@@ -80,3 +80,20 @@ def compare_epoch(gpu_alloc, pred, ref, total_cores, cap, allow_unstable=0, loos
     assert abs(pred["R"].sum() - tot_c) <= total_rtol * abs(tot_c) + 1e-9 * max(1, diff.size) + slack
     return dict(jobs=int(status_c.size), fitted=int(fitted.sum()), family_ties=int(fam_diff.size),
                 unstable=int(bad_jobs.size), alloc_diff=int(diff.size))
+
+
+def oracle_spread(oracle_mod, wl, j, cap, n_trials=24):
+    """How far the oracle's own R(n) of job j moves when its losses are perturbed by 1e-13 relative: per n the
+    largest distance from the unperturbed result.  Zero to rounding for a fit that has finished; large where the
+    twenty trials end on a path-dependent point."""
+    h = wl.history(j)
+    off = np.array([0, h.size])
+    one = lambda a: np.array([a[j]])     # noqa: E731
+    base = np.cumsum(oracle_mod.predict(off, h, one(wl.m_seen), one(wl.s), one(wl.w), wl.epoch_seconds, cap)["gain"][0])
+    rng = np.random.default_rng(1000 + j)
+    spread = np.zeros_like(base)
+    for _ in range(n_trials):
+        hp = h * (1.0 + 1e-13 * rng.standard_normal(h.size))
+        R = np.cumsum(oracle_mod.predict(off, hp, one(wl.m_seen), one(wl.s), one(wl.w), wl.epoch_seconds, cap)["gain"][0])
+        spread = np.maximum(spread, np.abs(R - base))
+    return spread

@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 
 from workloads import make_workload
-from gpu_common import compare_epoch, make_scheduler, oracle_epoch
+from gpu_common import compare_epoch, make_scheduler, oracle_epoch, oracle_spread
 
 pytestmark = pytest.mark.gpu
 
@@ -23,10 +23,12 @@ def test_config3_full_size_all_jobs(oracle_mod):
     assert alloc.sum() == wl.total_cores
 
 
-def test_config4_full_size_sampled(oracle_mod):
-    """1,000,000 jobs, ring of 64, 128 cores per job: predictions of a sample against the oracle one by one;
-    the allocation through properties that hold at any size and, entry by entry, against the oracle's greedy loop
-    fed the same gain table."""
+def test_config4_full_size_every_job(oracle_mod):
+    """1,000,000 jobs, ring of 64, 128 cores per job: the predictions of every job against the oracle one by one,
+    and the allocation entry by entry - against the oracle's greedy loop fed the GPU's gain table (bit for bit), and
+    against the oracle's own whole epoch (equal except within rounding of the threshold).
+    A job may miss the tolerance on R(n) only where the oracle's own result moves as much when its losses are
+    perturbed by 1e-13 (unfinished fits of nearly flat windows; measured: 9 of the 1,000,000)."""
     import paper_1802_04819_b200 as slaq
     slaq.build()
     wl = make_workload(4)
@@ -35,23 +37,24 @@ def test_config4_full_size_sampled(oracle_mod):
     assert rc == 0
     pred = sched.get_predictions()
     cap = wl.max_cores_per_job
-    # sample: every 53rd job plus all clones and their sources
-    dst = np.nonzero(wl.clone_of >= 0)[0]
-    sample = np.unique(np.concatenate([np.arange(0, wl.n_jobs, 53), dst, wl.clone_of[dst]]))
-    H = wl.hist_len[sample]
-    off = np.zeros(sample.size + 1, np.int64)
-    np.cumsum(H, out=off[1:])
-    idx = np.concatenate([np.arange(wl.offsets[j], wl.offsets[j + 1]) for j in sample])
-    ref = oracle_mod.predict(off, wl.losses[idx], wl.m_seen[sample], wl.s[sample], wl.w[sample], wl.epoch_seconds, cap)
-    np.testing.assert_array_equal(pred["status"][sample], ref["status"])
-    np.testing.assert_array_equal(pred["M"][sample], ref["M"])
-    Rg, Rc = np.cumsum(pred["gain"][sample], axis=1), np.cumsum(ref["gain"], axis=1)
-    tied = pred["family"][sample] != ref["family"]
-    bad = (np.abs(Rg - Rc) > 1e-6 * np.abs(Rc) + 1e-9).any(axis=1) & ~tied
-    assert bad.sum() == 0, f"{bad.sum()} of {sample.size} sampled jobs exceed the tolerance"
-    for j in np.nonzero(tied)[0]:
-        S = ref["S"][j]
-        assert abs(S[0] - S[1]) <= 1e-9 * max(abs(S[0]), abs(S[1]))
+    ref = oracle_mod.predict(wl.offsets, wl.losses, wl.m_seen, wl.s, wl.w, wl.epoch_seconds, cap)
+    np.testing.assert_array_equal(pred["status"], ref["status"])
+    np.testing.assert_array_equal(pred["M"], ref["M"])
+    tied = pred["family"] != ref["family"]          # flat windows: both families end as the same constant
+    S = ref["S"][tied]
+    assert (np.abs(S[:, 0] - S[:, 1]) <= 1e-9 * np.abs(S).max(axis=1)).all()
+    misses = []
+    for lo in range(0, wl.n_jobs, 100_000):          # in blocks, to bound the memory of the cumulative sums
+        hi = lo + 100_000
+        Rg, Rc = np.cumsum(pred["gain"][lo:hi], axis=1), np.cumsum(ref["gain"][lo:hi], axis=1)
+        tol = 1e-6 * np.abs(Rc) + 1e-9
+        width = (np.abs(Rg - Rc) / tol).max(axis=1)
+        for j in np.nonzero((width > 1.0) & ~tied[lo:hi])[0]:
+            spread = oracle_spread(oracle_mod, wl, lo + j, cap)
+            assert (np.abs(Rg[j] - Rc[j]) <= 4.0 * spread + tol[j]).all(), f"job {lo + j}: {width[j]:.2f} tolerances off"
+            misses.append((int(lo + j), float(width[j])))
+    print("config 4 full size: misses", misses, "tied winners", int(tied.sum()))
+    assert len(misses) <= wl.n_jobs // 25_000
     # allocation: all cores handed out, floor and cap respected, and it is a top-C selection of the GPU's own gains:
     # every gain taken beyond the floor is at least as large as every gain left
     assert alloc.sum() == wl.total_cores and alloc.min() >= 1 and alloc.max() <= cap
@@ -66,10 +69,16 @@ def test_config4_full_size_sampled(oracle_mod):
     at_tau_left = np.nonzero(((g == tau) & left).any(axis=1))[0]
     if at_tau_taken.size and at_tau_left.size:
         assert at_tau_taken.max() <= at_tau_left.min()
+    dst = np.nonzero(wl.clone_of >= 0)[0]
     np.testing.assert_array_equal(g[dst], g[wl.clone_of[dst]])
-    # and bit for bit the allocation of the literal greedy loop (a heap of one offer per job, one core per pop) run
+    # bit for bit the allocation of the literal greedy loop (a heap of one offer per job, one core per pop) run
     # on the CPU over the same 1,000,000 x 128 gain table, exact ties of the clones included
-    want = oracle_mod.allocate(g, np.ones(wl.n_jobs, np.uint8), wl.total_cores)
-    np.testing.assert_array_equal(alloc, want)
+    active = np.ones(wl.n_jobs, np.uint8)
+    np.testing.assert_array_equal(alloc, oracle_mod.allocate(g, active, wl.total_cores))
+    # and the oracle's own epoch (its own gains): different only where a deciding gain is within rounding of the threshold
+    own = oracle_mod.allocate(ref["gain"], active, wl.total_cores)
+    for j in np.nonzero(own != alloc)[0]:
+        a, b = sorted((int(own[j]), int(alloc[j])))
+        assert np.all(np.abs(ref["gain"][j, a:b] - tau) <= 1e-9 + 1e-6 * tau)
     R_direct = np.where(cols < alloc[:, None], g, 0.0).sum(axis=1)
     np.testing.assert_allclose(pred["R"], R_direct, rtol=1e-12, atol=1e-15)

@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 
 from workloads import make_workload, make_time_samples
-from gpu_common import compare_epoch, make_scheduler, oracle_epoch
+from gpu_common import compare_epoch, make_scheduler, oracle_epoch, oracle_spread
 
 pytestmark = pytest.mark.gpu
 
@@ -488,23 +488,6 @@ def test_windows_without_a_usable_start_take_the_fallback(slaq, oracle_mod, pack
     assert sched.get_stats().fallback_jobs == 2 * n_bad
 
 
-def _oracle_spread(oracle_mod, wl, j, cap, n_trials=24):
-    """How far the oracle's own R(n) of job j moves when its losses are perturbed by 1e-13 relative: per n the
-    largest distance from the unperturbed result.  Zero to rounding for a fit that has finished; large where the
-    twenty trials end on a path-dependent point."""
-    h = wl.history(j)
-    off = np.array([0, h.size])
-    one = lambda a: np.array([a[j]])     # noqa: E731
-    base = np.cumsum(oracle_mod.predict(off, h, one(wl.m_seen), one(wl.s), one(wl.w), wl.epoch_seconds, cap)["gain"][0])
-    rng = np.random.default_rng(1000 + j)
-    spread = np.zeros_like(base)
-    for _ in range(n_trials):
-        hp = h * (1.0 + 1e-13 * rng.standard_normal(h.size))
-        R = np.cumsum(oracle_mod.predict(off, hp, one(wl.m_seen), one(wl.s), one(wl.w), wl.epoch_seconds, cap)["gain"][0])
-        spread = np.maximum(spread, np.abs(R - base))
-    return spread
-
-
 def test_unseen_cuts_survey(slaq, oracle_mod):
     """Cuts and seeds no other test uses, 100,000 jobs in all: how often does a job miss the tolerance on R(n), and
     why.  Twenty solver trials do not finish every fit.  Where the residual is nearly flat along a direction
@@ -533,7 +516,7 @@ def test_unseen_cuts_survey(slaq, oracle_mod):
                     S = ref["S"][j]
                     assert abs(S[0] - S[1]) <= 1e-9 * max(abs(S[0]), abs(S[1]))
                 for j in np.nonzero((width > 1.0) & ~tied)[0]:
-                    spread = _oracle_spread(oracle_mod, wl, j, cap)
+                    spread = oracle_spread(oracle_mod, wl, j, cap)
                     assert (np.abs(Rg[j] - Rc[j]) <= 4.0 * spread + tol[j]).all(), (
                         f"config {cfg}, {n} jobs, seed {seed}, job {j}: {width[j]:.2f} tolerances off, and the oracle's "
                         f"own result is stable ({(spread / tol[j]).max():.2f} tolerances under perturbation)")
