@@ -560,6 +560,11 @@ int do_load(slaq_handle* h, int32_t n, const int32_t* ids, const int64_t* offset
     return SLAQ_OK;
 }
 
+// Without a gain table: only the plain prediction (no envelope, no target-loss hints) has its gains in closed form.
+bool epoch_is_table_free(const slaq_handle* h, bool only_allocate) {
+    return !only_allocate && h->selection == 1 && !h->gain_envelope && h->n_hinted == 0;
+}
+
 // The launches of one epoch, put on h->stream in order.  Returns the number of kernels or -1.
 // with_events: the stage boundaries are marked with the handle's events (left out of a captured
 // graph: events recorded by a graph cannot be timed).
@@ -574,8 +579,7 @@ int enqueue_epoch(slaq_handle* h, double T, int64_t want, int floor_units, int32
         launches += k;
     }
     if (with_events && cudaEventRecord(h->ev[1], st) != cudaSuccess) return -1;
-    // Without a table: only the plain prediction (no envelope, no target-loss hints) has gains in closed form.
-    const bool table_free = !only_allocate && h->selection == 1 && !h->gain_envelope && h->n_hinted == 0;
+    const bool table_free = epoch_is_table_free(h, only_allocate);
     if (!only_allocate && !table_free) {
         if ((k = launch_gain(h, T, floor_units + 1)) < 0) return -1;
         launches += k;
@@ -585,9 +589,6 @@ int enqueue_epoch(slaq_handle* h, double T, int64_t want, int floor_units, int32
     else k = launch_allocate(h, want, floor_units + 1, !only_allocate, d_out);
     if (k < 0) return -1;
     launches += k;
-    h->gain_table_current = !table_free;
-    h->last_T = T;
-    h->last_first_unit = floor_units + 1;
     if (with_events && cudaEventRecord(h->ev[3], st) != cudaSuccess) return -1;
     return launches;
 }
@@ -678,6 +679,11 @@ int run_epoch(slaq_handle* h, double T, int64_t C, int32_t* d_out, bool only_all
     h->have_epoch = true;
     h->last_launches = launches;
     h->last_cores = usable;
+    // whether h->gain holds this epoch's rows (plain launches and a replayed graph alike), and what a later
+    // request for them has to be predicted for
+    h->gain_table_current = !epoch_is_table_free(h, only_allocate);
+    h->last_T = T;
+    h->last_first_unit = floor_units + 1;
     if (active > 0 && C < active) return SLAQ_W_OVERSUBSCRIBED;
     if (C > active * cap) return SLAQ_W_UNDERFILLED;
     return SLAQ_OK;
