@@ -602,7 +602,8 @@ std::vector<long long> epoch_key(const slaq_handle* h, double T, int64_t want, i
     std::memcpy(&g_bits, &h->gamma, sizeof g_bits);
     return {t_bits, (long long)want, floor_units, (long long)(uintptr_t)d_out, only_allocate ? 1 : 0, h->n_active,
             h->max_cores, h->lm_trials, h->min_fit_points, h->warm_start ? 1 : 0, (long long)h->fit_slice_bytes,
-            (long long)h->fit_cluster_jobs, g_bits, h->gain_envelope ? 1 : 0, h->selection, h->n_hinted};
+            (long long)h->fit_cluster_jobs, g_bits, h->gain_envelope ? 1 : 0, h->selection, h->n_hinted,
+            (long long)(uintptr_t)h->job.packed_lo, (long long)(uintptr_t)h->job.packed_hi};
 }
 
 int run_epoch(slaq_handle* h, double T, int64_t C, int32_t* d_out, bool only_allocate) {
