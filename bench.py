@@ -307,6 +307,9 @@ def run_gpu(args):
     # N x 100,000 jobs, one shard per rank, sums over NCCL.  Reported beside the headline, never instead of it. ----
     sharded = None
     try:
+        if world > 1 and not args.sharded:
+            raise RuntimeError("not run: with several GPUs this leg needs --sharded (its NCCL path has never run on "
+                               "hardware; a rank that failed inside it would leave the others waiting)")
         sched.set_param(slaq.binding.P_WARM_START, 0)
         sched.set_param(slaq.binding.P_LM_TRIALS, 20)
         reps = max(3, min(args.steps, 20))
@@ -425,6 +428,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--cfg", type=int, default=CFG, choices=[2, 3, 4],
                     help="profiling aid: another workload generator (the reported line is then not the benchmark)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="with --gpus N > 1: also time the N partitions as ONE cluster sharded over the ranks (NCCL)")
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
                     help="the block of --steps steps is repeated until the timed region lasts this long (0: one block; "
                          "for runs under a profiler)")
