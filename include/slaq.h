@@ -134,6 +134,8 @@ typedef struct slaq_stats {
     int32_t sublinear_wins;
     int32_t exponential_wins;
     int32_t fallback_jobs;
+    int32_t nonconvex_fits;  /* fitted jobs whose winning curve is not convex ahead of the newest point (family I with
+                                b^2 < a c): their marginal gains rise before they fall, see SLAQ_P_GAIN_ENVELOPE */
 } slaq_stats;
 
 /*

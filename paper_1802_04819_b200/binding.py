@@ -37,6 +37,7 @@ class Stats(ctypes.Structure):
         ("launches", c_int32), ("active_jobs", c_int32), ("cores_handed_out", c_int64), ("points", c_int64),
         ("model_sweeps", c_int64), ("tie_units", c_int64), ("threshold", c_double), ("fitted_jobs", c_int32),
         ("sublinear_wins", c_int32), ("exponential_wins", c_int32), ("fallback_jobs", c_int32),
+        ("nonconvex_fits", c_int32),
     ]
 
     def as_dict(self):

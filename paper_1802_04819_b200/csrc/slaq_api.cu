@@ -1426,6 +1426,7 @@ int slaq_get_stats(slaq_t* h, slaq_stats* out) {
     out->sublinear_wins = (int32_t)counters[3];
     out->exponential_wins = (int32_t)counters[4];
     out->fallback_jobs = (int32_t)counters[5];
+    out->nonconvex_fits = (int32_t)counters[14];
     out->cores_handed_out = counters[6];
     out->tie_units = counters[7];
     double tau = 0.0;

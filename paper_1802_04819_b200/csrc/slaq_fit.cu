@@ -592,7 +592,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
     const int even = lane & ~1, oddl = lane | 1;
 
     long long n_points = 0, n_sweep_points = 0;
-    int n_fit = 0, n_sub = 0, n_exp = 0, n_fallback = 0;
+    int n_fit = 0, n_sub = 0, n_exp = 0, n_fallback = 0, n_nonconvex = 0;
     SLAQ_PHASE_DECL;
     for (;;) {
         int slot = 0;
@@ -757,6 +757,8 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
                 n_fit += 1;
                 n_sub += family == 0;
                 n_exp += family == 1;
+                // 1/(a x^2 + b x + c) is convex for all x >= 0 exactly when b^2 >= a c
+                n_nonconvex += family == 0 && p_out[1] * p_out[1] < p_out[0] * p_out[2];
             } else if (status == SLAQ_JOB_SHORT || status == SLAQ_JOB_NEW || status == SLAQ_JOB_FIT_FAILED) {
                 n_fallback += 1;
             }
@@ -788,6 +790,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         n_sub += __shfl_xor_sync(kFull, n_sub, o);
         n_exp += __shfl_xor_sync(kFull, n_exp, o);
         n_fallback += __shfl_xor_sync(kFull, n_fallback, o);
+        n_nonconvex += __shfl_xor_sync(kFull, n_nonconvex, o);
     }
     if (lane == 0 && n_points > 0) {
         atomicAdd((unsigned long long*)&counters[0], (unsigned long long)n_points);
@@ -796,6 +799,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         atomicAdd((unsigned long long*)&counters[3], (unsigned long long)n_sub);
         atomicAdd((unsigned long long*)&counters[4], (unsigned long long)n_exp);
         atomicAdd((unsigned long long*)&counters[5], (unsigned long long)n_fallback);
+        atomicAdd((unsigned long long*)&counters[14], (unsigned long long)n_nonconvex);
     }
 #ifdef SLAQ_PHASE_CLOCKS
     if (lane == 0)

@@ -26,7 +26,12 @@ def test_envelope_rows_match_the_oracle(slaq, oracle_mod, cfg, n_jobs, cap):
         wl.max_cores_per_job = cap
     sched = make_scheduler(wl)
     plain, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
-    g_plain = sched.get_predictions()["gain"]
+    first = sched.get_predictions()
+    g_plain = first["gain"]
+    # the statistics count the fits that are not convex ahead: family I with b^2 < a c (typed here from the curve)
+    p = first["params"]
+    typed = int(((first["status"] == 0) & (first["family"] == 0) & (p[:, 1] ** 2 < p[:, 0] * p[:, 2])).sum())
+    assert sched.get_stats().nonconvex_fits == typed > 0
     sched.set_param(slaq.binding.P_GAIN_ENVELOPE, 1)
     assert sched.get_param(slaq.binding.P_GAIN_ENVELOPE) == 1
     alloc, rc = sched.schedule(wl.epoch_seconds, wl.total_cores)
