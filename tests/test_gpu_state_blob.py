@@ -107,3 +107,17 @@ def test_blobs_that_do_not_fit_are_refused_and_leave_the_handle_alone(slaq):
     empty = slaq.Scheduler(8, 16, 4)
     empty.import_state(empty.export_state())
     assert empty.get_active_count() == 0
+    # a handle that holds a packed pool (other jobs, other seed) gives it up when it imports
+    other = make_workload(1, seed_offset=3)
+    packed = slaq.Scheduler(J, wl.max_hist, cap)
+    packed.load_histories(ids, other.offsets, other.losses, other.k_last, other.m_seen, packed=True)
+    packed.set_time_model(ids, other.s, other.w)
+    packed.set_target_loss(ids[:5], other.losses[other.offsets[1:6] - 1] * 0.5)
+    packed.schedule(wl.epoch_seconds, wl.total_cores)
+    packed.import_state(blob)
+    np.testing.assert_array_equal(packed.schedule(wl.epoch_seconds, wl.total_cores)[0], before)
+    np.testing.assert_array_equal(packed.export_state()[64:], blob[64:])
+    packed.append_losses(ids, wl.losses[wl.offsets[1:] - 1] * 0.98, wl.s + wl.w)       # its rings take new losses
+    a.append_losses(ids, wl.losses[wl.offsets[1:] - 1] * 0.98, wl.s + wl.w)
+    np.testing.assert_array_equal(packed.schedule(wl.epoch_seconds, wl.total_cores)[0],
+                                  a.schedule(wl.epoch_seconds, wl.total_cores)[0])
