@@ -212,6 +212,21 @@ int slaq_append_losses_ex(slaq_t* h, int32_t n, const int32_t* job_ids, const do
                           const double* iter_times, const int32_t* cores_used);
 
 /*
+ * The same update with all four arrays in device memory (d_iter_times and d_cores_used may be NULL),
+ * asynchronous on the handle's stream and without any wait of the host: for trainers that reduce
+ * their losses on this GPU.  The host never sees the values, so what slaq_append_losses checks
+ * before it applies anything is checked per entry on the device instead: an id outside
+ * 0 .. max_jobs-1, a job that has no loss yet (a job's FIRST loss must come through
+ * slaq_append_losses or a bulk load, which also count it as active), a loss or time that is not
+ * finite, a core count below 1 - such an entry is skipped and the next slaq_schedule returns
+ * SLAQ_E_CUDA with a message that says so.  A job id listed twice in one call gives an unspecified
+ * order of its two updates.  The arrays must stay valid until the stream has passed the call.
+ * Errors: SLAQ_E_ARG (null, n < 0, n > max_jobs, cores without times).  The paper has no counterpart.
+ */
+int slaq_append_losses_device(slaq_t* h, int32_t n, const int32_t* d_job_ids, const double* d_losses,
+                              const double* d_iter_times, const int32_t* d_cores_used);
+
+/*
  * Bulk load: replace the stored window of n_jobs jobs.  Histories are ragged, in CSR
  * form: job job_ids[i] owns losses[offsets[i] .. offsets[i+1]), oldest first; k_last[i]
  * is the iteration index of its newest loss; m_seen[i] (array may be NULL) the largest

@@ -19,7 +19,8 @@ W_OVERSUBSCRIBED, W_UNDERFILLED = 1, 2
 
 EXPORTED_SYMBOLS = [
     "slaq_create", "slaq_create_in", "slaq_workspace_bytes", "slaq_destroy", "slaq_last_error", "slaq_set_stream",
-    "slaq_set_param", "slaq_get_param", "slaq_append_losses", "slaq_append_losses_ex", "slaq_load_histories",
+    "slaq_set_param", "slaq_get_param", "slaq_append_losses", "slaq_append_losses_ex", "slaq_append_losses_device",
+    "slaq_load_histories",
     "slaq_load_histories_packed", "slaq_set_time_model", "slaq_set_target_loss", "slaq_remove_jobs", "slaq_schedule",
     "slaq_schedule_device",
     "slaq_get_predictions", "slaq_get_normalised", "slaq_get_time_model", "slaq_get_fit_state",
@@ -74,6 +75,7 @@ def load_library(variant: str | None = None):
         "slaq_get_param": (c_int, [vp, c_int, POINTER(c_double)]),
         "slaq_append_losses": (c_int, [vp, c_int32, vp, vp, vp]),
         "slaq_append_losses_ex": (c_int, [vp, c_int32, vp, vp, vp, vp]),
+        "slaq_append_losses_device": (c_int, [vp, c_int32, vp, vp, vp, vp]),
         "slaq_load_histories": (c_int, [vp, c_int32, vp, vp, vp, vp, vp]),
         "slaq_load_histories_packed": (c_int, [vp, c_int32, vp, vp, vp, vp, vp]),
         "slaq_set_time_model": (c_int, [vp, c_int32, vp, vp, vp]),
@@ -213,6 +215,14 @@ class Scheduler:
         if cs is None:
             return self._check(self._lib.slaq_append_losses(self._h, ids.size, _ptr(ids), _ptr(ls), _ptr(ts)))
         return self._check(self._lib.slaq_append_losses_ex(self._h, ids.size, _ptr(ids), _ptr(ls), _ptr(ts), _ptr(cs)))
+
+    def append_losses_device(self, d_job_ids, d_losses, d_iter_times=None, d_cores_used=None):
+        """One new iteration per listed job from torch CUDA tensors (int32 ids, float64 losses and times, int32
+        cores), asynchronous on the handle's stream; only for jobs that already have a loss."""
+        ptr = lambda t: None if t is None else c_void_p(t.data_ptr())   # noqa: E731
+        assert d_job_ids.is_contiguous() and d_losses.is_contiguous() and d_job_ids.numel() == d_losses.numel()
+        return self._check(self._lib.slaq_append_losses_device(self._h, d_job_ids.numel(), ptr(d_job_ids), ptr(d_losses),
+                                                               ptr(d_iter_times), ptr(d_cores_used)))
 
     def load_histories(self, job_ids, offsets, losses, k_last, m_seen=None, packed=False):
         ids, off = _arr(job_ids, np.int32), _arr(offsets, np.int64)

@@ -158,13 +158,27 @@ __global__ void init_jobs_kernel(JobArrays job, FitArrays fit, double* ring, int
 
 // One new iteration per listed job: ring write, iteration index, largest reduction seen,
 // and the sums of the iteration-time law (booked at the given or the current core count).
+// checked: the arrays come straight from the caller's device memory, unseen by the host - an id out of range,
+// a job without any loss yet, a loss or time that is not finite or a core count below 1 sets kErrInput and
+// that entry is skipped.
 __global__ void append_kernel(JobArrays job, FitArrays fit, int max_jobs, int n, const int32_t* ids,
-                              const double* losses, const double* times, const int32_t* cores) {
+                              const double* losses, const double* times, const int32_t* cores, int checked) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const int j = ids[i];
-    if (j < 0 || j >= max_jobs) return;
+    if (j < 0 || j >= max_jobs) {
+        if (checked) atomicOr(job.err_word, kErrInput);
+        return;
+    }
     const double loss = losses[i];
+    if (checked) {
+        const bool bad = !(fabs(loss) <= 1.7976931348623157e308) || job.count[j] <= 0 ||
+                         (times && !(fabs(times[i]) <= 1.7976931348623157e308)) || (times && cores && cores[i] < 1);
+        if (bad) {
+            atomicOr(job.err_word, kErrInput);
+            return;
+        }
+    }
     double* row = job.row[j];
     const int cap = job.cap[j];
     int head = job.head[j];
@@ -336,6 +350,8 @@ int check_device_errors(slaq_handle* h) {
         if (word & kErrSegment) what += " a candidate segment outside its row;";
         if (word & kErrBin) what += " a histogram bin out of range;";
         if (word & kErrJob) what += " a job id out of range;";
+        if (word & kErrInput) what += " slaq_append_losses_device was given an id out of range, a job without losses, a value that is not finite or a core count below 1 (those entries were skipped);";
+        cudaMemsetAsync(h->err_word, 0, sizeof word, h->stream);   // reported once: the next epoch starts clean
         return fail(h, SLAQ_E_CUDA, what);
     }
     return SLAQ_OK;
@@ -439,7 +455,7 @@ int do_append(slaq_handle* h, int32_t n, const int32_t* ids, const double* losse
     const int threads = 256;
     append_kernel<<<(n + threads - 1) / threads, threads, 0, st>>>(
         h->job, h->fit, h->max_jobs, n, h->stage.ids, h->stage.losses, times ? h->stage.times : nullptr,
-        (times && cores) ? h->stage.cores : nullptr);
+        (times && cores) ? h->stage.cores : nullptr, 0);
     CK(cudaGetLastError(), "append kernel");
     CK(cudaStreamSynchronize(st), "append");   // the caller may reuse its buffers
     if (h->n_active < h->max_jobs) {   // nothing to do once every id is active
@@ -823,6 +839,22 @@ int slaq_append_losses(slaq_t* h, int32_t n, const int32_t* job_ids, const doubl
 int slaq_append_losses_ex(slaq_t* h, int32_t n, const int32_t* job_ids, const double* losses, const double* iter_times,
                           const int32_t* cores_used) {
     return do_append(h, n, job_ids, losses, iter_times, cores_used);
+}
+
+int slaq_append_losses_device(slaq_t* h, int32_t n, const int32_t* d_job_ids, const double* d_losses,
+                               const double* d_iter_times, const int32_t* d_cores_used) {
+    if (!h) return SLAQ_E_ARG;
+    if (const int dc = check_device(h)) return dc;
+    if (n < 0) return fail(h, SLAQ_E_ARG, "negative count");
+    if (n > h->max_jobs) return fail(h, SLAQ_E_ARG, "more entries than job ids");
+    if (n > 0 && (!d_job_ids || !d_losses)) return fail(h, SLAQ_E_ARG, "job_ids or losses is null");
+    if (d_cores_used && !d_iter_times) return fail(h, SLAQ_E_ARG, "cores_used without iter_times");
+    if (n == 0) return SLAQ_OK;
+    const int threads = 256;
+    append_kernel<<<(n + threads - 1) / threads, threads, 0, h->stream>>>(h->job, h->fit, h->max_jobs, n, d_job_ids, d_losses,
+                                                                        d_iter_times, d_cores_used, 1);
+    CK(cudaGetLastError(), "append kernel");
+    return SLAQ_OK;
 }
 
 int slaq_load_histories(slaq_t* h, int32_t n_jobs, const int32_t* job_ids, const int64_t* offsets, const double* losses,

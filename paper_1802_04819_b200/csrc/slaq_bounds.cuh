@@ -5,7 +5,7 @@
 
 namespace slaq {
 
-// Bits of the device error word (slaq_handle::err_word).  kErrWindow is set by every build; the
+// Bits of the device error word (slaq_handle::err_word).  kErrWindow and kErrInput are set by every build; the
 // others only by the "bounds" build (-DSLAQ_DEBUG_BOUNDS), in which every index into a ring, the
 // packed pool, a shared-memory slice, the gain table, a candidate segment, a histogram or a per-job
 // array is compared with its extent first: a bad index sets its bit and the access is skipped (a
@@ -17,7 +17,8 @@ enum : int32_t {
     kErrGain = 8,       // an entry outside the gain table
     kErrSegment = 16,   // a candidate segment that does not lie inside its row
     kErrBin = 32,       // a histogram bin or window-length bucket out of range
-    kErrJob = 64        // a job id or work-list position out of range
+    kErrJob = 64,       // a job id or work-list position out of range
+    kErrInput = 128     // set by every build: device-side input of slaq_append_losses_device that had to be skipped
 };
 
 #ifdef SLAQ_DEBUG_BOUNDS

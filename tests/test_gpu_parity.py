@@ -561,3 +561,54 @@ def test_streaming_epochs_with_allocation_feedback(slaq, oracle_mod):
         np.testing.assert_array_equal(w, out["w"])
         alloc = got.copy()
     assert (k_next >= 7).all()
+
+
+def test_appends_from_device_memory(slaq, oracle_mod):
+    """slaq_append_losses_device: the same update as the host call, from CUDA tensors and without a host wait; what
+    the host call would refuse is skipped on the device and reported by the next epoch."""
+    import torch
+    wl = make_workload(1)
+    J, cap, max_hist = wl.n_jobs, wl.max_cores_per_job, 24
+    sched = slaq.Scheduler(J, max_hist, cap)
+    ref = oracle_mod.OracleScheduler(J, max_hist, cap)
+    ids = np.arange(J, dtype=np.int32)
+    rng = np.random.default_rng(12)
+    d_ids = torch.arange(J, dtype=torch.int32, device="cuda")
+    first = wl.losses[wl.offsets[:-1]]
+    sched.append_losses(ids, first, wl.s + wl.w)                  # the first loss activates a job: host call
+    ref.append_losses(ids, first, wl.s + wl.w)
+    for step in range(1, 40):                                    # the ring of 24 wraps
+        losses = first / (1.0 + 0.2 * step) * np.exp(0.01 * rng.standard_normal(J))
+        cores = np.full(J, 1 + step % 4, np.int32)
+        times = wl.s + wl.w / cores
+        sched.append_losses_device(d_ids, torch.from_numpy(losses).cuda(), torch.from_numpy(times).cuda(),
+                                   torch.from_numpy(cores).cuda())
+        ref.append_losses(ids, losses, times, cores)
+        if step % 13 == 0:
+            alloc, rc = sched.schedule(wl.epoch_seconds, wl.total_cores)
+            out = ref.schedule(wl.epoch_seconds, wl.total_cores)
+            compare_epoch(alloc, sched.get_predictions(), out, wl.total_cores, cap)
+            s, w = sched.get_time_model()
+            np.testing.assert_array_equal(s, out["s"])
+            np.testing.assert_array_equal(w, out["w"])
+    good, _ = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    # entries the host call would refuse: skipped, reported once, and the state is as before
+    bad_ids = torch.tensor([0, 1, J + 5, 2], dtype=torch.int32, device="cuda")
+    bad_losses = torch.tensor([float("nan"), float("inf"), 1.0, 1.0], dtype=torch.float64, device="cuda")
+    bad_times = torch.tensor([1.0, 1.0, 1.0, float("nan")], dtype=torch.float64, device="cuda")
+    sched.append_losses_device(bad_ids, bad_losses, bad_times)
+    with pytest.raises(slaq.SlaqError) as err:
+        sched.schedule(wl.epoch_seconds, wl.total_cores)
+    assert err.value.code == -5 and "slaq_append_losses_device" in str(err.value)
+    again, rc = sched.schedule(wl.epoch_seconds, wl.total_cores)
+    assert rc == 0
+    np.testing.assert_array_equal(again, good)
+    fresh = slaq.Scheduler(4, 8, 2)                               # a job's first loss cannot come this way
+    fresh.append_losses_device(torch.zeros(1, dtype=torch.int32, device="cuda"),
+                               torch.ones(1, dtype=torch.float64, device="cuda"))
+    with pytest.raises(slaq.SlaqError):
+        fresh.schedule(1.0, 4)
+    assert fresh.get_active_count() == 0
+    with pytest.raises(slaq.SlaqError):
+        sched.append_losses_device(d_ids, torch.ones(J, dtype=torch.float64, device="cuda"), None,
+                                   torch.ones(J, dtype=torch.int32, device="cuda"))
