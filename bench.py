@@ -39,9 +39,9 @@ FP64_LANES_PER_SM = 64          # fp64 FMA lanes per SM on B200
 SWEEP_ISSUE_CYCLES_IDEAL, SWEEP_ISSUE_CYCLES_MEASURED_RATES = 92.0, 107.0
 MIN_TIMED_SECONDS = 1.0   # the block of --steps steps is repeated until the timed region is at least this long
 # DRAM bytes per stored loss moved by the fit kernel (ncu: dram__bytes_read.sum + dram__bytes_write.sum =
-# 165.85 MB + 13.68 MB on a 20,068,408-loss cut of this workload, profiles/fit_kernel_40k_jobs.md; traffic grows
+# 165.75 MB + 13.79 MB on a 20,068,408-loss cut of this workload, profiles/fit_kernel_40k_jobs.md; traffic grows
 # with the stored losses)
-NCU_FIT_DRAM_BYTES_PER_LOSS = (165.85e6 + 13.68e6) / 20_068_408
+NCU_FIT_DRAM_BYTES_PER_LOSS = (165.75e6 + 13.79e6) / 20_068_408
 
 
 from paper_1802_04819_b200.partition import max_over_ranks, partition_seed_offset, rank_info, whole_job_rate  # noqa: E402

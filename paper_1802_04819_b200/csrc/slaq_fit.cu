@@ -626,6 +626,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
         double S_out[2] = {CUDART_INF, CUDART_INF};
         int sweeps_out[2] = {0, 0};
         int ended = 0;   // bit 0 / 1: family I / II ended with a finite residual
+        bool any_ended = false;
         double both_out[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};   // both families' end points
         const double span = (double)max(H - 1, 1);
         const bool fits = status == SLAQ_JOB_FITTED && H >= min_fit_points;   // this lane's job gets curves fitted
@@ -719,6 +720,9 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
                 if (ok_II) S_out[1] = S_II;
                 const bool okI = ok_I && finite_d(S_I), okII = ok_II && finite_d(S_II);
                 ended = (okI ? 1 : 0) | (okII ? 2 : 0);
+                // Kept as a flag of its own: a branch on `ended` placed here was compiled as never taken (nvcc 12.9,
+                // also with ptxas -O1) although the same value, stored below, is non-zero; a branch on okI || okII is taken.
+                any_ended = okI || okII;
 #pragma unroll
                 for (int a = 0; a < 4; ++a) both_out[a] = pI[a], both_out[4 + a] = pII[a];
                 if (okI && (!okII || S_I <= S_II)) {   // a tie goes to family I
@@ -764,7 +768,7 @@ fit_kernel(JobArrays job, FitArrays fit, const double* __restrict__ g_wtab, cons
             }
             fit.status[j] = status;
             fit.mask[j] = (uint8_t)ended;
-            if (ended) {   // what the next epoch may start from
+            if (any_ended) {   // what the next epoch may start from
                 fit.k_fit[j] = job.k_last[j];
 #pragma unroll
                 for (int a = 0; a < 8; ++a) fit.both[8 * (size_t)j + a] = both_out[a];
