@@ -68,33 +68,62 @@ struct SweepSums {
     bool usable;   // the model was defined at every point and all sums are finite
 };
 
+// Running sums to sums of powers of x.  A lane walks its points from the oldest to the newest and keeps, for a
+// weighted value a, the chain c0 += a, c1 += c0, c2 += c1, ... in which every link adds the value its
+// predecessor had one step earlier; after the walk c_p = sum a_k C(k, p), k = the row of the point counted from
+// the lane's newest.  Powers of k are fixed combinations with positive coefficients (k^2 = 2 C(k,2) + C(k,1),
+// k^3 = 6 C(k,3) + 6 C(k,2) + C(k,1), k^4 = 24 C(k,4) + 36 C(k,3) + 14 C(k,2) + C(k,1)); with x = x_l + g k
+// (x_l <= 0 the lane's newest point, g < 0 the row pitch) the powers of x follow from a scaling by g^p and a shift
+// of the origin, all of whose terms have the sign of (-1)^p: nothing cancels, the sums are as accurate as if the
+// powers had been multiplied out point by point.
+template <int P>
+__device__ __forceinline__ void chains_to_powers(double (&c)[P], double x_l, double g) {
+    const double c1 = P > 1 ? c[1] : 0.0, c2 = P > 2 ? c[2] : 0.0, c3 = P > 3 ? c[3] : 0.0;
+    if (P > 2) c[2] = fma(2.0, c2, c1);
+    if (P > 3) c[3] = fma(6.0, c3, fma(6.0, c2, c1));
+    if (P > 4) c[4] = fma(24.0, c[4], fma(36.0, c3, fma(14.0, c2, c1)));
+    double gp = g;
+#pragma unroll
+    for (int i = 1; i < P; ++i, gp *= g) c[i] *= gp;
+#pragma unroll
+    for (int j = 1; j < P; ++j)
+#pragma unroll
+        for (int p = P - 1; p >= j; --p) c[p] = fma(x_l, c[p - 1], c[p]);
+}
+
 // One sweep over the window: both families at once, each at its own point.  A lane adds up
-// both families over its points; the first reduction step hands each lane of a pair the other
-// lane's partial sums of its own family, the remaining steps run over lanes of the same parity.
+// both families over its points, oldest first, as running sums (see chains_to_powers: in the loop
+// every accumulation but the two objectives is an addition of two registers, which the fp64 pipe
+// issues in two cycles where a fused multiply-add on three registers takes three); the first
+// reduction step hands each lane of a pair the other lane's partial sums of its own family, the
+// remaining steps run over lanes of the same parity.
 __device__ __forceinline__ void sweep(const Lanes& S, int fam, int H, int k_all, double inv_span,
                                       const double (&pI)[4], bool doI, const double (&pII)[4], bool doII,
                                       SweepSums& out) {
-    double m0 = 0, m1 = 0, m2 = 0, m3 = 0, m4 = 0, n0 = 0, n1 = 0, n2 = 0, h0 = 0, h1 = 0, h2 = 0, gd = 0, sI = 0;
-    double e0 = 0, e1 = 0, e2 = 0, f0 = 0, f1 = 0, k0 = 0, k1 = 0, gc = 0, sII = 0;
+    double m[5] = {0, 0, 0, 0, 0}, n[3] = {0, 0, 0}, h[3] = {0, 0, 0}, gd = 0, sI = 0;
+    double ee[3] = {0, 0, 0}, f[2] = {0, 0}, kk[2] = {0, 0}, gc = 0, sII = 0;
     int feasible = 1;
-    // e = exp(alpha - beta x) with x = -m / span grows geometrically with m: one exact value at
-    // the lane's newest point, then a constant ratio per step.  The rounding of the recurrence
-    // accumulates towards the old points, whose weights gamma^m have long vanished.
+    const int shift = __ffs(S.L) - 1;                                      // L is a power of two
+    const int k_last = H - 1 - S.l >= 0 ? (H - 1 - S.l) >> shift : -1;     // the row of the lane's oldest point
+    int mi = S.l + (k_last << shift);
+    double md = (double)mi;
+    const double dL = (double)S.L;
+    // e = exp(alpha - beta x) with x = -m / span falls geometrically towards the newest point: one
+    // exact value at the lane's oldest point, then a constant ratio per step.  (Choosing the start such
+    // that the recurrence lands on the exact value at the newest point was measured: the predictions stay
+    // as close to the reference's either way, and the extra arithmetic costs 2 % of the kernel.)
     double e = 0.0, ratio = 1.0;
     if (doII) {
-        e = exp(fma(pII[1], (double)S.l * inv_span, pII[0]));
-        ratio = exp(pII[1] * ((double)S.L * inv_span));
+        e = exp(fma(pII[1], md * inv_span, pII[0]));
+        ratio = exp(-pII[1] * (dL * inv_span));
     }
-    double md = (double)S.l;
-    const double dL = (double)S.L;
-    const double* yp = S.y + S.lane;
+    const double* yp = S.y + S.lane + k_last * 32;
 #pragma unroll 1   // unrolling only adds register pressure here: the body already holds 22 independent sums
-    for (int k = 0, m = S.l; k < k_all; ++k, m += S.L, md += dL, yp += 32) {
-        if (m < H) {
+    for (int i = 0, k = k_last; i < k_all; ++i, --k, mi -= S.L, md -= dL, yp -= 32) {
+        if (k >= 0) {
             const double x = -md * inv_span;
-            const double w = S.weight(m);
+            const double w = S.weight(mi);
             const double y = S.holds(yp) ? *yp : 0.0;
-            const double x2 = x * x;
             if (doI) {
                 const double q = fma(fma(pI[0], x, pI[1]), x, pI[2]);
                 feasible &= q > 0.0 ? 1 : 0;
@@ -102,46 +131,41 @@ __device__ __forceinline__ void sweep(const Lanes& S, int fam, int H, int k_all,
                 const double r = y - (inv + pI[3]);
                 const double u = inv * inv;
                 const double wu = w * u, wuu = wu * u, wur = wu * r, wr = w * r;
-                const double t = wuu * x2;
-                m0 += wuu;
-                m1 = fma(wuu, x, m1);
-                m2 += t;
-                m3 = fma(t, x, m3);
-                m4 = fma(t, x2, m4);
-                n0 += wu;
-                n1 = fma(wu, x, n1);
-                n2 = fma(wu, x2, n2);
-                h0 += wur;
-                h1 = fma(wur, x, h1);
-                h2 = fma(wur, x2, h2);
+                m[4] += m[3]; m[3] += m[2]; m[2] += m[1]; m[1] += m[0]; m[0] += wuu;
+                n[2] += n[1]; n[1] += n[0]; n[0] += wu;
+                h[2] += h[1]; h[1] += h[0]; h[0] += wur;
                 gd += wr;
                 sI = fma(wr, r, sI);
             }
             if (doII) {
                 const double r = y - (e + pII[2]);
                 const double we = w * e, wee = we * e, wer = we * r, wr = w * r;
-                e0 += wee;
-                e1 = fma(wee, x, e1);
-                e2 = fma(wee, x2, e2);
-                f0 += we;
-                f1 = fma(we, x, f1);
-                k0 += wer;
-                k1 = fma(wer, x, k1);
+                ee[2] += ee[1]; ee[1] += ee[0]; ee[0] += wee;
+                f[1] += f[0]; f[0] += we;
+                kk[1] += kk[0]; kk[0] += wer;
                 gc += wr;
                 sII = fma(wr, r, sII);
             }
+            e *= ratio;
         }
-        e *= ratio;
     }
+    const double x_l = -(double)S.l * inv_span, g = -dL * inv_span;
+    chains_to_powers(m, x_l, g);
+    chains_to_powers(n, x_l, g);
+    chains_to_powers(h, x_l, g);
+    chains_to_powers(ee, x_l, g);
+    chains_to_powers(f, x_l, g);
+    chains_to_powers(kk, x_l, g);
     // pair step: an even lane hands over its family-II partials and receives family-I ones, an odd lane the reverse
     const bool odd = fam != 0;
     double v[13];
 #define SLAQ_PAIR(k, a, b) v[k] = (odd ? (b) : (a)) + __shfl_xor_sync(kFull, odd ? (a) : (b), 1)
-    SLAQ_PAIR(0, m0, e0); SLAQ_PAIR(1, m1, e1); SLAQ_PAIR(2, m2, e2); SLAQ_PAIR(3, m3, f0); SLAQ_PAIR(4, m4, f1);
-    SLAQ_PAIR(5, n0, k0); SLAQ_PAIR(6, n1, k1); SLAQ_PAIR(7, n2, gc); SLAQ_PAIR(8, h0, sII);
+    SLAQ_PAIR(0, m[0], ee[0]); SLAQ_PAIR(1, m[1], ee[1]); SLAQ_PAIR(2, m[2], ee[2]); SLAQ_PAIR(3, m[3], f[0]);
+    SLAQ_PAIR(4, m[4], f[1]); SLAQ_PAIR(5, n[0], kk[0]); SLAQ_PAIR(6, n[1], kk[1]); SLAQ_PAIR(7, n[2], gc);
+    SLAQ_PAIR(8, h[0], sII);
 #undef SLAQ_PAIR
-    v[9] = h1 + __shfl_xor_sync(kFull, h1, 1);    // family I only: odd lanes carry these along unused
-    v[10] = h2 + __shfl_xor_sync(kFull, h2, 1);
+    v[9] = h[1] + __shfl_xor_sync(kFull, h[1], 1);    // family I only: odd lanes carry these along unused
+    v[10] = h[2] + __shfl_xor_sync(kFull, h[2], 1);
     v[11] = gd + __shfl_xor_sync(kFull, gd, 1);
     v[12] = sI + __shfl_xor_sync(kFull, sI, 1);
     feasible &= __shfl_xor_sync(kFull, feasible, 1);
