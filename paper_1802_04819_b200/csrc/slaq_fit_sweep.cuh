@@ -46,6 +46,9 @@ struct Lanes {
     __device__ __forceinline__ double weight(int m) const {
         return index_ok(m, wtab_len, kErrShared, err_word) ? wtab[m] : 0.0;
     }
+    __device__ __forceinline__ double weight(const double* p) const {   // p = wtab + m
+        return index_ok(p - wtab, wtab_len, kErrShared, err_word) ? *p : 0.0;
+    }
     __device__ __forceinline__ double level(int k) const {   // the lane's point of row k
         const double* p = y + k * 32 + lane;
         return holds(p) ? *p : 0.0;
@@ -91,6 +94,67 @@ __device__ __forceinline__ void chains_to_powers(double (&c)[P], double x_l, dou
         for (int p = P - 1; p >= j; --p) c[p] = fma(x_l, c[p - 1], c[p]);
 }
 
+// The running sums of one lane: family I (m: w u^2, n: w u, h: w u r, gd: w r, sI: w r^2 with u = 1/q^2) and
+// family II (ee: w e^2, f: w e, kk: w e r, gc: w r, sII: w r^2).
+struct LaneSums {
+    double m[5], n[3], h[3], gd, sI;
+    double ee[3], f[2], kk[2], gc, sII;
+    int q_signs;     // OR of the high words of family I's denominators: negative if one of them had its sign bit set
+};
+
+// The walk over a lane's rows, oldest first.  kI / kII: whether the family is evaluated at all - the same for
+// the whole warp, so that the loop has no branch per family (a lane whose family has no trial computes it at
+// parameters nobody uses and its sums are discarded).
+template <bool kI, bool kII>
+__device__ __forceinline__ void walk_rows(const Lanes& S, int k_last, int k_all, double inv_span,
+                                          const double (&pI)[4], const double (&pII)[4], LaneSums& a) {
+    const int mi = S.l + k_last * S.L;
+    double md = (double)mi;
+    const double dL = (double)S.L;
+    // e = exp(alpha - beta x) with x = -m / span falls geometrically towards the newest point: one
+    // exact value at the lane's oldest point, then a constant ratio per step.  (Choosing the start such
+    // that the recurrence lands on the exact value at the newest point was measured: the predictions stay
+    // as close to the reference's either way, and the extra arithmetic costs 2 % of the kernel.)
+    double e = 0.0, ratio = 1.0;
+    if (kII) {
+        e = exp(fma(pII[1], md * inv_span, pII[0]));
+        ratio = exp(-pII[1] * (dL * inv_span));
+    }
+    const double* yp = S.y + S.lane + k_last * 32;
+    const double* wp = S.wtab + mi;
+#pragma unroll 1   // unrolling only adds register pressure here: the body already holds 22 independent sums
+    for (int i = 0; i < k_all; ++i, md -= dL, yp -= 32, wp -= S.L) {
+        if (i <= k_last) {   // rows k_last - i >= 0: the lane's own points
+            const double w = S.weight(wp);
+            const double y = S.holds(yp) ? *yp : 0.0;
+            if (kI) {
+                const double x = -md * inv_span;
+                const double q = fma(fma(pI[0], x, pI[1]), x, pI[2]);
+                a.q_signs |= __double2hiint(q);   // q = 0 or NaN makes the sums non-finite, which the caller sees
+                const double inv = fast_rcp(q);
+                const double r = y - (inv + pI[3]);
+                const double u = inv * inv;
+                const double wu = w * u, wuu = wu * u, wur = wu * r, wr = w * r;
+                a.m[4] += a.m[3]; a.m[3] += a.m[2]; a.m[2] += a.m[1]; a.m[1] += a.m[0]; a.m[0] += wuu;
+                a.n[2] += a.n[1]; a.n[1] += a.n[0]; a.n[0] += wu;
+                a.h[2] += a.h[1]; a.h[1] += a.h[0]; a.h[0] += wur;
+                a.gd += wr;
+                a.sI = fma(wr, r, a.sI);
+            }
+            if (kII) {
+                const double r = y - (e + pII[2]);
+                const double we = w * e, wee = we * e, wer = we * r, wr = w * r;
+                a.ee[2] += a.ee[1]; a.ee[1] += a.ee[0]; a.ee[0] += wee;
+                a.f[1] += a.f[0]; a.f[0] += we;
+                a.kk[1] += a.kk[0]; a.kk[0] += wer;
+                a.gc += wr;
+                a.sII = fma(wr, r, a.sII);
+                e *= ratio;
+            }
+        }
+    }
+}
+
 // One sweep over the window: both families at once, each at its own point.  A lane adds up
 // both families over its points, oldest first, as running sums (see chains_to_powers: in the loop
 // every accumulation but the two objectives is an addition of two registers, which the fp64 pipe
@@ -100,55 +164,20 @@ __device__ __forceinline__ void chains_to_powers(double (&c)[P], double x_l, dou
 __device__ __forceinline__ void sweep(const Lanes& S, int fam, int H, int k_all, double inv_span,
                                       const double (&pI)[4], bool doI, const double (&pII)[4], bool doII,
                                       SweepSums& out) {
-    double m[5] = {0, 0, 0, 0, 0}, n[3] = {0, 0, 0}, h[3] = {0, 0, 0}, gd = 0, sI = 0;
-    double ee[3] = {0, 0, 0}, f[2] = {0, 0}, kk[2] = {0, 0}, gc = 0, sII = 0;
-    int feasible = 1;
+    LaneSums a = {};
     const int shift = __ffs(S.L) - 1;                                      // L is a power of two
     const int k_last = H - 1 - S.l >= 0 ? (H - 1 - S.l) >> shift : -1;     // the row of the lane's oldest point
-    int mi = S.l + (k_last << shift);
-    double md = (double)mi;
+    const bool anyI = __any_sync(kFull, doI), anyII = __any_sync(kFull, doII);
+    if (anyI && anyII) {
+        walk_rows<true, true>(S, k_last, k_all, inv_span, pI, pII, a);
+    } else {   // one family has no trial left in the whole warp
+        if (anyI) walk_rows<true, false>(S, k_last, k_all, inv_span, pI, pII, a);
+        if (anyII) walk_rows<false, true>(S, k_last, k_all, inv_span, pI, pII, a);
+    }
+    double (&m)[5] = a.m, (&n)[3] = a.n, (&h)[3] = a.h, (&ee)[3] = a.ee, (&f)[2] = a.f, (&kk)[2] = a.kk;
+    const double gd = a.gd, sI = a.sI, gc = a.gc, sII = a.sII;
+    int feasible = a.q_signs >= 0 ? 1 : 0;
     const double dL = (double)S.L;
-    // e = exp(alpha - beta x) with x = -m / span falls geometrically towards the newest point: one
-    // exact value at the lane's oldest point, then a constant ratio per step.  (Choosing the start such
-    // that the recurrence lands on the exact value at the newest point was measured: the predictions stay
-    // as close to the reference's either way, and the extra arithmetic costs 2 % of the kernel.)
-    double e = 0.0, ratio = 1.0;
-    if (doII) {
-        e = exp(fma(pII[1], md * inv_span, pII[0]));
-        ratio = exp(-pII[1] * (dL * inv_span));
-    }
-    const double* yp = S.y + S.lane + k_last * 32;
-#pragma unroll 1   // unrolling only adds register pressure here: the body already holds 22 independent sums
-    for (int i = 0, k = k_last; i < k_all; ++i, --k, mi -= S.L, md -= dL, yp -= 32) {
-        if (k >= 0) {
-            const double x = -md * inv_span;
-            const double w = S.weight(mi);
-            const double y = S.holds(yp) ? *yp : 0.0;
-            if (doI) {
-                const double q = fma(fma(pI[0], x, pI[1]), x, pI[2]);
-                feasible &= q > 0.0 ? 1 : 0;
-                const double inv = fast_rcp(q);
-                const double r = y - (inv + pI[3]);
-                const double u = inv * inv;
-                const double wu = w * u, wuu = wu * u, wur = wu * r, wr = w * r;
-                m[4] += m[3]; m[3] += m[2]; m[2] += m[1]; m[1] += m[0]; m[0] += wuu;
-                n[2] += n[1]; n[1] += n[0]; n[0] += wu;
-                h[2] += h[1]; h[1] += h[0]; h[0] += wur;
-                gd += wr;
-                sI = fma(wr, r, sI);
-            }
-            if (doII) {
-                const double r = y - (e + pII[2]);
-                const double we = w * e, wee = we * e, wer = we * r, wr = w * r;
-                ee[2] += ee[1]; ee[1] += ee[0]; ee[0] += wee;
-                f[1] += f[0]; f[0] += we;
-                kk[1] += kk[0]; kk[0] += wer;
-                gc += wr;
-                sII = fma(wr, r, sII);
-            }
-            e *= ratio;
-        }
-    }
     const double x_l = -(double)S.l * inv_span, g = -dL * inv_span;
     chains_to_powers(m, x_l, g);
     chains_to_powers(n, x_l, g);
