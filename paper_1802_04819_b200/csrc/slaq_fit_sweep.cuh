@@ -102,9 +102,43 @@ struct LaneSums {
     int q_signs;     // OR of the high words of family I's denominators: negative if one of them had its sign bit set
 };
 
+// One point of a lane's walk: both families' values at the point and their running sums.
+template <bool kI, bool kII>
+__device__ __forceinline__ void add_point(const Lanes& S, const double* wp, const double* yp, double md, double inv_span,
+                                          const double (&pI)[4], const double (&pII)[4], double& e, double ratio,
+                                          LaneSums& a) {
+    const double w = S.weight(wp);
+    const double y = S.holds(yp) ? *yp : 0.0;
+    if (kI) {
+        const double x = -md * inv_span;
+        const double q = fma(fma(pI[0], x, pI[1]), x, pI[2]);
+        a.q_signs |= __double2hiint(q);   // q = 0 or NaN makes the sums non-finite, which the caller sees
+        const double inv = fast_rcp(q);
+        const double r = y - (inv + pI[3]);
+        const double u = inv * inv;
+        const double wu = w * u, wuu = wu * u, wur = wu * r, wr = w * r;
+        a.m[4] += a.m[3]; a.m[3] += a.m[2]; a.m[2] += a.m[1]; a.m[1] += a.m[0]; a.m[0] += wuu;
+        a.n[2] += a.n[1]; a.n[1] += a.n[0]; a.n[0] += wu;
+        a.h[2] += a.h[1]; a.h[1] += a.h[0]; a.h[0] += wur;
+        a.gd += wr;
+        a.sI = fma(wr, r, a.sI);
+    }
+    if (kII) {
+        const double r = y - (e + pII[2]);
+        const double we = w * e, wee = we * e, wer = we * r, wr = w * r;
+        a.ee[2] += a.ee[1]; a.ee[1] += a.ee[0]; a.ee[0] += wee;
+        a.f[1] += a.f[0]; a.f[0] += we;
+        a.kk[1] += a.kk[0]; a.kk[0] += wer;
+        a.gc += wr;
+        a.sII = fma(wr, r, a.sII);
+        e *= ratio;
+    }
+}
+
 // The walk over a lane's rows, oldest first.  kI / kII: whether the family is evaluated at all - the same for
 // the whole warp, so that the loop has no branch per family (a lane whose family has no trial computes it at
-// parameters nobody uses and its sums are discarded).
+// parameters nobody uses and its sums are discarded).  Branches inside the loop cost issue slots on every row:
+// the rows that every lane of the warp has are walked without a test, only the ragged rest with one.
 template <bool kI, bool kII>
 __device__ __forceinline__ void walk_rows(const Lanes& S, int k_last, int k_all, double inv_span,
                                           const double (&pI)[4], const double (&pII)[4], LaneSums& a) {
@@ -122,37 +156,13 @@ __device__ __forceinline__ void walk_rows(const Lanes& S, int k_last, int k_all,
     }
     const double* yp = S.y + S.lane + k_last * 32;
     const double* wp = S.wtab + mi;
-#pragma unroll 1   // unrolling only adds register pressure here: the body already holds 22 independent sums
-    for (int i = 0; i < k_all; ++i, md -= dL, yp -= 32, wp -= S.L) {
-        if (i <= k_last) {   // rows k_last - i >= 0: the lane's own points
-            const double w = S.weight(wp);
-            const double y = S.holds(yp) ? *yp : 0.0;
-            if (kI) {
-                const double x = -md * inv_span;
-                const double q = fma(fma(pI[0], x, pI[1]), x, pI[2]);
-                a.q_signs |= __double2hiint(q);   // q = 0 or NaN makes the sums non-finite, which the caller sees
-                const double inv = fast_rcp(q);
-                const double r = y - (inv + pI[3]);
-                const double u = inv * inv;
-                const double wu = w * u, wuu = wu * u, wur = wu * r, wr = w * r;
-                a.m[4] += a.m[3]; a.m[3] += a.m[2]; a.m[2] += a.m[1]; a.m[1] += a.m[0]; a.m[0] += wuu;
-                a.n[2] += a.n[1]; a.n[1] += a.n[0]; a.n[0] += wu;
-                a.h[2] += a.h[1]; a.h[1] += a.h[0]; a.h[0] += wur;
-                a.gd += wr;
-                a.sI = fma(wr, r, a.sI);
-            }
-            if (kII) {
-                const double r = y - (e + pII[2]);
-                const double we = w * e, wee = we * e, wer = we * r, wr = w * r;
-                a.ee[2] += a.ee[1]; a.ee[1] += a.ee[0]; a.ee[0] += wee;
-                a.f[1] += a.f[0]; a.f[0] += we;
-                a.kk[1] += a.kk[0]; a.kk[0] += wer;
-                a.gc += wr;
-                a.sII = fma(wr, r, a.sII);
-                e *= ratio;
-            }
-        }
-    }
+    const int k_min = __reduce_min_sync(kFull, k_last);
+    int i = 0;
+#pragma unroll 1   // unrolling was measured (2 rows per step): slower, more spills
+    for (; i <= k_min; ++i, md -= dL, yp -= 32, wp -= S.L) add_point<kI, kII>(S, wp, yp, md, inv_span, pI, pII, e, ratio, a);
+#pragma unroll 1
+    for (; i < k_all; ++i, md -= dL, yp -= 32, wp -= S.L)
+        if (i <= k_last) add_point<kI, kII>(S, wp, yp, md, inv_span, pI, pII, e, ratio, a);   // row k_last - i >= 0
 }
 
 // One sweep over the window: both families at once, each at its own point.  A lane adds up
