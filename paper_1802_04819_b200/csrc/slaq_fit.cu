@@ -130,14 +130,32 @@ __device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double 
     Normalised out;
     out.M = CUDART_NAN;
     out.rho = 0.0;
+    // Rows of the lane with a point (m < H), and with a point that has an older neighbour (m + 1 < H).  The rows
+    // that every lane of the warp has are walked without a test per row (a branch in these loops costs issue
+    // slots on every row), the ragged rest with one.
+    const int shift = __ffs(S.L) - 1;
+    const int rows = H - 1 - S.l >= 0 ? ((H - 1 - S.l) >> shift) + 1 : 0;
+    const int rows_nb = H - 2 - S.l >= 0 ? ((H - 2 - S.l) >> shift) + 1 : 0;
+    const int full_nb = __reduce_min_sync(kFull, rows_nb);
+    const int nb_off = S.l + 1 < S.L ? 1 : 32 - (S.L - 1);   // from a point to its older neighbour
     int fin = 1;
     double dmax = -CUDART_INF;
-    for (int k = 0; k < k_all; ++k) {
-        const int m = S.l + S.L * k;
-        if (m < H) {
-            const double v = S.level(k);
+    {
+        const double* yp = S.y + S.lane;
+        int k = 0;
+#pragma unroll 2
+        for (; k < full_nb; ++k, yp += 32) {
+            const double v = S.holds(yp) ? *yp : 0.0;
+            const double older = S.holds(yp + nb_off) ? yp[nb_off] : 0.0;
             fin &= finite_d(v) ? 1 : 0;
-            if (m + 1 < H) dmax = fmax(dmax, older_neighbour(S, k) - v);
+            dmax = fmax(dmax, older - v);
+        }
+        for (; k < k_all; ++k, yp += 32) {
+            if (k < rows) {
+                const double v = S.holds(yp) ? *yp : 0.0;
+                fin &= finite_d(v) ? 1 : 0;
+                if (k < rows_nb) dmax = fmax(dmax, (S.holds(yp + nb_off) ? yp[nb_off] : 0.0) - v);
+            }
         }
     }
     fin = group_and(fin, S.L);
@@ -157,29 +175,44 @@ __device__ Normalised normalise_window(const Lanes& S, int H, int k_all, double 
     // the normalised changes feed only the linear extrapolation of short windows (and the export)
     const bool want_changes = usable && (H < min_fit_points || changes_out != nullptr);
     double num = 0.0, den = 0.0;
-    for (int k = 0; k < k_all; ++k) {
-        const int m = S.l + S.L * k;
-        if (want_changes && m + 1 < H) {
-            const double change = __ddiv_rn(older_neighbour(S, k) - S.level(k), M);
-            const double w = S.weight(m);
-            num = fma(w, change, num);
-            den += w;
-            if (changes_out) changes_out[H - 1 - m] = change;
+    if (__any_sync(kFull, want_changes)) {
+        for (int k = 0; k < k_all; ++k) {
+            const int m = S.l + S.L * k;
+            if (want_changes && m + 1 < H) {
+                const double change = __ddiv_rn(older_neighbour(S, k) - S.level(k), M);
+                const double w = S.weight(m);
+                num = fma(w, change, num);
+                den += w;
+                if (changes_out) changes_out[H - 1 - m] = change;
+            }
         }
+        if (changes_out && usable && S.l == 0) changes_out[0] = 0.0;
+        num = group_sum(num, S.L);
+        den = group_sum(den, S.L);
+        out.rho = fmax(num / den, 0.0);
     }
-    if (changes_out && usable && S.l == 0) changes_out[0] = 0.0;
-    num = group_sum(num, S.L);
-    den = group_sum(den, S.L);
-    out.rho = fmax(num / den, 0.0);
     __syncwarp();   // all neighbour reads are done before the window is overwritten
     double lo = CUDART_INF, hi = -CUDART_INF;
-    for (int k = 0; k < k_all; ++k) {
-        const int m = S.l + S.L * k;
-        if (usable && m < H) {
-            const double y = __ddiv_rn(S.level(k), M);
-            if (S.holds(S.y + k * 32 + S.lane)) S.y[k * 32 + S.lane] = y;
+    {
+        // unusable jobs keep their window as it is: they count as lanes without rows
+        const int own = usable ? rows : 0;
+        const int full = __reduce_min_sync(kFull, own);
+        double* yp = S.y + S.lane;
+        int k = 0;
+#pragma unroll 2
+        for (; k < full; ++k, yp += 32) {
+            const double y = __ddiv_rn(S.holds(yp) ? *yp : 0.0, M);
+            if (S.holds(yp)) *yp = y;
             lo = fmin(lo, y);
             hi = fmax(hi, y);
+        }
+        for (; k < k_all; ++k, yp += 32) {
+            if (k < own) {
+                const double y = __ddiv_rn(S.holds(yp) ? *yp : 0.0, M);
+                if (S.holds(yp)) *yp = y;
+                lo = fmin(lo, y);
+                hi = fmax(hi, y);
+            }
         }
     }
     out.ymin = group_min(lo, S.L);
@@ -407,40 +440,74 @@ struct Moments {
 // and log(y - d0) is a line in x (family II: weighted linear regression).  needI / needII: the
 // job wants that family's guess (a family that starts from last epoch's parameters does not);
 // the weight sums in `mom` are always produced.
+struct GuessSums {
+    double sw, swx, swx2, swx3, swx4, swy2, r0, r1, r2, su, sxu;
+};
+
+// One point of the first-guess pass.  kI / kII: the transformed values of family I (1 / (y - d0)) and of
+// family II (log(y - d0)) are wanted by some lane of the warp.
+template <bool kI, bool kII>
+__device__ __forceinline__ void guess_point(const Lanes& S, const double* wp, const double* yp, double md, double inv_span,
+                                            double d0, GuessSums& g) {
+    const double x = -md * inv_span;
+    const double w = S.weight(wp);
+    const double y = S.holds(yp) ? *yp : 0.0;
+    g.sw += w;
+    g.swy2 = fma(w * y, y, g.swy2);
+    if (kI || kII) {
+        const double wx = w * x, wx2 = wx * x;
+        g.swx += wx;
+        g.swx2 += wx2;
+        g.swx3 = fma(wx2, x, g.swx3);
+        g.swx4 = fma(wx2 * x, x, g.swx4);
+    }
+    if (kI) {
+        const double wz = w * fast_rcp(y - d0);
+        g.r2 += wz;
+        g.r1 = fma(wz, x, g.r1);
+        g.r0 = fma(wz * x, x, g.r0);
+    }
+    if (kII) {
+        const double wu = w * log(y - d0);
+        g.su += wu;
+        g.sxu = fma(wu, x, g.sxu);
+    }
+}
+
+// The rows every lane of the warp has without a test per row, the ragged rest with one.
+template <bool kI, bool kII>
+__device__ __forceinline__ void guess_rows(const Lanes& S, int own, int k_all, double inv_span, double d0, GuessSums& g) {
+    const int full = __reduce_min_sync(kFull, own);
+    const double* yp = S.y + S.lane;
+    const double* wp = S.wtab + S.l;
+    double md = (double)S.l;
+    const double dL = (double)S.L;
+    int k = 0;
+#pragma unroll 1
+    for (; k < full; ++k, md += dL, yp += 32, wp += S.L) guess_point<kI, kII>(S, wp, yp, md, inv_span, d0, g);
+#pragma unroll 1
+    for (; k < k_all; ++k, md += dL, yp += 32, wp += S.L)
+        if (k < own) guess_point<kI, kII>(S, wp, yp, md, inv_span, d0, g);
+}
+
 __device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span, double ymin, double ymax, bool busy,
                               bool needI, bool needII, Moments& mom, double (&pI)[4], double (&pII)[4]) {
     const double d0 = ymax > ymin ? ymin - 0.1 * (ymax - ymin) : ymin - 1e-3 * fmax(fabs(ymin), 1.0);
-    double sw = 0, swx = 0, swx2 = 0, swx3 = 0, swx4 = 0, swy2 = 0, r0 = 0, r1 = 0, r2 = 0, su = 0, sxu = 0;
-    double md = (double)S.l;
-    const bool any_guess = needI || needII;
-    for (int k = 0; k < k_all; ++k, md += (double)S.L) {
-        const int m = S.l + S.L * k;
-        if (busy && m < H) {
-            const double x = -md * inv_span;
-            const double w = S.weight(m);
-            const double y = S.level(k);
-            sw += w;
-            swy2 = fma(w * y, y, swy2);
-            if (any_guess) {
-                const double wx = w * x, wx2 = wx * x;
-                swx += wx;
-                swx2 += wx2;
-                swx3 = fma(wx2, x, swx3);
-                swx4 = fma(wx2 * x, x, swx4);
-            }
-            if (needI) {
-                const double wz = w * fast_rcp(y - d0);
-                r2 += wz;
-                r1 = fma(wz, x, r1);
-                r0 = fma(wz * x, x, r0);
-            }
-            if (needII) {
-                const double wu = w * log(y - d0);
-                su += wu;
-                sxu = fma(wu, x, sxu);
-            }
-        }
+    GuessSums g = {};
+    const int shift = __ffs(S.L) - 1;
+    const int own = busy && H - 1 - S.l >= 0 ? ((H - 1 - S.l) >> shift) + 1 : 0;   // the lane's rows
+    // a family that no lane of the warp wants a guess for is left out of the pass; a lane that does not want
+    // what the warp computes gets sums it does not use
+    const bool anyI = __any_sync(kFull, needI), anyII = __any_sync(kFull, needII);
+    if (anyI && anyII) {
+        guess_rows<true, true>(S, own, k_all, inv_span, d0, g);
+    } else {
+        if (anyI) guess_rows<true, false>(S, own, k_all, inv_span, d0, g);
+        else if (anyII) guess_rows<false, true>(S, own, k_all, inv_span, d0, g);
+        else guess_rows<false, false>(S, own, k_all, inv_span, d0, g);
     }
+    double sw = g.sw, swx = g.swx, swx2 = g.swx2, swx3 = g.swx3, swx4 = g.swx4, swy2 = g.swy2;
+    double r0 = g.r0, r1 = g.r1, r2 = g.r2, su = g.su, sxu = g.sxu;
     for (int o = S.L >> 1; o > 0; o >>= 1) {
         sw += __shfl_xor_sync(kFull, sw, o); swx += __shfl_xor_sync(kFull, swx, o);
         swx2 += __shfl_xor_sync(kFull, swx2, o); swx3 += __shfl_xor_sync(kFull, swx3, o);
@@ -460,12 +527,21 @@ __device__ void first_guesses(const Lanes& S, int H, int k_all, double inv_span,
         double sol[4] = {0.0, 0.0, 0.0, 0.0};
         bool good = needI && ldl_solve(B, rhs, sol) && sol[0] >= 0.0 && sol[1] >= 0.0;
         int pos = 1;
-        md = (double)S.l;
-        for (int k = 0; k < k_all; ++k, md += (double)S.L) {
-            const int m = S.l + S.L * k;
-            if (needI && m < H) {
+        {
+            const int mine = needI ? own : 0;
+            const int full = __reduce_min_sync(kFull, mine);
+            const double dL = (double)S.L;
+            double md = (double)S.l;
+            int k = 0;
+            for (; k < full; ++k, md += dL) {
                 const double x = -md * inv_span;
                 pos &= fma(fma(sol[0], x, sol[1]), x, sol[2]) > 0.0 ? 1 : 0;
+            }
+            for (; k < k_all; ++k, md += dL) {
+                if (k < mine) {
+                    const double x = -md * inv_span;
+                    pos &= fma(fma(sol[0], x, sol[1]), x, sol[2]) > 0.0 ? 1 : 0;
+                }
             }
         }
         pos = group_and(pos, S.L);
