@@ -82,6 +82,14 @@ def compare_epoch(gpu_alloc, pred, ref, total_cores, cap, allow_unstable=0, loos
                 unstable=int(bad_jobs.size), alloc_diff=int(diff.size))
 
 
+def tolerance_widths(pred, ref):
+    """Per job the largest |R_gpu(n) - R_cpu(n)| over n in units of the tolerance (1 = at the tolerance); jobs whose
+    winner differs are left out (judged separately by compare_epoch)."""
+    Rg, Rc = np.cumsum(pred["gain"], axis=1), np.cumsum(ref["gain"], axis=1)
+    width = (np.abs(Rg - Rc) / (R_RTOL * np.abs(Rc) + R_ATOL)).max(axis=1)
+    return width[pred["family"] == ref["family"]]
+
+
 def oracle_spread(oracle_mod, wl, j, cap, n_trials=24):
     """How far the oracle's own R(n) of job j moves when its losses are perturbed by 1e-13 relative: per n the
     largest distance from the unperturbed result.  Zero to rounding for a fit that has finished; large where the
