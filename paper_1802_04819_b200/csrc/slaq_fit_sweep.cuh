@@ -104,13 +104,12 @@ struct LaneSums {
 
 // One point of a lane's walk: both families' values at the point and their running sums.
 template <bool kI, bool kII>
-__device__ __forceinline__ void add_point(const Lanes& S, const double* wp, const double* yp, double md, double inv_span,
+__device__ __forceinline__ void add_point(const Lanes& S, const double* wp, const double* yp, double x,
                                           const double (&pI)[4], const double (&pII)[4], double& e, double ratio,
                                           LaneSums& a) {
     const double w = S.weight(wp);
     const double y = S.holds(yp) ? *yp : 0.0;
     if (kI) {
-        const double x = -md * inv_span;
         const double q = fma(fma(pI[0], x, pI[1]), x, pI[2]);
         a.q_signs |= __double2hiint(q);   // q = 0 or NaN makes the sums non-finite, which the caller sees
         const double inv = fast_rcp(q);
@@ -143,8 +142,12 @@ template <bool kI, bool kII>
 __device__ __forceinline__ void walk_rows(const Lanes& S, int k_last, int k_all, double inv_span,
                                           const double (&pI)[4], const double (&pII)[4], LaneSums& a) {
     const int mi = S.l + k_last * S.L;
-    double md = (double)mi;
+    const double md = (double)mi;
     const double dL = (double)S.L;
+    // x from the lane's oldest point by one addition per row (its rounding, at most a few 1e-15 absolute at the
+    // newest point, moves the predictions as little as the exponential's recurrence does: measured)
+    double x = -md * inv_span;
+    const double hx = dL * inv_span;
     // e = exp(alpha - beta x) with x = -m / span falls geometrically towards the newest point: one
     // exact value at the lane's oldest point, then a constant ratio per step.  (Choosing the start such
     // that the recurrence lands on the exact value at the newest point was measured: the predictions stay
@@ -159,10 +162,10 @@ __device__ __forceinline__ void walk_rows(const Lanes& S, int k_last, int k_all,
     const int k_min = __reduce_min_sync(kFull, k_last);
     int i = 0;
 #pragma unroll 1   // unrolling was measured (2 rows per step): slower, more spills
-    for (; i <= k_min; ++i, md -= dL, yp -= 32, wp -= S.L) add_point<kI, kII>(S, wp, yp, md, inv_span, pI, pII, e, ratio, a);
+    for (; i <= k_min; ++i, x += hx, yp -= 32, wp -= S.L) add_point<kI, kII>(S, wp, yp, x, pI, pII, e, ratio, a);
 #pragma unroll 1
-    for (; i < k_all; ++i, md -= dL, yp -= 32, wp -= S.L)
-        if (i <= k_last) add_point<kI, kII>(S, wp, yp, md, inv_span, pI, pII, e, ratio, a);   // row k_last - i >= 0
+    for (; i < k_all; ++i, x += hx, yp -= 32, wp -= S.L)
+        if (i <= k_last) add_point<kI, kII>(S, wp, yp, x, pI, pII, e, ratio, a);   // row k_last - i >= 0
 }
 
 // One sweep over the window: both families at once, each at its own point.  A lane adds up
