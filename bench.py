@@ -34,16 +34,16 @@ WARM_TRIALS = 5   # trials per epoch of the warm-started loop reported beside th
 # algorithmic fp64 work of the fit, per stored point: one sweep of family I, one of family II, set-up
 FLOP_SWEEP_I, FLOP_SWEEP_II, FLOP_SETUP = 40.0, 25.0, 40.0
 FP64_LANES_PER_SM = 64          # fp64 FMA lanes per SM on B200
-# The sweep of the fit issues 44 fp64 arithmetic instructions per point for its 65 algorithmic flop: 88 cycles per
-# warp row of 32 points and sub-partition at the pipe's 2 cycles per instruction, 92 with the 4 fused multiply-adds on
+# The sweep of the fit issues 43 fp64 arithmetic instructions per point for its 65 algorithmic flop: 86 cycles per
+# warp row of 32 points and sub-partition at the pipe's 2 cycles per instruction, 90 with the 4 fused multiply-adds on
 # three different registers, which take 3 (measured with bench_probes/fp64_issue_probe)
-SWEEP_FLOP_PER_POINT, SWEEP_ISSUE_CYCLES_PER_ROW = FLOP_SWEEP_I + FLOP_SWEEP_II, 92.0
+SWEEP_FLOP_PER_POINT, SWEEP_ISSUE_CYCLES_PER_ROW = FLOP_SWEEP_I + FLOP_SWEEP_II, 90.0
 SUBPARTITIONS_PER_SM = 4
 MIN_TIMED_SECONDS = 1.0   # the block of --steps steps is repeated until the timed region is at least this long
 # DRAM bytes per stored loss moved by the fit kernel (ncu: dram__bytes_read.sum + dram__bytes_write.sum =
-# 166.13 MB + 13.01 MB on a 20,068,408-loss cut of this workload, profiles/fit_kernel_40k_jobs.md; traffic grows
+# 166.16 MB + 13.31 MB on a 20,068,408-loss cut of this workload, profiles/fit_kernel_40k_jobs.md; traffic grows
 # with the stored losses)
-NCU_FIT_DRAM_BYTES_PER_LOSS = (166.13e6 + 13.01e6) / 20_068_408
+NCU_FIT_DRAM_BYTES_PER_LOSS = (166.16e6 + 13.31e6) / 20_068_408
 
 
 from paper_1802_04819_b200.partition import max_over_ranks, partition_seed_offset, rank_info, whole_job_rate  # noqa: E402
@@ -397,7 +397,7 @@ def run_gpu(args):
                          "algorithmic_flops_per_launch": fit_flops, "ms_per_launch": fit_ms_avg,
                          "issue_bound_peak": issue_bound, "frac_of_issue_bound": achieved / issue_bound,
                          "issue_bound_note": "a loop of nothing but the fit's sweeps at the measured issue rates: 65 flop "
-                                             "per point on 44 fp64 instructions, 92 cycles per warp row of 32 points",
+                                             "per point on 43 fp64 instructions, 90 cycles per warp row of 32 points",
                          "peak_is": f"{sm_count} SMs x {FP64_LANES_PER_SM} fp64 FMA lanes x 2 x {sm_max:.0f} MHz "
                                     f"(clock from MEASURED_PEAKS.json: {peak_kind}; that file holds no fp64 figure)",
                          "peak_measured": fp64_peak_measured,

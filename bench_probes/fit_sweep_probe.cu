@@ -7,7 +7,7 @@
 // with clock64() around it, divided by (rows x sweeps x warps per sub-partition) give the cycles
 // one sub-partition spends per warp row of 32 points when the fp64 pipe sees nothing but sweeps.
 // Printed per (lanes per job L, rows per lane): cycles per warp row, and the same as a
-// fraction of the 2-cycle issue rate of the variant's fp64 instructions (44 per point in the library's sweep).
+// fraction of the 2-cycle issue rate of the variant's fp64 instructions (43 per point in the library's sweep).
 //
 //   fit_sweep_probe [n_sweeps]
 #include <algorithm>
@@ -123,7 +123,7 @@ __device__ __forceinline__ void sweep_tables(const slaq::Lanes& S, int ts, int f
 
 // A second alternative, the library's sweep until the running sums replaced it: the powers of x multiplied out
 // point by point (x, x^2 and w u^2 x^2 formed in the loop, 13 of the 22 accumulations fused multiply-adds on three
-// different registers): 46 fp64 instructions per point instead of 44, 19 fused multiply-adds instead of 8.
+// different registers): 46 fp64 instructions per point instead of 43, 19 fused multiply-adds instead of 8.
 __device__ __forceinline__ void sweep_products(const slaq::Lanes& S, int fam, int H, int k_all, double inv_span,
                                                const double (&pI)[4], bool doI, const double (&pII)[4], bool doII,
                                                slaq::SweepSums& out) {
@@ -307,7 +307,7 @@ int main(int argc, char** argv) {
     std::vector<double> last_lib(5 * 32 * 13, 0.0), last(32 * 13);
     const char* const names[3] = {"the library's sweep (powers of x by running sums)", "weighted powers from tables",
                                   "powers of x multiplied in the loop"};
-    const double kInstr[3] = {44.0, 41.0, 46.0};   // fp64 arithmetic instructions per point in the loop, from the source
+    const double kInstr[3] = {43.0, 41.0, 46.0};   // fp64 arithmetic instructions per point in the loop, from the source
     for (int variant = 0; variant < 3; ++variant) {
         // the tables take 4 x kTable doubles more of the SM's shared memory: the sixteen slices shrink accordingly
         const int slice_doubles = variant != 1 ? kSliceDoubles : (kSliceDoubles * kWarps - 4 * kTable) / kWarps / 32 * 32;

@@ -23,4 +23,6 @@ def test_running_sums_equal_the_multiplied_out_sums():
                          text=True, timeout=300).stdout
     worst = [float(x) for x in re.findall(r"largest relative difference of a sum from the library's sweep: (\S+)", out)]
     assert len(worst) == 5, out            # one per lanes-per-job setting (2, 4, 8, 16, 32)
-    assert max(worst) < 1e-13, worst       # measured: 6e-16 to 8e-15
+    # measured: 6e-16 to 6e-14 (the library steps x by one addition per row, the other form multiplies the running
+    # index out, so the two evaluate the model a few 1e-15 apart in x); a wrong coefficient shows as 1e-3 or more
+    assert max(worst) < 1e-11, worst
