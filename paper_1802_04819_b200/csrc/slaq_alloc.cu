@@ -118,18 +118,29 @@ select_pass_kernel(const double* __restrict__ gain, const int32_t* __restrict__ 
             const int j = j0 + r;
             const int lo = __shfl_sync(kFull, my_lo, r), hi = __shfl_sync(kFull, my_hi, r);
             int above = 0, same = 0;
-            for (int base = lo; base < hi; base += 32) {
-                const int i = base + lane;
-                const bool in = i < hi;
-                unsigned long long key = 0;
-                if (in && index_ok((long long)j * cap + i, (long long)max_jobs * cap, kErrGain, err_word))
-                    key = keys[(size_t)j * cap + i];
+            auto take = [&](unsigned long long key, bool in) {
                 const unsigned d_prev = (unsigned)(key >> prev_shift) & ((1u << prev_bits) - 1u);
                 const bool match = in && d_prev == prev_bin;
                 above += __popc(__ballot_sync(kFull, in && d_prev > prev_bin));
                 same += __popc(__ballot_sync(kFull, match));
                 const unsigned bin = (unsigned)(key >> shift) & ((1u << bits) - 1u);
                 if (match && index_ok(bin, kRadixBins, kErrBin, err_word)) atomicAdd(&sh_hist[bin], 1u);
+            };
+            auto fetch = [&](int i) -> unsigned long long {
+                return (i < hi && index_ok((long long)j * cap + i, (long long)max_jobs * cap, kErrGain, err_word))
+                           ? keys[(size_t)j * cap + i] : 0ull;
+            };
+            if (hi - lo <= 128) {
+                // a segment of up to four chunks (a whole row of the first table-wide pass): all its loads are
+                // issued before the first is used, so that a warp keeps four of them in flight instead of one
+                unsigned long long k4[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) k4[c] = fetch(lo + 32 * c + lane);
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (lo + 32 * c < hi) take(k4[c], lo + 32 * c + lane < hi);
+            } else {
+                for (int base = lo; base < hi; base += 32) take(fetch(base + lane), base + lane < hi);
             }
             if (lane == r) {
                 my_lo = lo + above;
