@@ -314,7 +314,6 @@ finalise_kernel(const double* __restrict__ gain, const int32_t* __restrict__ cou
                 long long ties_before, const long long* __restrict__ d_ties_before, int32_t* err_word) {
     __shared__ long long sh_pre[kJobsPerBlock];
     if (d_ties_before) ties_before += *d_ties_before;   // the count held by lower shards, left on the device by the caller
-    __shared__ int sh_alloc[kJobsPerBlock];
     const int t = threadIdx.x;
     const int j0 = blockIdx.x * kJobsPerBlock;
     const int jt = j0 + t;
@@ -343,7 +342,6 @@ finalise_kernel(const double* __restrict__ gain, const int32_t* __restrict__ cou
         }
 #endif
     }
-    sh_alloc[t] = a;
     if (jt < max_jobs) {
         alloc[jt] = a;
         if (out_alloc) out_alloc[jt] = a;
@@ -361,13 +359,22 @@ finalise_kernel(const double* __restrict__ gain, const int32_t* __restrict__ cou
         atomicAdd((unsigned long long*)&counters[6], (unsigned long long)(sh_pre[0] >> 20));
         atomicAdd((unsigned long long*)&counters[7], (unsigned long long)(sh_pre[0] & ((1ll << 20) - 1)));
     }
-    // predicted reduction at the allocation: the job's first a_j gains, one warp per job
+    // predicted reduction at the allocation: the job's first a_j gains.  Most jobs get a few cores: their own thread
+    // adds them in order (all threads of the block load at once); a row with more than 32 is left to its warp.
     const int warp = t >> 5, lane = t & 31;
-    for (int i = 0; i < 32; ++i) {
-        const int local = warp * 32 + i;
-        const int j = j0 + local;
-        if (j >= max_jobs) break;
-        const int aj = sh_alloc[local];
+    const bool mine = jt < max_jobs;
+    if (mine && a <= 32) {
+        double R = 0.0;
+        const double* row = gain + (size_t)jt * cap;
+        for (int n = 0; n < a; ++n) R += row[n];
+        reduction[jt] = R;
+    }
+    unsigned big = __ballot_sync(kFull, mine && a > 32);
+    while (big) {
+        const int r = __ffs(big) - 1;
+        big &= big - 1;
+        const int j = j0 + warp * 32 + r;
+        const int aj = __shfl_sync(kFull, a, r);
         double R = 0.0;
         for (int n = lane; n < aj; n += 32) R += gain[(size_t)j * cap + n];
 #pragma unroll
